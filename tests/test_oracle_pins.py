@@ -1,0 +1,236 @@
+"""Pins for the fp64 oracle: properties the paper and the mathematics fix, each computed here
+independently of the oracle's own loop (no formula of the oracle is re-typed as the check)."""
+import numpy as np
+import pytest
+
+import oracle
+from oracle.chunkwise import forward_chunkwise
+
+RNG = np.random.default_rng
+
+
+def _rand_problem(rng, B=1, T=12, H=2, d_k=5, d_v=3, eta=None, la=None):
+    q = rng.standard_normal((B, T, H, d_k))
+    k = rng.standard_normal((B, T, H, d_k))
+    v = rng.standard_normal((B, T, H, d_v))
+    eta = 1.0 / (1.0 + np.exp(-rng.standard_normal((B, T, H)))) if eta is None else np.full((B, T, H), eta)
+    la = -np.log1p(np.exp(rng.standard_normal((B, T, H)))) if la is None else np.full((B, T, H), la)
+    s0 = 0.3 * rng.standard_normal((B, H, d_k, d_v))
+    return q, k, v, la, eta, s0
+
+
+def _states_after_each_token(q, k, v, la, eta, eps, s0):
+    """All intermediate states, obtained by calling the oracle on prefixes (state hand-off is
+    pinned separately below, so prefixes are run from the original initial state)."""
+    B, T, H, d_k = q.shape
+    states = []
+    for t in range(1, T + 1):
+        _, fin, _ = oracle.forward(q[:, :t], k[:, :t], v[:, :t], la[:, :t], eta[:, :t], eps, s0)
+        states.append(fin)
+    return states
+
+
+def test_p1_kaczmarz_projection_theorem1():
+    # eta = 1, eps = 0, any decay: after the write, the state reproduces v_t on key k_t exactly.
+    rng = RNG(1)
+    q, k, v, la, eta, s0 = _rand_problem(rng, eta=1.0)
+    states = _states_after_each_token(q, k, v, la, eta, 0.0, s0)
+    for t, S in enumerate(states):
+        pred = np.einsum("bhkv,bhk->bhv", S, k[:, t])
+        np.testing.assert_allclose(pred, v[:, t], rtol=0, atol=1e-12)
+
+
+def test_p2_residual_contraction_eq5():
+    rng = RNG(2)
+    q, k, v, la, eta, s0 = _rand_problem(rng)
+    eps = 0.37
+    states = _states_after_each_token(q, k, v, la, eta, eps, s0)
+    prev = s0
+    for t, S in enumerate(states):
+        alpha = np.exp(la[:, t])[..., None, None]
+        e_before = v[:, t] - np.einsum("bhkv,bhk->bhv", alpha * prev, k[:, t])
+        e_after = v[:, t] - np.einsum("bhkv,bhk->bhv", S, k[:, t])
+        nk = np.sum(k[:, t] ** 2, axis=-1)
+        factor = 1.0 - eta[:, t] * nk / (nk + eps)
+        np.testing.assert_allclose(e_after, factor[..., None] * e_before, rtol=0, atol=1e-12)
+        prev = S
+
+
+def test_p3_proximal_stationarity_prop1():
+    # S_t is the stationary point of 1/2||S - S~||^2 + mu/2 ||S^T k - v||^2, mu = eta/((1-eta)||k||^2+eps).
+    rng = RNG(3)
+    q, k, v, la, eta, s0 = _rand_problem(rng, T=6)
+    eps = 0.05
+    states = _states_after_each_token(q, k, v, la, eta, eps, s0)
+    prev = s0
+    for t, S in enumerate(states):
+        St = np.exp(la[:, t])[..., None, None] * prev
+        nk = np.sum(k[:, t] ** 2, axis=-1)
+        mu = eta[:, t] / ((1.0 - eta[:, t]) * nk + eps)
+        resid = np.einsum("bhkv,bhk->bhv", S, k[:, t]) - v[:, t]
+        grad = S - St + mu[..., None, None] * np.einsum("bhk,bhv->bhkv", k[:, t], resid)
+        assert np.abs(grad).max() < 1e-12
+        prev = S
+
+
+def test_p4_minimum_norm_change():
+    # eta=1, eps=0: S_t - S~ is Frobenius-orthogonal to every H with H^T k = 0 (orthogonal projection).
+    rng = RNG(4)
+    q, k, v, la, eta, s0 = _rand_problem(rng, T=4, eta=1.0)
+    states = _states_after_each_token(q, k, v, la, eta, 0.0, s0)
+    prev = s0
+    for t, S in enumerate(states):
+        delta = S - np.exp(la[:, t])[..., None, None] * prev
+        for _ in range(5):
+            Hm = rng.standard_normal(delta.shape)
+            kk = k[:, t]
+            # project rows so that H^T k = 0
+            Hm = Hm - np.einsum("bhk,bhv->bhkv", kk, np.einsum("bhkv,bhk->bhv", Hm, kk)) / np.sum(kk * kk, -1)[..., None, None]
+            assert np.abs(np.einsum("bhkv,bhk->bhv", Hm, kk)).max() < 1e-12
+            assert abs(np.sum(delta * Hm)) < 1e-11
+        prev = S
+
+
+def test_p5_pure_decay_when_eta_zero():
+    rng = RNG(5)
+    q, k, v, la, eta, s0 = _rand_problem(rng, eta=0.0)
+    out, fin, _ = oracle.forward(q, k, v, la, eta, 1e-6, s0)
+    gamma = np.exp(np.cumsum(la, axis=1))                      # [B, T, H]
+    expect = gamma[..., None] * np.einsum("bhkv,bthk->bthv", s0, q)
+    np.testing.assert_allclose(out, expect, rtol=0, atol=1e-13)
+    np.testing.assert_allclose(fin, gamma[:, -1][..., None, None] * s0, rtol=0, atol=1e-13)
+
+
+@pytest.mark.parametrize("chunk", [1, 2, 3, 5, 16, 64, 100])
+def test_p6_chunkwise_equals_tokenwise(chunk):
+    rng = RNG(6)
+    q, k, v, la, eta, s0 = _rand_problem(rng, B=2, T=37, H=2, d_k=6, d_v=4)
+    out, fin, _ = oracle.forward(q, k, v, la, eta, 1e-3, s0)
+    out_c, fin_c = forward_chunkwise(q, k, v, la, eta, 1e-3, chunk, s0)
+    np.testing.assert_allclose(out_c, out, rtol=0, atol=1e-11)
+    np.testing.assert_allclose(fin_c, fin, rtol=0, atol=1e-11)
+
+
+def test_p7_brute_force_unrolled_products_table7():
+    # o_t = sum_{j<=t} beta_j (q_t^T [prod_{s=j+1..t} alpha_s (I - beta_s k_s k_s^T)] k_j) v_j
+    #       + q_t^T [prod_{s=1..t} alpha_s (I - beta_s k_s k_s^T)] S_0     (explicit d_k x d_k matrices)
+    rng = RNG(7)
+    T, d_k, d_v = 8, 4, 3
+    q, k, v, la, eta, s0 = _rand_problem(rng, B=1, T=T, H=1, d_k=d_k, d_v=d_v)
+    eps = 0.01
+    out, fin, _ = oracle.forward(q, k, v, la, eta, eps, s0)
+    kk, qq, vv = k[0, :, 0], q[0, :, 0], v[0, :, 0]
+    beta = eta[0, :, 0] / (np.sum(kk * kk, axis=1) + eps)
+    alpha = np.exp(la[0, :, 0])
+    Ms = [alpha[s] * (np.eye(d_k) - beta[s] * np.outer(kk[s], kk[s])) for s in range(T)]
+    for t in range(T):
+        acc = np.zeros(d_v)
+        for j in range(t + 1):
+            P = np.eye(d_k)
+            for s in range(j + 1, t + 1):      # later factors applied later: M_t ... M_{j+1}
+                P = Ms[s] @ P
+            acc += beta[j] * (qq[t] @ P @ kk[j]) * vv[j]
+        P = np.eye(d_k)
+        for s in range(0, t + 1):
+            P = Ms[s] @ P
+        acc += qq[t] @ P @ s0[0, 0]
+        np.testing.assert_allclose(out[0, t, 0], acc, rtol=0, atol=1e-12)
+    # final state in the same unrolled form
+    S = np.zeros((d_k, d_v))
+    for j in range(T):
+        P = np.eye(d_k)
+        for s in range(j + 1, T):
+            P = Ms[s] @ P
+        S += beta[j] * np.outer(P @ kk[j], vv[j])
+    P = np.eye(d_k)
+    for s in range(T):
+        P = Ms[s] @ P
+    S += P @ s0[0, 0]
+    np.testing.assert_allclose(fin[0, 0], S, rtol=0, atol=1e-12)
+
+
+def test_p8_reduces_to_causal_linear_attention_on_orthonormal_keys():
+    rng = RNG(8)
+    d_k, d_v, T = 8, 5, 8
+    Qm, _ = np.linalg.qr(rng.standard_normal((d_k, d_k)))
+    k = Qm[:T][None, :, None, :]                                 # orthonormal rows
+    q = rng.standard_normal((1, T, 1, d_k))
+    v = rng.standard_normal((1, T, 1, d_v))
+    la = np.zeros((1, T, 1))
+    eta = np.ones((1, T, 1))
+    out, fin, _ = oracle.forward(q, k, v, la, eta, 0.0, None)
+    scores = np.tril(q[0, :, 0] @ k[0, :, 0].T)                  # causal mask
+    np.testing.assert_allclose(out[0, :, 0], scores @ v[0, :, 0], rtol=0, atol=1e-12)
+    np.testing.assert_allclose(fin[0, 0], k[0, :, 0].T @ v[0, :, 0], rtol=0, atol=1e-12)
+
+
+def test_p9_row_scaling_invariance_at_eps_zero():
+    rng = RNG(9)
+    q, k, v, la, eta, s0 = _rand_problem(rng)
+    c = np.exp(rng.standard_normal(k.shape[:3]))[..., None]
+    out1, fin1, _ = oracle.forward(q, k, v, la, eta, 0.0, s0)
+    out2, fin2, _ = oracle.forward(q, c * k, c * v, la, eta, 0.0, s0)
+    np.testing.assert_allclose(out2, out1, rtol=0, atol=1e-11)
+    np.testing.assert_allclose(fin2, fin1, rtol=0, atol=1e-11)
+
+
+def test_p10_state_handoff_and_decode_equals_forward():
+    rng = RNG(10)
+    q, k, v, la, eta, s0 = _rand_problem(rng, B=2, T=20)
+    eps = 1e-4
+    out, fin, _ = oracle.forward(q, k, v, la, eta, eps, s0)
+    o1, f1, _ = oracle.forward(q[:, :7], k[:, :7], v[:, :7], la[:, :7], eta[:, :7], eps, s0)
+    o2, f2, _ = oracle.forward(q[:, 7:], k[:, 7:], v[:, 7:], la[:, 7:], eta[:, 7:], eps, f1)
+    np.testing.assert_allclose(np.concatenate([o1, o2], 1), out, rtol=0, atol=1e-13)
+    np.testing.assert_allclose(f2, fin, rtol=0, atol=1e-13)
+    st = np.array(s0, dtype=np.float64)
+    for t in range(q.shape[1]):
+        o = oracle.decode_step(q[:, t], k[:, t], v[:, t], la[:, t], eta[:, t], eps, st)
+        np.testing.assert_allclose(o, out[:, t], rtol=0, atol=1e-13)
+    np.testing.assert_allclose(st, fin, rtol=0, atol=1e-13)
+
+
+def test_init_state_is_decayed_by_first_alpha_and_readout_is_post_write():
+    # One token, hand-computed: distinguishes "decay before write", "read after write",
+    # a transposed state, and eps placement.
+    k = np.array([[[[2.0, 0.0]]]])
+    q = np.array([[[[1.0, 1.0]]]])
+    v = np.array([[[[3.0]]]])
+    s0 = np.array([[[[1.0], [5.0]]]])          # d_k = 2, d_v = 1
+    la = np.log(np.array([[[0.5]]]))
+    eta = np.array([[[0.5]]])
+    eps = 1.0
+    out, fin, _ = oracle.forward(q, k, v, la, eta, eps, s0)
+    # S~ = [0.5, 2.5]; e = 3 - 2*0.5 = 2; beta = 0.5/(4+1) = 0.1; S = [0.5 + 0.1*2*2, 2.5] = [0.9, 2.5]
+    np.testing.assert_allclose(fin[0, 0, :, 0], [0.9, 2.5], atol=1e-15)
+    np.testing.assert_allclose(out[0, 0, 0, 0], 3.4, atol=1e-15)
+
+
+def test_packed_equals_per_sequence_and_zero_length():
+    rng = RNG(11)
+    H, d_k, d_v = 2, 4, 3
+    lens = [3, 0, 5, 1]
+    cu = np.concatenate([[0], np.cumsum(lens)])
+    n_tok = int(cu[-1])
+    q = rng.standard_normal((n_tok, H, d_k)); k = rng.standard_normal((n_tok, H, d_k))
+    v = rng.standard_normal((n_tok, H, d_v))
+    la = -np.abs(rng.standard_normal((n_tok, H))); eta = rng.uniform(0, 1, (n_tok, H))
+    s0 = rng.standard_normal((len(lens), H, d_k, d_v))
+    out, fin, _ = oracle.forward_packed(q, k, v, la, eta, 1e-6, cu, s0)
+    for n, L in enumerate(lens):
+        a, b = cu[n], cu[n + 1]
+        if L == 0:
+            np.testing.assert_array_equal(fin[n], s0[n])
+            continue
+        o, f, _ = oracle.forward(q[None, a:b], k[None, a:b], v[None, a:b], la[None, a:b], eta[None, a:b], 1e-6, s0[n:n + 1])
+        np.testing.assert_array_equal(out[a:b], o[0])
+        np.testing.assert_array_equal(fin[n], f[0])
+
+
+def test_zero_key_with_eps_is_pure_decay_and_zero_eps_is_nan():
+    q = np.ones((1, 1, 1, 2)); k = np.zeros((1, 1, 1, 2)); v = np.ones((1, 1, 1, 2))
+    s0 = np.ones((1, 1, 2, 2)); la = np.log(np.full((1, 1, 1), 0.25)); eta = np.ones((1, 1, 1))
+    out, fin, _ = oracle.forward(q, k, v, la, eta, 1e-6, s0)
+    np.testing.assert_allclose(fin, 0.25 * s0, atol=1e-15)
+    out, fin, _ = oracle.forward(q, k, v, la, eta, 0.0, s0)
+    assert np.isnan(fin).all()

@@ -1,0 +1,384 @@
+#!/usr/bin/env python
+"""Benchmark of the KLA hot path on B200.
+
+A "step" is one chunkwise forward (prologue + UT/WY transform + inter-chunk scan, one kernel
+launch) over one batch of the headline workload: bf16, B=8, H=8, T=4096, d_k=d_v=128, chunk=64,
+synthetic inputs with the value distributions of the 0.4B-layer recipe.  The metric is
+chunk-forward throughput in Mtok/s (one token = one position of one sequence, all heads).
+With N GPUs every rank processes its own batch (independent sequences, no collective on the data
+path): weak scaling, value = N * tokens / max-over-ranks time.
+
+Reported beside it, from the same run: the decode step (B=64, H=8, d=128, 1024 consecutive steps),
+the long-context and varlen workloads, an end-to-end figure with host buffers, the roofline
+fraction of the chunk kernel, and the fp64 oracle timed on the host cores (a baseline, not the
+target).  `--impl reference` times only that oracle.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "chunk_fwd_throughput"
+UNIT = "Mtok/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            with open(path) as f:
+                pk = json.load(f)
+            return pk, "measured"
+        except Exception:
+            pass
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+# ---- workload accounting (algorithmic bytes / flops per token-head) -----------------------------------
+def algorithmic_bytes(n_tok, H, d, n_seq, io_bytes, out_bytes, has_init, want_final):
+    """q, k, v read + out written + the two fp32 gates, plus the states that are read/written."""
+    per_token_head = d * io_bytes * 3 + d * out_bytes + 8
+    state = n_seq * H * d * d * 4
+    return n_tok * H * per_token_head + (state if has_init else 0) + (state if want_final else 0)
+
+
+def algorithmic_flops(n_tok, H, d, C=64):
+    """Causal-half count of Algorithm 1 (right): K K^T, K S0, T.rhs, Q S0, Q K^T, (A o QK^T) U, K^T D U, solve."""
+    per_token_head = 2 * C * (d + d) + 6 * d * d + C * C / 3.0
+    return n_tok * H * per_token_head
+
+
+# ---- clocks sampling ------------------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.samples = []
+        self._stop = threading.Event()
+        self._thr = None
+
+    def _run(self):
+        while not self._stop.is_set():
+            try:
+                out = subprocess.run(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
+                                      "--format=csv,noheader,nounits"], capture_output=True, text=True, timeout=5).stdout
+                parts = [x.strip() for x in out.strip().split(",")]
+                if len(parts) >= 7:
+                    self.samples.append(parts)
+            except Exception:
+                pass
+            self._stop.wait(0.1)
+
+    def __enter__(self):
+        self._thr = threading.Thread(target=self._run, daemon=True)
+        self._thr.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        self._thr.join(timeout=10)
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for s in self.samples:
+            try:
+                sm.append(float(s[0]))
+                mx.append(float(s[1]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, s[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ---- the oracle leg (CPU baseline / reference arm) ---------------------------------------------------------
+def oracle_sample_run(seed=1, B=2, H=8, T=4096, d=128, repeats=1):
+    """Time the fp64 oracle, as it stands, on a bounded sample of the headline workload:
+    B sequences (of the workload's 8) x all heads x all T tokens.  Returns (Mtok/s, threads, seconds)."""
+    import oracle
+    from paper_2605_08587_b200 import workloads as W
+    w = W.config2(B=B, H=H, T=T, d=d, seed=seed)
+    args = [a.float().numpy() for a in (w.q, w.k, w.v)] + [w.log_alpha.numpy(), w.eta.numpy()]
+    best, thr = None, 1
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        _, _, thr = oracle.forward(*args, w.eps)
+        dt = time.perf_counter() - t0
+        best = dt if best is None else min(best, dt)
+    return B * T / best / 1e6, thr, best
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    sample = dict(B=1, H=8, T=4096, d=128)
+    for _ in range(args.warmup):
+        oracle_sample_run(**sample)
+    times, thr = [], 1
+    for _ in range(args.steps):
+        v, thr, dt = oracle_sample_run(**sample)
+        times.append(dt)
+    ms = 1e3 * sum(times) / len(times)
+    value = sample["B"] * sample["T"] / (ms / 1e3) / 1e6
+    desc = "%d of 8 sequences x 8 heads x 4096 tokens of the headline workload per step" % sample["B"]
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": "cfg2_bf16_B8_H8_T4096_d128_chunk64", "sampled": desc},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": thr, "kind": "oracle", "sample": desc},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ---- GPU legs ----------------------------------------------------------------------------------------------------
+def time_launches(fn, steps, warmup, stream):
+    """Average device time per call of fn() in ms: CUDA events on the launching stream."""
+    import torch
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    e0 = torch.cuda.Event(enable_timing=True)
+    e1 = torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(steps):
+        fn()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / steps
+
+
+def to_dev(w, dev):
+    return dict(q=w.q.to(dev), k=w.k.to(dev), v=w.v.to(dev), log_alpha=w.log_alpha.to(dev), eta=w.eta.to(dev),
+                init_state=None if w.init_state is None else w.init_state.to(dev),
+                cu_seqlens=None if w.cu_seqlens is None else w.cu_seqlens.to(dev), host_seqlens=w.cu_seqlens)
+
+
+def chunk_leg(w, dev, steps, warmup, peaks, out_dtype):
+    """Time one chunk-forward workload; returns a dict of figures."""
+    import torch
+    from paper_2605_08587_b200 import kla_chunk_fwd
+    t = to_dev(w, dev)
+    B, T, H, d = w.q.shape
+    n_seq = w.n_seq
+    out = torch.empty((B, T, H, d), device=dev, dtype=out_dtype)
+    fin = torch.empty((n_seq, H, d, d), device=dev, dtype=torch.float32)
+
+    def step():
+        kla_chunk_fwd(t["q"], t["k"], t["v"], t["log_alpha"], t["eta"], w.eps, chunk=w.chunk,
+                      init_state=t["init_state"], out=out, final_state=fin, cu_seqlens=t["cu_seqlens"],
+                      host_seqlens=t["host_seqlens"])
+
+    ms = time_launches(step, steps, warmup, torch.cuda.current_stream())
+    nbytes = algorithmic_bytes(B * T, H, d, n_seq, w.q.element_size(), out.element_size(), w.init_state is not None, True)
+    flops = algorithmic_flops(B * T, H, d, w.chunk)
+    gbs = nbytes / (ms * 1e-3) / 1e9
+    tfs = flops / (ms * 1e-3) / 1e12
+    t_hbm = nbytes / (peaks["hbm_gbs"] * 1e9)
+    t_tc = flops / (peaks["bf16_tflops"] * 1e12)
+    return {"workload": w.name, "ms": ms, "mtok_per_s": B * T / (ms * 1e-3) / 1e6, "tokens": B * T,
+            "algorithmic_bytes": nbytes, "algorithmic_flops": flops, "achieved_gbs": gbs, "achieved_tflops": tfs,
+            "roofline_ms": 1e3 * max(t_hbm, t_tc), "roofline_frac": max(t_hbm, t_tc) / (ms * 1e-3),
+            "bound": "hbm" if t_hbm >= t_tc else "tensor"}
+
+
+def decode_leg(dev, steps_per_call, calls, warmup, peaks, B=64, H=8, d=128, l2_defeat=False):
+    import torch
+    from paper_2605_08587_b200 import kla_decode_steps, workloads as W
+    w = W.config4(B=B, H=H, d=d, steps=steps_per_call)
+    args = [a.to(dev) for a in (w.q, w.k, w.v, w.log_alpha, w.eta)]
+    st = w.state.to(dev).clone()
+    out = torch.empty((steps_per_call, B, H, d), device=dev, dtype=torch.bfloat16)
+
+    def step():
+        kla_decode_steps(*args, w.eps, st, out=out)
+
+    ms = time_launches(step, calls, warmup, torch.cuda.current_stream()) / steps_per_call
+    state_bytes = 2 * B * H * d * d * 4
+    vec_bytes = B * H * (3 * d * 2 + d * 2 + 8)
+    nbytes = state_bytes + vec_bytes
+    gbs = nbytes / (ms * 1e-3) / 1e9
+    return {"workload": w.name, "us_per_step": ms * 1e3, "tok_per_s": B / (ms * 1e-3), "bytes_per_step": nbytes,
+            "effective_gbs": gbs, "frac_of_hbm_peak": gbs / peaks["hbm_gbs"],
+            "state_mb": state_bytes / 2 / 1e6, "state_fits_l2": state_bytes / 2 < 126e6}
+
+
+def e2e_leg(w, dev, steps, warmup):
+    """Same step, host buffers: pinned host -> device copies of every input, the launch, and the
+    device -> host read of out and final state, all inside the timed region."""
+    import torch
+    from paper_2605_08587_b200 import kla_chunk_fwd
+    host = {k: getattr(w, k).pin_memory() for k in ("q", "k", "v", "log_alpha", "eta")}
+    B, T, H, d = w.q.shape
+    devbuf = {k: torch.empty_like(v, device=dev) for k, v in host.items()}
+    out = torch.empty((B, T, H, d), device=dev, dtype=torch.bfloat16)
+    fin = torch.empty((w.n_seq, H, d, d), device=dev, dtype=torch.float32)
+    out_h = torch.empty(out.shape, dtype=out.dtype).pin_memory()
+    fin_h = torch.empty(fin.shape, dtype=fin.dtype).pin_memory()
+    h2d = sum(v.numel() * v.element_size() for v in host.values())
+    d2h = out.numel() * out.element_size() + fin.numel() * fin.element_size()
+
+    def step():
+        for k in host:
+            devbuf[k].copy_(host[k], non_blocking=True)
+        kla_chunk_fwd(devbuf["q"], devbuf["k"], devbuf["v"], devbuf["log_alpha"], devbuf["eta"], w.eps,
+                      chunk=w.chunk, out=out, final_state=fin)
+        out_h.copy_(out, non_blocking=True)
+        fin_h.copy_(fin, non_blocking=True)
+
+    ms = time_launches(step, steps, warmup, torch.cuda.current_stream())
+    return ms, h2d, d2h
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2605_08587_b200 import launch_count, workloads as W
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback for the product path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    peaks, peak_src = load_peaks()
+
+    # every rank owns an independent batch of the headline workload (weak scaling)
+    w = W.config2(seed=1 + rank)
+    t = to_dev(w, dev)
+    B, T, H, d = w.q.shape
+    out = torch.empty((B, T, H, d), device=dev, dtype=torch.bfloat16)
+    fin = torch.empty((B, H, d, d), device=dev, dtype=torch.float32)
+    from paper_2605_08587_b200 import kla_chunk_fwd
+
+    def step():
+        kla_chunk_fwd(t["q"], t["k"], t["v"], t["log_alpha"], t["eta"], w.eps, chunk=w.chunk, out=out, final_state=fin)
+
+    stream = torch.cuda.current_stream()
+    for _ in range(max(3, args.warmup)):
+        step()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    n0 = launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local) as clk:
+        e0.record(stream)
+        for _ in range(args.steps):
+            step()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        # keep sampling under load if the timed region was shorter than a few sampling periods
+        t_end = time.time() + 0.6
+        while time.time() < t_end:
+            step()
+        torch.cuda.synchronize()
+    launches = None
+    total_ms = e0.elapsed_time(e1)
+    launches = launch_count() - n0
+    if world > 1:
+        dist.barrier()
+        tm = torch.tensor([total_ms], device=dev)
+        dist.all_reduce(tm, op=dist.ReduceOp.MAX)
+        total_ms = float(tm.item())
+    ms = total_ms / args.steps
+    tokens_all = world * B * T
+    value = tokens_all / (ms * 1e-3) / 1e6
+
+    e2e_ms, h2d, d2h = e2e_leg(w, dev, max(2, min(args.steps, 5)), 2)
+    if world > 1:
+        tm = torch.tensor([e2e_ms], device=dev)
+        dist.all_reduce(tm, op=dist.ReduceOp.MAX)
+        e2e_ms = float(tm.item())
+
+    if rank != 0:
+        if world > 1:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
+
+    nbytes = algorithmic_bytes(B * T, H, d, B, 2, 2, False, True)
+    flops = algorithmic_flops(B * T, H, d, w.chunk)
+    t_hbm = nbytes / (peaks["hbm_gbs"] * 1e9)
+    t_tc = flops / (peaks["bf16_tflops"] * 1e12)
+    achieved = nbytes / (ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": peak_src + " (burst copy)",
+                "kernel": "kla_chunk_tc_kernel" if os.environ.get("KLA_BENCH_SIMT") is None else "kla_chunk_simt_kernel",
+                "algorithmic_bytes_per_launch": nbytes, "algorithmic_flops_per_launch": flops,
+                "tensor_time_us_at_peak": t_tc * 1e6, "hbm_time_us_at_peak": t_hbm * 1e6,
+                "frac_of_roofline_time": max(t_hbm, t_tc) / (ms * 1e-3)}
+    traffic_file = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(traffic_file):
+        try:
+            roofline["traffic"] = json.load(open(traffic_file)).get("chunk_fwd_cfg2_dram_bytes_per_launch")
+        except Exception:
+            pass
+
+    extras = {}
+    if not args.quick:
+        extras["decode_cfg4"] = decode_leg(dev, 256, 4, 2, peaks)
+        extras["decode_l2_defeating_B512"] = decode_leg(dev, 32, 4, 2, peaks, B=512)
+        extras["chunk_cfg3_long_context"] = chunk_leg(W.config3(), dev, 5, 3, peaks, torch.bfloat16)
+        extras["chunk_cfg5_varlen"] = chunk_leg(W.config5(), dev, 5, 3, peaks, torch.bfloat16)
+
+    cpu = None
+    if not args.no_cpu_baseline:
+        v, thr, dt = oracle_sample_run(B=4)
+        cpu = {"value": v, "unit": UNIT, "cores": thr, "kind": "oracle",
+               "sample": "4 of 8 sequences x 8 heads x 4096 tokens of the headline workload, %.1f s" % dt}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(3, args.warmup), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16 inputs, fp32 accumulate/state", "data": "synthetic",
+            "config": {"workload": "cfg2_bf16_B8_H8_T4096_d128_chunk64 per GPU", "tokens_per_step": tokens_all,
+                       "l2": "inputs+outputs per step are 271 MB > 126 MB L2, no flush needed",
+                       "parallelism": "independent batches per GPU, no collective"},
+            "clocks": clk.summary(), "roofline": roofline, "cpu_baseline": cpu,
+            "e2e": {"value": tokens_all / (e2e_ms * 1e-3) / 1e6, "unit": UNIT, "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
+            "gpu_launches": launches, "extras": extras}
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--quick", action="store_true", help="headline workload only (no decode/long/varlen legs)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

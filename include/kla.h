@@ -1,0 +1,144 @@
+/*
+ * kla.h -- C ABI of the B200 (sm_100a) Kaczmarz Linear Attention hot path.
+ *
+ * Two operations, both defined by the same per-head recurrence on a d_k x d_v state S
+ * (Algorithm 1, left panel; coefficient of Eq. 3; transposed form Eq. 6):
+ *
+ *     S~  = exp(log_alpha_t) * S_{t-1}
+ *     e_t = v_t - S~^T k_t
+ *     beta_t = eta_t / (||k_t||^2 + eps)
+ *     S_t = S~ + beta_t * k_t e_t^T
+ *     o_t = S_t^T q_t            (no division by ||q_t||, no 1/sqrt(d_k) scale: the caller
+ *                                 passes the q it wants read out)
+ *
+ * kla_chunk_fwd evaluates it for whole sequences with the chunkwise-parallel solver
+ * (Algorithm 1, right panel; Eqs. 7-9); kla_decode_step applies it to one new token per
+ * sequence with the state updated in place.  The result does not depend on the chunk length.
+ *
+ * General rules
+ *  - Every data pointer is a DEVICE pointer unless stated otherwise; every buffer is owned by the
+ *    caller.  The library allocates nothing and keeps no state between calls.
+ *  - All arrays are dense, row-major, last index contiguous, 16-byte aligned.
+ *  - Work is enqueued on desc->stream and the call returns without synchronising.  Argument
+ *    errors are detected on the host before anything is launched and reported through the
+ *    return value; nothing is launched in that case.
+ *  - There is no CPU fallback: a device that is not compute capability 10.x gives KLA_ERR_ARCH.
+ *  - Not thread-safe per stream beyond what CUDA itself guarantees; calls on different streams
+ *    with disjoint buffers may overlap.
+ */
+#ifndef KLA_H_
+#define KLA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    KLA_OK = 0,
+    KLA_ERR_NULL = -1,      /* a required pointer is NULL                                  */
+    KLA_ERR_SHAPE = -2,     /* unsupported or inconsistent B/T/H/d_k/d_v/n_seq             */
+    KLA_ERR_DTYPE = -3,     /* io_dtype / out_dtype not one of kla_dtype                   */
+    KLA_ERR_ALIGN = -4,     /* a pointer is not 16-byte aligned                            */
+    KLA_ERR_CHUNK = -5,     /* chunk not in {16, 32, 64}                                   */
+    KLA_ERR_SEQLENS = -6,   /* host_seqlens not monotone / does not end at T               */
+    KLA_ERR_WORKSPACE = -7, /* workspace missing or smaller than the query says            */
+    KLA_ERR_EPS = -8,       /* eps < 0 or not finite                                       */
+    KLA_ERR_LAUNCH = -9,    /* the CUDA runtime rejected a launch (see cudaGetLastError)   */
+    KLA_ERR_TIMEOUT = -10,  /* written to *status_word by a kernel whose bounded wait ran out */
+    KLA_ERR_ARCH = -11      /* current device is not sm_100                                */
+} kla_status;
+
+typedef enum { KLA_F32 = 0, KLA_BF16 = 1 } kla_dtype;
+
+/* desc->flags */
+#define KLA_FLAG_NONE 0
+/* Force the CUDA-core fp32 chunk kernel even where the tensor-core kernel applies (used to
+ * cross-check the two device paths against each other and against the oracle). */
+#define KLA_FLAG_FORCE_SIMT 1
+
+typedef struct {
+    int32_t B;        /* sequences in the batch; packed (varlen) input: 1                       */
+    int32_t T;        /* tokens per sequence; packed input: total number of tokens              */
+    int32_t H;        /* heads                                                                  */
+    int32_t d_k;      /* key/query head dimension, 64 or 128                                    */
+    int32_t d_v;      /* value head dimension, equal to d_k                                     */
+    int32_t n_seq;    /* packed input: number of sequences; otherwise equal to B                */
+    const int32_t *cu_seqlens;   /* DEVICE int32[n_seq + 1] cumulative token offsets, or NULL for
+                                    fixed-length input.  Sequence n owns tokens
+                                    cu_seqlens[n] .. cu_seqlens[n+1]-1 of the packed arrays.    */
+    const int32_t *host_seqlens; /* HOST copy of the same array (used for validation and work
+                                    partitioning); required when cu_seqlens is given            */
+    int32_t io_dtype;   /* kla_dtype of q, k, v                                                 */
+    int32_t out_dtype;  /* kla_dtype of out                                                     */
+    int32_t flags;      /* KLA_FLAG_*                                                           */
+    void *workspace;           /* DEVICE scratch of at least kla_chunk_fwd_workspace_bytes()    */
+    size_t workspace_bytes;
+    int32_t *status_word;      /* optional DEVICE int32, zeroed by the caller; a kernel whose
+                                  bounded wait expires stores KLA_ERR_TIMEOUT there and exits  */
+    void *stream;              /* cudaStream_t (NULL = default stream)                          */
+} kla_desc;
+
+/*
+ * Scratch needed by kla_chunk_fwd for this descriptor and chunk length (may be 0).
+ * Host-only computation; returns 0 for an invalid descriptor.
+ */
+size_t kla_chunk_fwd_workspace_bytes(const kla_desc *desc, int32_t chunk);
+
+/*
+ * Chunkwise-parallel forward (Algorithm 1 right; Eqs. 7-9; Props. 3-4).
+ *
+ *   q, k        [B, T, H, d_k]   io_dtype          (packed: [1, n_tok, H, d_k])
+ *   v           [B, T, H, d_v]   io_dtype
+ *   log_alpha   [B, T, H]        fp32, log of the scalar decay alpha_t in (0, 1]
+ *   eta         [B, T, H]        fp32, relaxation gate (a sigmoid output in the paper)
+ *   eps         stabiliser of Eq. 3, >= 0.  eps = 0 with an all-zero key gives NaN (IEEE 0/0).
+ *   chunk       chunk length C in {16, 32, 64}; the tensor-core kernel requires 64
+ *   init_state  [n_seq, H, d_k, d_v] fp32 state before the first token, or NULL for zeros;
+ *               never written
+ *   out         [B, T, H, d_v]   out_dtype, fully overwritten
+ *   final_state [n_seq, H, d_k, d_v] fp32 state after the last token, or NULL to skip; fully
+ *               overwritten; a zero-length sequence gets its initial state
+ *
+ * State layout: S[i][j], i over d_k, j over d_v, j contiguous (Section 2), so o_t = S_t^T q_t.
+ * Arithmetic: bf16 inputs are used exactly; every contraction accumulates in fp32 and the
+ * carried state stays in fp32.
+ */
+kla_status kla_chunk_fwd(const kla_desc *desc, const void *q, const void *k, const void *v,
+                         const float *log_alpha, const float *eta, float eps, int32_t chunk,
+                         const float *init_state, void *out, float *final_state);
+
+/*
+ * One recurrent decode step (Algorithm 1 left) for B sequences x H heads; desc->T must be 1 and
+ * desc->cu_seqlens NULL.
+ *
+ *   q, k [B, H, d_k]   v [B, H, d_v]  io_dtype;   log_alpha, eta [B, H] fp32
+ *   state_inout [B, H, d_k, d_v] fp32, read once and overwritten in place with S_t
+ *   out [B, H, d_v] out_dtype
+ */
+kla_status kla_decode_step(const kla_desc *desc, const void *q, const void *k, const void *v,
+                           const float *log_alpha, const float *eta, float eps,
+                           float *state_inout, void *out);
+
+/*
+ * n_steps consecutive decode steps enqueued back to back on desc->stream (Algorithm 1 left applied
+ * to tokens 0 .. n_steps-1).  Step s reads q + s*B*H*d_k (and likewise k, v, log_alpha, eta) and
+ * writes out + s*B*H*d_v; the state is carried in place.  Equivalent to n_steps calls of
+ * kla_decode_step; exists so that a host loop in an interpreted language is not the bottleneck.
+ */
+kla_status kla_decode_steps(const kla_desc *desc, int32_t n_steps, const void *q, const void *k,
+                            const void *v, const float *log_alpha, const float *eta, float eps,
+                            float *state_inout, void *out);
+
+/* Static, NUL-terminated description of a status code. */
+const char *kla_status_str(kla_status s);
+
+/* Number of kernels the library has launched in this process so far (monotone counter; host). */
+uint64_t kla_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KLA_H_ */

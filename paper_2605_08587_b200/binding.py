@@ -1,0 +1,190 @@
+"""Thin Python binding of the C ABI declared in include/kla.h: argument marshalling only.
+
+PyTorch supplies device memory and the current stream; every arithmetic step of the path runs in
+the library's CUDA kernels.  There is no fallback: a missing library raises at import of the
+symbols, and a non-zero status raises `KlaError`.
+"""
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libkla_b200.so")
+
+KLA_F32, KLA_BF16 = 0, 1
+KLA_FLAG_NONE, KLA_FLAG_FORCE_SIMT = 0, 1
+
+EXPORTS = ["kla_chunk_fwd_workspace_bytes", "kla_chunk_fwd", "kla_decode_step", "kla_decode_steps",
+           "kla_status_str", "kla_launch_count"]
+
+
+class KlaError(RuntimeError):
+    def __init__(self, code, msg):
+        super().__init__("kla status %d: %s" % (code, msg))
+        self.code = code
+
+
+class KlaDesc(ctypes.Structure):
+    _fields_ = [("B", ctypes.c_int32), ("T", ctypes.c_int32), ("H", ctypes.c_int32),
+                ("d_k", ctypes.c_int32), ("d_v", ctypes.c_int32), ("n_seq", ctypes.c_int32),
+                ("cu_seqlens", ctypes.c_void_p), ("host_seqlens", ctypes.c_void_p),
+                ("io_dtype", ctypes.c_int32), ("out_dtype", ctypes.c_int32), ("flags", ctypes.c_int32),
+                ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
+                ("status_word", ctypes.c_void_p), ("stream", ctypes.c_void_p)]
+
+
+_lib = None
+
+
+def load():
+    """Load libkla_b200.so (built in-tree by `paper_2605_08587_b200.build`).  Raises if absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise FileNotFoundError("%s not found: run `python -m paper_2605_08587_b200.build` "
+                                "(there is no CPU or PyTorch fallback)" % LIB_PATH)
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, fp, dp = ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(KlaDesc)
+    lib.kla_chunk_fwd_workspace_bytes.restype = ctypes.c_size_t
+    lib.kla_chunk_fwd_workspace_bytes.argtypes = [dp, ctypes.c_int32]
+    lib.kla_chunk_fwd.restype = ctypes.c_int
+    lib.kla_chunk_fwd.argtypes = [dp, vp, vp, vp, fp, fp, ctypes.c_float, ctypes.c_int32, fp, vp, fp]
+    lib.kla_decode_step.restype = ctypes.c_int
+    lib.kla_decode_step.argtypes = [dp, vp, vp, vp, fp, fp, ctypes.c_float, fp, vp]
+    lib.kla_decode_steps.restype = ctypes.c_int
+    lib.kla_decode_steps.argtypes = [dp, ctypes.c_int32, vp, vp, vp, fp, fp, ctypes.c_float, fp, vp]
+    lib.kla_status_str.restype = ctypes.c_char_p
+    lib.kla_status_str.argtypes = [ctypes.c_int]
+    lib.kla_launch_count.restype = ctypes.c_uint64
+    lib.kla_launch_count.argtypes = []
+    _lib = lib
+    return lib
+
+
+def status_str(code: int) -> str:
+    return load().kla_status_str(int(code)).decode()
+
+
+def launch_count() -> int:
+    return int(load().kla_launch_count())
+
+
+def _check(code):
+    if code != 0:
+        raise KlaError(code, status_str(code))
+
+
+def _dt(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return KLA_F32
+    if t.dtype == torch.bfloat16:
+        return KLA_BF16
+    raise TypeError("q, k, v, out must be float32 or bfloat16, got %s" % t.dtype)
+
+
+def _dev(t, name, dtype=None):
+    if t is None:
+        return None
+    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.is_contiguous()):
+        raise ValueError("%s must be a contiguous CUDA tensor" % name)
+    if dtype is not None and t.dtype != dtype:
+        raise TypeError("%s must be %s" % (name, dtype))
+    return t.data_ptr()
+
+
+def _stream(dev):
+    return torch.cuda.current_stream(dev).cuda_stream
+
+
+def kla_chunk_fwd(q, k, v, log_alpha, eta, eps, chunk=64, init_state=None, out=None, final_state=None,
+                  cu_seqlens=None, host_seqlens=None, out_dtype=None, flags=KLA_FLAG_NONE,
+                  want_final_state=True, status_word=None):
+    """Chunkwise forward (include/kla.h: kla_chunk_fwd).
+
+    q, k [B, T, H, d_k]; v [B, T, H, d_v]; log_alpha, eta [B, T, H] fp32; all CUDA, contiguous.
+    Packed input: B = 1, cu_seqlens int32 CUDA [n_seq + 1] plus `host_seqlens` (CPU int32 copy;
+    made from cu_seqlens with one D2H copy if omitted).
+    Returns (out, final_state); buffers are allocated here unless passed in.
+    """
+    lib = load()
+    B, T, H, d_k = q.shape
+    d_v = v.shape[-1]
+    if tuple(k.shape) != (B, T, H, d_k) or tuple(v.shape) != (B, T, H, d_v):
+        raise ValueError("q, k, v shapes disagree")
+    if tuple(log_alpha.shape) != (B, T, H) or tuple(eta.shape) != (B, T, H):
+        raise ValueError("log_alpha, eta must be [B, T, H]")
+    if k.dtype != q.dtype or v.dtype != q.dtype:
+        raise TypeError("q, k, v must share one dtype")
+    n_seq = B
+    hs = None
+    if cu_seqlens is not None:
+        if cu_seqlens.dtype != torch.int32:
+            raise TypeError("cu_seqlens must be int32")
+        hs = (cu_seqlens.cpu() if host_seqlens is None else host_seqlens).contiguous()
+        if hs.dtype != torch.int32 or hs.is_cuda:
+            raise TypeError("host_seqlens must be a CPU int32 tensor")
+        n_seq = cu_seqlens.numel() - 1
+    if out is None:
+        out = torch.empty((B, T, H, d_v), device=q.device, dtype=out_dtype or q.dtype)
+    if final_state is None and want_final_state:
+        final_state = torch.empty((n_seq, H, d_k, d_v), device=q.device, dtype=torch.float32)
+    if init_state is not None and tuple(init_state.shape) != (n_seq, H, d_k, d_v):
+        raise ValueError("init_state must be [n_seq, H, d_k, d_v]")
+    desc = KlaDesc(B=B, T=T, H=H, d_k=d_k, d_v=d_v, n_seq=n_seq,
+                   cu_seqlens=_dev(cu_seqlens, "cu_seqlens"), host_seqlens=hs.data_ptr() if hs is not None else None,
+                   io_dtype=_dt(q), out_dtype=_dt(out), flags=flags, workspace=None, workspace_bytes=0,
+                   status_word=_dev(status_word, "status_word", torch.int32), stream=_stream(q.device))
+    ws = None
+    need = lib.kla_chunk_fwd_workspace_bytes(ctypes.byref(desc), chunk)
+    if need:
+        ws = torch.empty(need, device=q.device, dtype=torch.uint8)
+        desc.workspace, desc.workspace_bytes = ws.data_ptr(), need
+    with torch.cuda.device(q.device):
+        code = lib.kla_chunk_fwd(ctypes.byref(desc), _dev(q, "q"), _dev(k, "k"), _dev(v, "v"),
+                                 _dev(log_alpha, "log_alpha", torch.float32), _dev(eta, "eta", torch.float32),
+                                 float(eps), int(chunk), _dev(init_state, "init_state", torch.float32),
+                                 _dev(out, "out"), _dev(final_state, "final_state", torch.float32))
+    _check(code)
+    return out, final_state
+
+
+def _decode_desc(q, v, out, B, H, d_k, d_v):
+    return KlaDesc(B=B, T=1, H=H, d_k=d_k, d_v=d_v, n_seq=B, cu_seqlens=None, host_seqlens=None,
+                   io_dtype=_dt(q), out_dtype=_dt(out), flags=0, workspace=None, workspace_bytes=0,
+                   status_word=None, stream=_stream(q.device))
+
+
+def kla_decode_step(q, k, v, log_alpha, eta, eps, state_inout, out=None, out_dtype=None):
+    """One decode step (include/kla.h: kla_decode_step).  q, k [B, H, d_k]; v [B, H, d_v];
+    log_alpha, eta [B, H] fp32; state_inout [B, H, d_k, d_v] fp32, updated in place."""
+    lib = load()
+    B, H, d_k = q.shape
+    d_v = v.shape[-1]
+    if out is None:
+        out = torch.empty((B, H, d_v), device=q.device, dtype=out_dtype or q.dtype)
+    desc = _decode_desc(q, v, out, B, H, d_k, d_v)
+    with torch.cuda.device(q.device):
+        code = lib.kla_decode_step(ctypes.byref(desc), _dev(q, "q"), _dev(k, "k"), _dev(v, "v"),
+                                   _dev(log_alpha, "log_alpha", torch.float32), _dev(eta, "eta", torch.float32),
+                                   float(eps), _dev(state_inout, "state_inout", torch.float32), _dev(out, "out"))
+    _check(code)
+    return out
+
+
+def kla_decode_steps(q, k, v, log_alpha, eta, eps, state_inout, out=None, out_dtype=None):
+    """n consecutive decode steps (include/kla.h: kla_decode_steps).  q, k [n, B, H, d_k];
+    v [n, B, H, d_v]; log_alpha, eta [n, B, H]; state carried in place; out [n, B, H, d_v]."""
+    lib = load()
+    n, B, H, d_k = q.shape
+    d_v = v.shape[-1]
+    if out is None:
+        out = torch.empty((n, B, H, d_v), device=q.device, dtype=out_dtype or q.dtype)
+    desc = _decode_desc(q, v, out, B, H, d_k, d_v)
+    with torch.cuda.device(q.device):
+        code = lib.kla_decode_steps(ctypes.byref(desc), n, _dev(q, "q"), _dev(k, "k"), _dev(v, "v"),
+                                    _dev(log_alpha, "log_alpha", torch.float32), _dev(eta, "eta", torch.float32),
+                                    float(eps), _dev(state_inout, "state_inout", torch.float32), _dev(out, "out"))
+    _check(code)
+    return out

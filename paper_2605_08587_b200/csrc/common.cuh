@@ -1,0 +1,76 @@
+// Shared device/host helpers for the KLA kernels (sm_100a).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "kla.h"
+
+namespace kla {
+
+// Everything a chunk-forward kernel needs; passed by value.
+struct ChunkParams {
+    const void *q, *k, *v;
+    const float *log_alpha, *eta;
+    const float *init_state;  // may be null
+    void *out;
+    float *final_state;       // may be null
+    const int32_t *cu_seqlens;  // device, may be null (fixed length)
+    int32_t *status_word;       // may be null
+    int32_t B, T, H, n_seq;
+    float eps;
+};
+
+struct DecodeParams {
+    const void *q, *k, *v;
+    const float *log_alpha, *eta;
+    float *state;
+    void *out;
+    int32_t BH;
+    float eps;
+};
+
+// Launchers implemented in the kernel translation units.  Each returns cudaGetLastError().
+cudaError_t launch_decode(const DecodeParams &p, int d, int io_dtype, int out_dtype,
+                          cudaStream_t stream);
+cudaError_t launch_chunk_simt(const ChunkParams &p, int d, int chunk, int io_dtype, int out_dtype,
+                              cudaStream_t stream);
+cudaError_t launch_chunk_tc(const ChunkParams &p, int d, int io_dtype, int out_dtype,
+                            cudaStream_t stream);
+// True when the tensor-core kernel covers this case.
+bool chunk_tc_supported(int d, int chunk, int io_dtype);
+
+void count_launch(int n);
+
+// ---- device helpers -------------------------------------------------------------------------
+__device__ __forceinline__ float to_f32(float x) { return x; }
+__device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }
+
+template <typename T>
+__device__ __forceinline__ T from_f32(float x);
+template <>
+__device__ __forceinline__ float from_f32<float>(float x) { return x; }
+template <>
+__device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float x) { return __float2bfloat16_rn(x); }
+
+// Load 4 consecutive elements (16-byte aligned for fp32, 8-byte aligned for bf16) as fp32.
+__device__ __forceinline__ float4 load4(const float *p) { return *reinterpret_cast<const float4 *>(p); }
+__device__ __forceinline__ float4 load4(const __nv_bfloat16 *p)
+{
+    uint2 raw = *reinterpret_cast<const uint2 *>(p);
+    __nv_bfloat162 a = *reinterpret_cast<__nv_bfloat162 *>(&raw.x);
+    __nv_bfloat162 b = *reinterpret_cast<__nv_bfloat162 *>(&raw.y);
+    float2 fa = __bfloat1622float2(a), fb = __bfloat1622float2(b);
+    return make_float4(fa.x, fa.y, fb.x, fb.y);
+}
+__device__ __forceinline__ void store4(float *p, float4 x) { *reinterpret_cast<float4 *>(p) = x; }
+__device__ __forceinline__ void store4(__nv_bfloat16 *p, float4 x)
+{
+    __nv_bfloat162 a = __floats2bfloat162_rn(x.x, x.y), b = __floats2bfloat162_rn(x.z, x.w);
+    uint2 raw;
+    raw.x = *reinterpret_cast<uint32_t *>(&a);
+    raw.y = *reinterpret_cast<uint32_t *>(&b);
+    *reinterpret_cast<uint2 *>(p) = raw;
+}
+
+}  // namespace kla

@@ -1,0 +1,182 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 oracle on identical
+seeded inputs.  Tolerances: max|err|/rms(ref) <= 2e-3 for bf16 inputs (fp32 `out` and the fp32
+final state), <= 1e-5 for fp32 inputs; a bf16 `out` is allowed its own rounding on top."""
+import numpy as np
+import pytest
+import torch
+
+from helpers import (TOL_BF16, TOL_F32, assert_bf16_out_close, gpu_chunk, np64, oracle_chunk, rel_err)
+from paper_2605_08587_b200 import KLA_FLAG_FORCE_SIMT, workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+def _check_fixed(w, tol, flags=0, chunk=None, out_dtype=torch.float32):
+    out, fin = gpu_chunk(w, out_dtype=out_dtype, flags=flags, chunk=chunk)
+    ro, rf = oracle_chunk(w)
+    if out_dtype == torch.bfloat16:
+        assert_bf16_out_close(out, ro, tol)
+    else:
+        assert rel_err(np64(out), ro) <= tol
+    assert rel_err(np64(fin), rf) <= tol
+    return out, fin
+
+
+# ---- config 1: fp32, exact shape ------------------------------------------------------------------
+@pytest.mark.parametrize("chunk", [16, 32, 64])
+def test_config1_fp32_exact_shape(chunk):
+    _check_fixed(W.config1(), TOL_F32, chunk=chunk)
+
+
+def test_config1_fp32_d128_ragged():
+    _check_fixed(W.config1(B=2, H=3, T=200, d=128, seed=11), TOL_F32)
+
+
+# ---- configs 2/3 at sizes the oracle finishes in seconds (several chunks + ragged tail) -----------
+@pytest.mark.parametrize("flags", [0, KLA_FLAG_FORCE_SIMT])
+def test_config2_small_bf16(flags):
+    _check_fixed(W.config2(B=2, H=3, T=1000), TOL_BF16, flags=flags)
+
+
+@pytest.mark.parametrize("flags", [0, KLA_FLAG_FORCE_SIMT])
+def test_config2_small_bf16_out_bf16(flags):
+    _check_fixed(W.config2(B=1, H=2, T=333, seed=21), TOL_BF16, flags=flags, out_dtype=torch.bfloat16)
+
+
+@pytest.mark.parametrize("flags", [0, KLA_FLAG_FORCE_SIMT])
+def test_config3_small_with_init_state(flags):
+    _check_fixed(W.config3(B=1, H=4, T=2048 + 17), TOL_BF16, flags=flags)
+
+
+@pytest.mark.parametrize("flags", [0, KLA_FLAG_FORCE_SIMT])
+@pytest.mark.parametrize("d", [64, 128])
+@pytest.mark.parametrize("T", [1, 5, 63, 64, 65, 128, 129])
+def test_short_and_boundary_lengths(T, d, flags):
+    w = W.config3(B=2, H=2, T=T, d=d, seed=100 + T)
+    _check_fixed(w, TOL_BF16, flags=flags)
+
+
+# ---- config 5: packed variable-length ----------------------------------------------------------------
+@pytest.mark.parametrize("flags", [0, KLA_FLAG_FORCE_SIMT])
+def test_config5_small_varlen(flags):
+    w = W.config5(H=4, lengths=[1, 63, 64, 65, 300, 1, 129, 2, 517])
+    out, fin = gpu_chunk(w, flags=flags)
+    ro, rf, _ = oracle_chunk(w)
+    assert rel_err(np64(out)[0], ro) <= TOL_BF16
+    assert rel_err(np64(fin), rf) <= TOL_BF16
+    cu = w.cu_seqlens.numpy()
+    worst = max(rel_err(np64(out)[0, cu[n]:cu[n + 1]], ro[cu[n]:cu[n + 1]]) for n in range(len(cu) - 1))
+    assert worst <= 5 * TOL_BF16   # per-sequence figure, reported for the heavy-tailed keys
+
+
+@pytest.mark.parametrize("flags", [0, KLA_FLAG_FORCE_SIMT])
+def test_varlen_zero_length_sequences_keep_their_initial_state(flags):
+    w = W.config5(H=2, lengths=[0, 70, 0, 3, 0], seed=5)
+    gen = torch.Generator().manual_seed(77)
+    w.init_state = (0.05 * torch.randn(5, 2, 64, 64, generator=gen)).float()
+    out, fin = gpu_chunk(w, flags=flags)
+    ro, rf, _ = oracle_chunk(w)
+    assert rel_err(np64(out)[0], ro) <= TOL_BF16
+    assert rel_err(np64(fin), rf) <= TOL_BF16
+    for n in (0, 2, 4):
+        assert torch.equal(fin[n].cpu(), w.init_state[n])
+
+
+def test_varlen_equals_fixed_length_bitwise():
+    """Packing B equal-length sequences must give exactly the fixed-length result."""
+    w = W.config2(B=3, H=2, T=130, seed=31)
+    out_f, fin_f = gpu_chunk(w)
+    wp = W.ChunkWorkload("packed", w.q.reshape(1, -1, 2, 128), w.k.reshape(1, -1, 2, 128), w.v.reshape(1, -1, 2, 128),
+                         w.log_alpha.reshape(1, -1, 2), w.eta.reshape(1, -1, 2), w.eps, w.chunk,
+                         cu_seqlens=torch.tensor([0, 130, 260, 390], dtype=torch.int32))
+    out_p, fin_p = gpu_chunk(wp)
+    assert torch.equal(out_p.reshape(3, 130, 2, 128), out_f)
+    assert torch.equal(fin_p, fin_f)
+
+
+# ---- properties that hold at any size -------------------------------------------------------------------
+@pytest.mark.parametrize("flags", [0, KLA_FLAG_FORCE_SIMT])
+def test_state_handoff_on_gpu(flags):
+    w = W.config2(B=2, H=2, T=512, seed=41)
+    out, fin = gpu_chunk(w, flags=flags)
+    T1 = 192
+    def part(a, b, s0):
+        return W.ChunkWorkload("p", w.q[:, a:b].contiguous(), w.k[:, a:b].contiguous(), w.v[:, a:b].contiguous(),
+                               w.log_alpha[:, a:b].contiguous(), w.eta[:, a:b].contiguous(), w.eps, w.chunk, init_state=s0)
+    o1, f1 = gpu_chunk(part(0, T1, None), flags=flags)
+    o2, f2 = gpu_chunk(part(T1, 512, f1.cpu()), flags=flags)
+    ref = np64(out)
+    assert rel_err(np64(torch.cat([o1, o2], 1)), ref) <= 1e-5   # T1 is a chunk multiple: same arithmetic
+    assert rel_err(np64(f2), np64(fin)) <= 1e-5
+
+
+@pytest.mark.parametrize("flags", [0, KLA_FLAG_FORCE_SIMT])
+def test_eta_zero_is_pure_decay(flags):
+    w = W.config3(B=1, H=2, T=150, seed=51)
+    w.eta = torch.zeros_like(w.eta)
+    out, fin = gpu_chunk(w, flags=flags)
+    gamma = torch.exp(torch.cumsum(w.log_alpha.double(), 1))
+    expect = gamma[..., None] * torch.einsum("bhkv,bthk->bthv", w.init_state.double(), w.q.double())
+    assert rel_err(np64(out), expect.numpy()) <= 1e-5
+    assert rel_err(np64(fin), (gamma[:, -1][..., None, None] * w.init_state.double()).numpy()) <= 1e-5
+
+
+@pytest.mark.parametrize("flags", [0, KLA_FLAG_FORCE_SIMT])
+def test_kaczmarz_projection_on_gpu(flags):
+    """eta = 1, eps = 0: reading the final state with the last key returns the last value."""
+    w = W.config2(B=2, H=2, T=100, seed=61)
+    w.eta = torch.ones_like(w.eta)
+    w.eps = 0.0
+    out, fin = gpu_chunk(w, flags=flags)
+    pred = torch.einsum("bhkv,bhk->bhv", fin.double().cpu(), w.k[:, -1].double())
+    assert rel_err(pred.numpy(), w.v[:, -1].double().numpy()) <= TOL_BF16
+
+
+def test_run_to_run_determinism():
+    w = W.config2(B=2, H=2, T=700, seed=71)
+    a = gpu_chunk(w)
+    b = gpu_chunk(w)
+    assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
+
+
+def test_final_state_optional_and_out_untouched_outside():
+    w = W.config2(B=1, H=2, T=100, seed=81)
+    out, fin = gpu_chunk(w, want_final_state=False)
+    assert fin is None
+    ro, _ = oracle_chunk(w)
+    assert rel_err(np64(out), ro) <= TOL_BF16
+
+
+# ---- full-size configurations, in the launch configuration the benchmark times ---------------------------
+# The oracle is run on a sample of (sequence, head) pairs; each pair is an independent problem, so the
+# sampled comparison is exact for the pairs it covers.
+def test_config2_full_size_sampled():
+    w = W.config2()
+    out, fin = gpu_chunk(w)
+    heads, seqs = [0, 5], [1, 6]
+    ro, rf = oracle_chunk(w, heads=heads, seqs=seqs)
+    assert rel_err(np64(out[seqs][:, :, heads]), ro) <= TOL_BF16
+    assert rel_err(np64(fin[seqs][:, heads]), rf) <= TOL_BF16
+    assert torch.isfinite(out).all() and torch.isfinite(fin).all()
+
+
+def test_config3_full_size_sampled():
+    w = W.config3()
+    out, fin = gpu_chunk(w)
+    heads = [3]
+    ro, rf = oracle_chunk(w, heads=heads)
+    assert rel_err(np64(out[:, :, heads]), ro) <= TOL_BF16
+    assert rel_err(np64(fin[:, heads]), rf) <= TOL_BF16
+    assert torch.isfinite(out).all() and torch.isfinite(fin).all()
+
+
+def test_config5_full_size_sampled():
+    w = W.config5()
+    out, fin = gpu_chunk(w)
+    lens = np.diff(w.cu_seqlens.numpy())
+    seqs = sorted({int(np.argmax(lens)), int(np.argmin(lens)), 0, 31})
+    heads = [2, 11]
+    ro, rf, idx = oracle_chunk(w, heads=heads, seqs=seqs)
+    assert rel_err(np64(out[0][idx][:, heads]), ro) <= TOL_BF16
+    assert rel_err(np64(fin[seqs][:, heads]), rf) <= TOL_BF16
+    assert torch.isfinite(out).all() and torch.isfinite(fin).all()

@@ -290,7 +290,7 @@ def run_ours(args):
         e1.record(stream)
         torch.cuda.synchronize()
         # keep sampling under load if the timed region was shorter than a few sampling periods
-        t_end = time.time() + 0.6
+        t_end = time.time() + (0.0 if args.quick else 0.6)
         while time.time() < t_end:
             step()
         torch.cuda.synchronize()
@@ -306,7 +306,7 @@ def run_ours(args):
     tokens_all = world * B * T
     value = tokens_all / (ms * 1e-3) / 1e6
 
-    e2e_ms, h2d, d2h = e2e_leg(w, dev, max(2, min(args.steps, 5)), 2)
+    e2e_ms, h2d, d2h = (float("nan"), 0, 0) if args.quick else e2e_leg(w, dev, max(2, min(args.steps, 5)), 2)
     if world > 1:
         tm = torch.tensor([e2e_ms], device=dev)
         dist.all_reduce(tm, op=dist.ReduceOp.MAX)
@@ -344,7 +344,7 @@ def run_ours(args):
         extras["chunk_cfg5_varlen"] = chunk_leg(W.config5(), dev, 5, 3, peaks, torch.bfloat16)
 
     cpu = None
-    if not args.no_cpu_baseline:
+    if not (args.no_cpu_baseline or args.quick):
         v, thr, dt = oracle_sample_run(B=4)
         cpu = {"value": v, "unit": UNIT, "cores": thr, "kind": "oracle",
                "sample": "4 of 8 sequences x 8 heads x 4096 tokens of the headline workload, %.1f s" % dt}
@@ -371,7 +371,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--quick", action="store_true", help="headline workload only (no decode/long/varlen legs)")
+    ap.add_argument("--quick", action="store_true", help="profiling mode: headline kernel only (no e2e, decode, long-context, varlen or CPU legs)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":

@@ -37,7 +37,9 @@ struct SimtSmem {
     float S[D][NS];
     float L[C][LDL];
     float P[C][LDL];
-    float beta[C], g[C], la[C], eta[C];
+    double g[C];       // chunk-local running sum of log alpha; kept in fp64 so that the
+                       // differences g_i - g_j below do not cancel away fp32 digits
+    float beta[C], la[C], eta[C];
 };
 
 template <typename IO>
@@ -176,21 +178,21 @@ __global__ void __launch_bounds__(NTHREADS) kla_chunk_simt_kernel(ChunkParams p)
         if (warp == 0) {
             // inclusive scan of C values, C/32 (or fewer) per lane
             constexpr int PER = (C + 31) / 32;
-            float loc[PER];
-            float run = 0.f;
+            double loc[PER];
+            double run = 0.0;
 #pragma unroll
             for (int u = 0; u < PER; ++u) {
                 const int i = lane * PER + u;
-                run += (i < C) ? sm.la[i] : 0.f;
+                run += (i < C) ? (double)sm.la[i] : 0.0;
                 loc[u] = run;
             }
-            float incl = run;
+            double incl = run;
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
-                const float t = __shfl_up_sync(0xffffffffu, incl, o);
+                const double t = __shfl_up_sync(0xffffffffu, incl, o);
                 if (lane >= o) incl += t;
             }
-            const float excl = incl - run;
+            const double excl = incl - run;
 #pragma unroll
             for (int u = 0; u < PER; ++u) {
                 const int i = lane * PER + u;
@@ -225,7 +227,7 @@ __global__ void __launch_bounds__(NTHREADS) kla_chunk_simt_kernel(ChunkParams p)
 #pragma unroll
                     for (int b = 0; b < 4; ++b) {
                         const int i = 4 * ti + a, j = 4 * tj + b;
-                        const float ratio = (j <= i) ? expf(sm.g[i] - sm.g[j]) : 0.f;
+                        const float ratio = (j <= i) ? expf((float)(sm.g[i] - sm.g[j])) : 0.f;
                         sm.L[i][j] = (j < i) ? sm.beta[i] * ratio * aG[a][b] : 0.f;
                         sm.P[i][j] = ratio * aP[a][b];
                     }
@@ -256,7 +258,7 @@ __global__ void __launch_bounds__(NTHREADS) kla_chunk_simt_kernel(ChunkParams p)
 #pragma unroll
             for (int a = 0; a < 4; ++a) {
                 const int i = 4 * ti + a;
-                const float gam = expf(sm.g[i]);
+                const float gam = expf((float)sm.g[i]);
                 if (which == 0) {
                     const float b = sm.beta[i];
                     const float4 vv = *reinterpret_cast<const float4 *>(&sm.V[i][4 * tc]);
@@ -345,8 +347,8 @@ __global__ void __launch_bounds__(NTHREADS) kla_chunk_simt_kernel(ChunkParams p)
         // ---- state: S <- gamma_C S + K^T diag(exp(g_C - g_j)) U -------------------------------
         {
             const int tc = tid % 8, td = tid / 8;  // RD rows x 4 columns per thread
-            const float gC = sm.g[C - 1];
-            const float gamC = expf(gC);
+            const double gC = sm.g[C - 1];
+            const float gamC = expf((float)gC);
             float acc[RD][4];
 #pragma unroll
             for (int a = 0; a < RD; ++a) {
@@ -354,7 +356,7 @@ __global__ void __launch_bounds__(NTHREADS) kla_chunk_simt_kernel(ChunkParams p)
                 acc[a][0] = gamC * s0.x; acc[a][1] = gamC * s0.y; acc[a][2] = gamC * s0.z; acc[a][3] = gamC * s0.w;
             }
             for (int j = 0; j < C; ++j) {
-                const float dj = expf(gC - sm.g[j]);
+                const float dj = expf((float)(gC - sm.g[j]));
                 float4 u = *reinterpret_cast<const float4 *>(&sm.X[j][4 * tc]);
                 u.x *= dj; u.y *= dj; u.z *= dj; u.w *= dj;
 #pragma unroll

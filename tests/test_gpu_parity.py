@@ -117,8 +117,9 @@ def test_eta_zero_is_pure_decay(flags):
     out, fin = gpu_chunk(w, flags=flags)
     gamma = torch.exp(torch.cumsum(w.log_alpha.double(), 1))
     expect = gamma[..., None] * torch.einsum("bhkv,bthk->bthv", w.init_state.double(), w.q.double())
-    assert rel_err(np64(out), expect.numpy()) <= 1e-5
-    assert rel_err(np64(fin), (gamma[:, -1][..., None, None] * w.init_state.double()).numpy()) <= 1e-5
+    tol = 1e-5 if flags else 3e-4   # fp32 CUDA-core path / split-bf16 tensor-core path
+    assert rel_err(np64(out), expect.numpy()) <= tol
+    assert rel_err(np64(fin), (gamma[:, -1][..., None, None] * w.init_state.double()).numpy()) <= tol
 
 
 @pytest.mark.parametrize("flags", [0, KLA_FLAG_FORCE_SIMT])

@@ -93,6 +93,7 @@ kla_status kla_chunk_fwd(const kla_desc *desc, const void *q, const void *k, con
     p.final_state = final_state;
     p.cu_seqlens = desc->cu_seqlens;
     p.status_word = desc->status_word;
+    p.trace = nullptr;
     p.B = desc->B; p.T = desc->T; p.H = desc->H; p.n_seq = desc->n_seq;
     p.eps = eps;
     if (desc->T == 0) {

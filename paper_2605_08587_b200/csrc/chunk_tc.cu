@@ -29,6 +29,8 @@
 // KLA_ERR_TIMEOUT through the status word, releases its TMEM and exits.
 #include <cuda.h>
 
+#include <cstdio>
+#include <cstring>
 #include <mutex>
 
 #include "common.cuh"
@@ -42,10 +44,11 @@ using namespace umma;
 
 constexpr int C = 64;    // chunk length
 constexpr int NS = 64;   // state columns per CTA
-constexpr int PG_T = 128, CG_T = 256;
+constexpr int PG_T = 256, CG_T = 256;
 constexpr int NT = PG_T + CG_T + 32;
 constexpr int NSTAGE = 3;
 constexpr long long WAIT_LIMIT = 2000000000LL;  // SM clocks (~1 s) before a wait gives up
+constexpr float LOG2E = 1.4426950408889634f;
 
 // TMEM columns (fp32, 128 lanes each)
 constexpr uint32_t TM_D1 = 0, TM_KS = 64, TM_QS0 = 128, TM_QS1 = 192, TM_U = 256, TM_PU = 320, TM_DS = 384, TM_COLS = 512;
@@ -59,12 +62,12 @@ enum Bar {
     B_D1_FREE = 4,           // pre group finished reading D1(c)
     B_TP_READY = 5,          // T(c), P(c), scalars(c) written
     B_S_READY = 6,           // state tiles for chunk c written
-    B_D2_DONE = 7,           // MMA-2(c) complete
+    B_D2_DONE = 7,           // K S_0 of chunk c complete
     B_RHS_READY = 8,
     B_D3_DONE = 9,
     B_U_READY = 10,
     B_D5_DONE = 11,
-    B_D4_DONE = 12,
+    B_D4_DONE = 12,          // P U (and, earlier in the pipe, Q S_0) of chunk c complete
     B_TAIL_READY = 13,       // masked rows of the last chunk zeroed
     B_COUNT = 14
 };
@@ -87,46 +90,54 @@ struct TcSmem {
     alignas(1024) unsigned char du_lo[8192];
     alignas(16) float tl[64 * LDT];             // L, overwritten in place by T = (I + L)^-1
     alignas(16) float mm[32 * LDM];             // scratch for the block products of the solve
+    alignas(16) float g2[64];                   // log2(e) * chunk-local running sum of log alpha
     float beta[NSTAGE][64];
     float gam[NSTAGE][64];                      // exp(g_i)
     float dec[NSTAGE][64];                      // exp(g_C - g_i)
-    float la[64];
-    double g[64];
     alignas(8) uint64_t bar[B_COUNT];
     uint32_t tmem_base;
     volatile int abort_flag;
 };
 
 // ---- small fp32 block products on shared memory, used by the triangular solve ------------------------
-// Cm[r][c] = sign * sum_{k = klo(c) .. khi(r)} A[r][k] * Bm[k][c]   for an R x 16*NC4/4.. tile set.
-// Each calling thread owns ROWS x 4 outputs: rows r0.., columns c4..c4+3.
-// b_lower: Bm is lower triangular (Bm[k][c] = 0 for k < c)  -> start k at c4
-// a_lower: A  is lower triangular (A[r][k]  = 0 for k > r)  -> stop k at the tile's last row
-template <int ROWS>
-__device__ __forceinline__ void tile_mm(float *Cm, int ldc, const float *A, int lda, const float *Bm, int ldb, int r0,
-                                        int c4, int K, bool b_lower, bool a_lower, float sign)
+// Cm[r][c4..c4+CW) = sign * sum_k A[r][k] * Bm[k][c4..c4+CW) for one row r; K is a compile-time bound.
+// b_lower: Bm is lower triangular (Bm[k][c] = 0 for k < c)  -> terms with k < c4 are skipped
+// a_lower: A  is lower triangular (A[r][k]  = 0 for k > r)  -> terms with k > r are skipped
+template <int K, int CW>
+__device__ __forceinline__ void row_mm(float *Cm, int ldc, const float *A, int lda, const float *Bm, int ldb, int r,
+                                       int c4, bool b_lower, bool a_lower, float sign)
 {
-    float acc[ROWS][4];
+    float acc[CW];
 #pragma unroll
-    for (int a = 0; a < ROWS; ++a) acc[a][0] = acc[a][1] = acc[a][2] = acc[a][3] = 0.f;
+    for (int e = 0; e < CW; ++e) acc[e] = 0.f;
     const int k0 = b_lower ? c4 : 0;
-    const int k1 = a_lower ? min(K, r0 + ROWS) : K;
-#pragma unroll 4
-    for (int k = k0; k < k1; ++k) {
-        const float4 b = *reinterpret_cast<const float4 *>(Bm + k * ldb + c4);
+    const int k1 = a_lower ? (r + 1) : K;
 #pragma unroll
-        for (int a = 0; a < ROWS; ++a) {
-            const float x = A[(r0 + a) * lda + k];
-            acc[a][0] += x * b.x; acc[a][1] += x * b.y; acc[a][2] += x * b.z; acc[a][3] += x * b.w;
+    for (int kk = 0; kk < K; kk += 4) {
+        if (kk + 4 > k0 && kk < k1) {
+            const float4 a = *reinterpret_cast<const float4 *>(A + r * lda + kk);
+            const float av[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int k = kk + u;
+                // zero operands outside the triangular ranges contribute exact zeros; no predicate needed
+                if (CW == 4) {
+                    const float4 b = *reinterpret_cast<const float4 *>(Bm + k * ldb + c4);
+                    acc[0] += av[u] * b.x; acc[1] += av[u] * b.y; acc[2] += av[u] * b.z; acc[3] += av[u] * b.w;
+                } else {
+                    const float2 b = *reinterpret_cast<const float2 *>(Bm + k * ldb + c4);
+                    acc[0] += av[u] * b.x; acc[1] += av[u] * b.y;
+                }
+            }
         }
     }
-#pragma unroll
-    for (int a = 0; a < ROWS; ++a)
-        *reinterpret_cast<float4 *>(Cm + (r0 + a) * ldc + c4) =
-            make_float4(sign * acc[a][0], sign * acc[a][1], sign * acc[a][2], sign * acc[a][3]);
+    if (CW == 4)
+        *reinterpret_cast<float4 *>(Cm + r * ldc + c4) = make_float4(sign * acc[0], sign * acc[1], sign * acc[2], sign * acc[3]);
+    else
+        *reinterpret_cast<float2 *>(Cm + r * ldc + c4) = make_float2(sign * acc[0], sign * acc[1]);
 }
 
-__device__ __forceinline__ void pg_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+__device__ __forceinline__ void pg_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 __device__ __forceinline__ void pg_half_sync() { asm volatile("bar.sync 2, 64;" ::: "memory"); }
 // Barrier over the pre group that also ORs a flag: makes "some thread's wait gave up" a collective
 // decision, so that no thread is left alone at a later pg_sync().
@@ -135,12 +146,23 @@ __device__ __forceinline__ bool pg_any(bool flag)
     uint32_t r;
     asm volatile(
         "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 p, %1, 0;\n\t"
-        "bar.red.or.pred q, 3, 128, p;\n\tselp.u32 %0, 1, 0, q;\n\t}"
+        "bar.red.or.pred q, 3, 256, p;\n\tselp.u32 %0, 1, 0, q;\n\t}"
         : "=r"(r)
         : "r"((uint32_t)flag)
         : "memory");
     return r != 0;
 }
+
+#ifdef KLA_TRACE
+// role r (0 control, 1 pre, 2 chain), chunk c, event e -> trace[(r * 64 + c) * 16 + e]
+#define KLA_TR(r, c, e)                                                                        \
+    do {                                                                                       \
+        if (p.trace && blockIdx.x == 0 && (c) < 64 && (((r) == 0) || ((r) == 1 && tid == 0) || ((r) == 2 && tid == PG_T))) \
+            p.trace[((r) * 64 + (c)) * 16 + (e)] = clock64();                                  \
+    } while (0)
+#else
+#define KLA_TR(r, c, e) do { } while (0)
+#endif
 
 template <int D, typename OUT>
 __global__ void __launch_bounds__(NT, 1)
@@ -248,13 +270,21 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     tma_load_2d(sm.kq[st] + kb * 16384 + 8192, &tm_q, h * D + kb * 64, row, &sm.bar[B_FULL0 + st]);
                 }
             };
+            // Descriptors: everything except the 14-bit start-address field is fixed, so a K-step is an add.
+            const uint64_t d_kq0 = smem_desc_sw128(smem_u32(sm.kq[0]), 16, 1024);             // K-major views of a stage
+            const uint64_t d_kt0 = smem_desc_sw128(smem_u32(sm.kq[0]), KB * 8192, 1024);      // K^T (MN-major) view
+            const uint64_t d_sh = smem_desc_sw128(smem_u32(sm.s_hi), 16, 1024), d_sl = smem_desc_sw128(smem_u32(sm.s_lo), 16, 1024);
+            const uint64_t d_th = smem_desc_sw128(smem_u32(sm.t_hi), 16, 1024), d_tl = smem_desc_sw128(smem_u32(sm.t_lo), 16, 1024);
+            const uint64_t d_ph = smem_desc_sw128(smem_u32(sm.p_hi), 16, 1024), d_pl = smem_desc_sw128(smem_u32(sm.p_lo), 16, 1024);
+            const uint64_t d_rh = smem_desc_sw128(smem_u32(sm.ru_hi), 16, 1024), d_rl = smem_desc_sw128(smem_u32(sm.ru_lo), 16, 1024);
+            const uint64_t d_dh = smem_desc_sw128(smem_u32(sm.du_hi), 16, 1024), d_dl = smem_desc_sw128(smem_u32(sm.du_lo), 16, 1024);
+            constexpr uint64_t STAGE_STEP = (uint64_t)(Smem::KQ_BYTES >> 4);
+            auto kstep = [](int s) -> uint64_t { return (uint64_t)(((s / 4) * 16384 + (s % 4) * 32) >> 4); };
+
             auto mma1 = [&](int c) {  // [K;Q] K^T -> D1
-                const uint32_t a0 = smem_u32(sm.kq[c % NSTAGE]);
+                const uint64_t a0 = d_kq0 + (uint64_t)(c % NSTAGE) * STAGE_STEP;
 #pragma unroll
-                for (int s = 0; s < KSTEPS; ++s) {
-                    const uint32_t off = (uint32_t)((s / 4) * 16384 + (s % 4) * 32);
-                    mma_bf16_ss(tmem + TM_D1, smem_desc_sw128(a0 + off, 16, 1024), smem_desc_sw128(a0 + off, 16, 1024), ID_G, s > 0);
-                }
+                for (int s = 0; s < KSTEPS; ++s) mma_bf16_ss(tmem + TM_D1, a0 + kstep(s), a0 + kstep(s), ID_G, s > 0);
                 mma_commit(&sm.bar[B_D1_DONE]);
             };
             bool ok = true;
@@ -268,7 +298,8 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             }
             for (int c = 0; ok && c < nchunks; ++c) {
                 const uint32_t ph = (uint32_t)(c & 1);
-                const uint32_t k0 = smem_u32(sm.kq[c % NSTAGE]);
+                const uint64_t k0 = d_kq0 + (uint64_t)(c % NSTAGE) * STAGE_STEP;
+                const uint64_t kt0 = d_kt0 + (uint64_t)(c % NSTAGE) * STAGE_STEP;
                 // MMA-1(c+1): as early as its inputs and the D1 buffer allow
                 if (c + 1 < nchunks) {
                     if (!(ok = wait(B_FULL0 + (c + 1) % NSTAGE, (uint32_t)(((c + 1) / NSTAGE) & 1)))) break;
@@ -278,75 +309,61 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     tc_fence_after();
                     mma1(c + 1);
                 }
-                // MMA-2(c): K S_0 -> TM_KS, Q S_0 -> TM_QS[c&1]
+                KLA_TR(0, c, 0);
+                // MMA-2(c): K S_0 -> TM_KS (on the chain), then Q S_0 -> TM_QS[c&1] (needed only for the outputs)
                 if (!(ok = wait(B_S_READY, ph))) break;
+                KLA_TR(0, c, 1);
                 tc_fence_after();
                 {
-                    const uint32_t bh = smem_u32(sm.s_hi), bl = smem_u32(sm.s_lo);
+#pragma unroll
+                    for (int s = 0; s < KSTEPS; ++s) mma_bf16_ss(tmem + TM_KS, k0 + kstep(s), d_sh + (uint64_t)(s * 128), ID_S, s > 0);
+#pragma unroll
+                    for (int s = 0; s < KSTEPS; ++s) mma_bf16_ss(tmem + TM_KS, k0 + kstep(s), d_sl + (uint64_t)(s * 128), ID_S, 1);
+                    mma_commit(&sm.bar[B_D2_DONE]);
                     const uint32_t tq = tmem + ((c & 1) ? TM_QS1 : TM_QS0);
 #pragma unroll
-                    for (int half = 0; half < 2; ++half) {
-                        const uint32_t b0 = half ? bl : bh;
+                    for (int s = 0; s < KSTEPS; ++s) mma_bf16_ss(tq, k0 + 512 + kstep(s), d_sh + (uint64_t)(s * 128), ID_S, s > 0);
 #pragma unroll
-                        for (int s = 0; s < KSTEPS; ++s) {
-                            const uint32_t off = (uint32_t)((s / 4) * 16384 + (s % 4) * 32);
-                            mma_bf16_ss(tmem + TM_KS, smem_desc_sw128(k0 + off, 16, 1024), smem_desc_sw128(b0 + s * 2048, 16, 1024), ID_S, (half | s) > 0);
-                        }
-                    }
-#pragma unroll
-                    for (int half = 0; half < 2; ++half) {
-                        const uint32_t b0 = half ? bl : bh;
-#pragma unroll
-                        for (int s = 0; s < KSTEPS; ++s) {
-                            const uint32_t off = (uint32_t)((s / 4) * 16384 + (s % 4) * 32 + 8192);
-                            mma_bf16_ss(tq, smem_desc_sw128(k0 + off, 16, 1024), smem_desc_sw128(b0 + s * 2048, 16, 1024), ID_S, (half | s) > 0);
-                        }
-                    }
-                    mma_commit(&sm.bar[B_D2_DONE]);
+                    for (int s = 0; s < KSTEPS; ++s) mma_bf16_ss(tq, k0 + 512 + kstep(s), d_sl + (uint64_t)(s * 128), ID_S, 1);
                 }
+                KLA_TR(0, c, 2);
                 // MMA-3(c): U = T rhs
                 if (!(ok = wait(B_TP_READY, ph))) break;
+                KLA_TR(0, c, 3);
                 if (!(ok = wait(B_RHS_READY, ph))) break;
+                KLA_TR(0, c, 4);
                 tc_fence_after();
                 {
-                    const uint32_t th = smem_u32(sm.t_hi), tl = smem_u32(sm.t_lo), rh = smem_u32(sm.ru_hi), rl = smem_u32(sm.ru_lo);
 #pragma unroll
-                    for (int s = 0; s < 4; ++s)
-                        mma_bf16_ss(tmem + TM_U, smem_desc_sw128(th + s * 32, 16, 1024), smem_desc_sw128(rh + s * 2048, 16, 1024), ID_S, s > 0);
+                    for (int s = 0; s < 4; ++s) mma_bf16_ss(tmem + TM_U, d_th + (uint64_t)(s * 2), d_rh + (uint64_t)(s * 128), ID_S, s > 0);
 #pragma unroll
-                    for (int s = 0; s < 4; ++s)
-                        mma_bf16_ss(tmem + TM_U, smem_desc_sw128(th + s * 32, 16, 1024), smem_desc_sw128(rl + s * 2048, 16, 1024), ID_S, 1);
+                    for (int s = 0; s < 4; ++s) mma_bf16_ss(tmem + TM_U, d_th + (uint64_t)(s * 2), d_rl + (uint64_t)(s * 128), ID_S, 1);
 #pragma unroll
-                    for (int s = 0; s < 4; ++s)
-                        mma_bf16_ss(tmem + TM_U, smem_desc_sw128(tl + s * 32, 16, 1024), smem_desc_sw128(rh + s * 2048, 16, 1024), ID_S, 1);
+                    for (int s = 0; s < 4; ++s) mma_bf16_ss(tmem + TM_U, d_tl + (uint64_t)(s * 2), d_rh + (uint64_t)(s * 128), ID_S, 1);
                     mma_commit(&sm.bar[B_D3_DONE]);
                 }
+                KLA_TR(0, c, 5);
                 // MMA-5(c): K^T (D U)   then   MMA-4(c): P U
                 if (!(ok = wait(B_U_READY, ph))) break;
+                KLA_TR(0, c, 6);
                 tc_fence_after();
                 {
-                    const uint32_t dh = smem_u32(sm.du_hi), dl = smem_u32(sm.du_lo);
                     // A = K^T: M = d_k (64-wide blocks KB*8192 bytes apart; for d_k = 64 the second block
                     // is the Q tile, whose rows land in TMEM lanes 64..127 and are ignored), K = tokens
 #pragma unroll
-                    for (int s = 0; s < 4; ++s)
-                        mma_bf16_ss(tmem + TM_DS, smem_desc_sw128(k0 + s * 2048, KB * 8192, 1024), smem_desc_sw128(dh + s * 2048, 16, 1024), ID_DS, s > 0);
+                    for (int s = 0; s < 4; ++s) mma_bf16_ss(tmem + TM_DS, kt0 + (uint64_t)(s * 128), d_dh + (uint64_t)(s * 128), ID_DS, s > 0);
 #pragma unroll
-                    for (int s = 0; s < 4; ++s)
-                        mma_bf16_ss(tmem + TM_DS, smem_desc_sw128(k0 + s * 2048, KB * 8192, 1024), smem_desc_sw128(dl + s * 2048, 16, 1024), ID_DS, 1);
+                    for (int s = 0; s < 4; ++s) mma_bf16_ss(tmem + TM_DS, kt0 + (uint64_t)(s * 128), d_dl + (uint64_t)(s * 128), ID_DS, 1);
                     mma_commit(&sm.bar[B_D5_DONE]);
-                    const uint32_t phh = smem_u32(sm.p_hi), pl = smem_u32(sm.p_lo), uh = smem_u32(sm.ru_hi), ul = smem_u32(sm.ru_lo);
 #pragma unroll
-                    for (int s = 0; s < 4; ++s)
-                        mma_bf16_ss(tmem + TM_PU, smem_desc_sw128(phh + s * 32, 16, 1024), smem_desc_sw128(uh + s * 2048, 16, 1024), ID_S, s > 0);
+                    for (int s = 0; s < 4; ++s) mma_bf16_ss(tmem + TM_PU, d_ph + (uint64_t)(s * 2), d_rh + (uint64_t)(s * 128), ID_S, s > 0);
 #pragma unroll
-                    for (int s = 0; s < 4; ++s)
-                        mma_bf16_ss(tmem + TM_PU, smem_desc_sw128(phh + s * 32, 16, 1024), smem_desc_sw128(ul + s * 2048, 16, 1024), ID_S, 1);
+                    for (int s = 0; s < 4; ++s) mma_bf16_ss(tmem + TM_PU, d_ph + (uint64_t)(s * 2), d_rl + (uint64_t)(s * 128), ID_S, 1);
 #pragma unroll
-                    for (int s = 0; s < 4; ++s)
-                        mma_bf16_ss(tmem + TM_PU, smem_desc_sw128(pl + s * 32, 16, 1024), smem_desc_sw128(uh + s * 2048, 16, 1024), ID_S, 1);
+                    for (int s = 0; s < 4; ++s) mma_bf16_ss(tmem + TM_PU, d_pl + (uint64_t)(s * 2), d_rh + (uint64_t)(s * 128), ID_S, 1);
                     mma_commit(&sm.bar[B_D4_DONE]);
                 }
+                KLA_TR(0, c, 7);
                 // the K/Q stage of chunk c is free once MMA-5(c) has read it
                 if (c + NSTAGE < nchunks) {
                     if (!(ok = wait(B_D5_DONE, ph))) break;
@@ -356,31 +373,59 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         }
     } else if (warp < PG_T / 32) {
         // =============================== pre group ==========================================================
-        const int pt = tid;  // 0..127
-        float la_next = 0.f, eta_next = 0.f;
-        if (pt < C) {
-            const bool valid = pt < len;
-            la_next = valid ? p.log_alpha[(size_t)(tok0 + pt) * p.H + h] : 0.f;
-            eta_next = valid ? p.eta[(size_t)(tok0 + pt) * p.H + h] : 0.f;
-        }
+        const int pt = tid;                       // 0..255
+        const int q = warp & 3, chh = warp >> 2;  // TMEM lane quadrant, column half of D1
+        const int lrow = q * 32 + lane;           // D1 row held by this thread: G row (< 64) or Q K^T row
+        const bool is_g = lrow < 64;
+        const int i = lrow & 63;
+        const int nrow = pt >> 2, npart = pt & 3; // norm work: 4 threads per token
+        const bool scan_warp = warp == PG_T / 32 - 1;
+        float la_next0 = 0.f, la_next1 = 0.f, eta_next = 0.f;
+        auto fetch_gates = [&](int c) {
+            if (scan_warp) {
+                const int t = c * C + 2 * lane;
+                la_next0 = (t < len) ? p.log_alpha[(size_t)(tok0 + t) * p.H + h] : 0.f;
+                la_next1 = (t + 1 < len) ? p.log_alpha[(size_t)(tok0 + t + 1) * p.H + h] : 0.f;
+            }
+            if (npart == 0) {
+                const int t = c * C + nrow;
+                eta_next = (t < len) ? p.eta[(size_t)(tok0 + t) * p.H + h] : 0.f;
+            }
+        };
+        fetch_gates(0);
         for (int c = 0; c < nchunks; ++c) {
             const uint32_t ph = (uint32_t)(c & 1);
             const int rows = (c == nchunks - 1) ? last_rows : C;
             const int sc = c % NSTAGE;
-            const float la_cur = la_next, eta_cur = eta_next;
-            if (pt < C && c + 1 < nchunks) {
-                const int t = (c + 1) * C + pt;
-                const bool valid = t < len;
-                la_next = valid ? p.log_alpha[(size_t)(tok0 + t) * p.H + h] : 0.f;
-                eta_next = valid ? p.eta[(size_t)(tok0 + t) * p.H + h] : 0.f;
+            const float la0 = la_next0, la1 = la_next1, eta_cur = eta_next;
+            if (c + 1 < nchunks) fetch_gates(c + 1);
+            // ---- g_i, gamma_i, exp(g_C - g_i): fp64 scan by one warp (needs no tile) -----------------------------
+            if (scan_warp) {
+                const double v0 = (double)la0, v1 = (double)la1;
+                const double run = v0 + v1;
+                double incl = run;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const double t = __shfl_up_sync(0xffffffffu, incl, o);
+                    if (lane >= o) incl += t;
+                }
+                const double gC = __shfl_sync(0xffffffffu, incl, 31);
+                const double ga = incl - v1, gb = incl;
+                const float a2 = (float)(ga * (double)LOG2E), b2 = (float)(gb * (double)LOG2E);
+                *reinterpret_cast<float2 *>(&sm.g2[2 * lane]) = make_float2(a2, b2);
+                *reinterpret_cast<float2 *>(&sm.gam[sc][2 * lane]) = make_float2(ex2_approx(a2), ex2_approx(b2));
+                *reinterpret_cast<float2 *>(&sm.dec[sc][2 * lane]) =
+                    make_float2(ex2_approx((float)((gC - ga) * (double)LOG2E)), ex2_approx((float)((gC - gb) * (double)LOG2E)));
             }
+            KLA_TR(1, c, 0);
             if (pg_any(!wait(B_FULL0 + sc, (uint32_t)((c / NSTAGE) & 1)))) break;
+            KLA_TR(1, c, 1);
             unsigned char *kq = sm.kq[sc];
             if (rows < C) {
                 // last chunk: rows past the end of the sequence hold a neighbour's tokens (or TMA zero
                 // fill); zero them so that they are inert in every product
-                for (int i = pt; i < (C - rows) * 8; i += PG_T) {
-                    const int r = rows + i / 8, ch = i % 8;
+                for (int e = pt; e < (C - rows) * 8; e += PG_T) {
+                    const int r = rows + e / 8, ch = e % 8;
                     const uint4 z = make_uint4(0, 0, 0, 0);
 #pragma unroll
                     for (int kb = 0; kb < KB; ++kb) {
@@ -391,163 +436,155 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 fence_async_smem();
                 warp_arrive(B_TAIL_READY);
             }
-            // ---- beta_i, g_i, gamma_i, exp(g_C - g_i) ------------------------------------------------------
-            if (pt < C) {
-                float nk = 0.f;
-                if (pt < rows) {
+            // ---- beta_i = eta_i / (||k_i||^2 + eps): 4 threads per token ------------------------------------------
+            {
+                float n0 = 0.f, n1 = 0.f;
+                if (nrow < rows) {
 #pragma unroll
                     for (int kb = 0; kb < KB; ++kb)
 #pragma unroll
-                        for (int ch = 0; ch < 8; ++ch) {
-                            const uint4 raw = *reinterpret_cast<const uint4 *>(kq + kb * 16384 + sw128(pt, ch));
+                        for (int cc = 0; cc < 2; ++cc) {
+                            const uint4 raw = *reinterpret_cast<const uint4 *>(kq + kb * 16384 + sw128(nrow, npart * 2 + cc));
                             const __nv_bfloat162 *h2 = reinterpret_cast<const __nv_bfloat162 *>(&raw);
-#pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                const float2 f = __bfloat1622float2(h2[e]);
-                                nk += f.x * f.x + f.y * f.y;
-                            }
+                            const float2 f0 = __bfloat1622float2(h2[0]), f1 = __bfloat1622float2(h2[1]);
+                            const float2 f2 = __bfloat1622float2(h2[2]), f3 = __bfloat1622float2(h2[3]);
+                            n0 += f0.x * f0.x + f0.y * f0.y + f2.x * f2.x + f2.y * f2.y;
+                            n1 += f1.x * f1.x + f1.y * f1.y + f3.x * f3.x + f3.y * f3.y;
                         }
                 }
-                sm.beta[sc][pt] = (pt < rows) ? eta_cur / (nk + p.eps) : 0.f;
-                sm.la[pt] = la_cur;
+                float nk = n0 + n1;
+                nk += __shfl_xor_sync(0xffffffffu, nk, 1);
+                nk += __shfl_xor_sync(0xffffffffu, nk, 2);
+                if (npart == 0) sm.beta[sc][nrow] = (nrow < rows) ? eta_cur / (nk + p.eps) : 0.f;
             }
             pg_sync();
-            if (warp == 2) {
-                // inclusive scan of the 64 log-decays in fp64 (differences g_i - g_j must not cancel)
-                const double v0 = (double)sm.la[2 * lane], v1 = (double)sm.la[2 * lane + 1];
-                const double run = v0 + v1;
-                double incl = run;
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    const double t = __shfl_up_sync(0xffffffffu, incl, o);
-                    if (lane >= o) incl += t;
-                }
-                const double excl = incl - run;
-                sm.g[2 * lane] = excl + v0;
-                sm.g[2 * lane + 1] = excl + run;
-            }
-            pg_sync();
-            if (pt < C) {
-                const double gC = sm.g[C - 1];
-                sm.gam[sc][pt] = __expf((float)sm.g[pt]);
-                sm.dec[sc][pt] = __expf((float)(gC - sm.g[pt]));
-            }
-            // ---- L (lanes 0..63) and P (lanes 64..127) from MMA-1 -------------------------------------------
+            KLA_TR(1, c, 2);
+            // ---- L (lanes 0..63) and P (lanes 64..127) from MMA-1; this thread: row i, 32 columns ---------------------
             if (pg_any(!wait(B_D1_DONE, ph))) break;
+            KLA_TR(1, c, 3);
             tc_fence_after();
-            uint32_t p_hi[32], p_lo[32];  // this thread's P row, packed bf16 pairs (warps 2, 3 only)
+            uint32_t p_hi[16], p_lo[16];  // this thread's half P row, packed bf16 pairs (Q K^T rows only)
             {
-                const int i = pt & 63;
-                const double gi = sm.g[i];
+                const float gi2 = sm.g2[i];
                 const float bi = sm.beta[sc][i];
                 float acc[32];
+                tmem_ld32(tm_lane + TM_D1 + chh * 32, acc);
 #pragma unroll
-                for (int half = 0; half < 2; ++half) {
-                    tmem_ld32(tm_lane + TM_D1 + half * 32, acc);
-                    if (pt < 64) {
-#pragma unroll
-                        for (int q4 = 0; q4 < 8; ++q4) {
-                            float4 o;
-                            float *of = reinterpret_cast<float *>(&o);
-#pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                const int j = half * 32 + q4 * 4 + e;
-                                of[e] = (j < i) ? bi * __expf((float)(gi - sm.g[j])) * acc[q4 * 4 + e] : 0.f;
-                            }
-                            *reinterpret_cast<float4 *>(&sm.tl[i * LDT + half * 32 + q4 * 4]) = o;
-                        }
+                for (int j4 = 0; j4 < 8; ++j4) {
+                    const float4 gj = *reinterpret_cast<const float4 *>(&sm.g2[chh * 32 + 4 * j4]);
+                    const int j = chh * 32 + 4 * j4;
+                    const float e0 = ex2_approx(gi2 - gj.x), e1 = ex2_approx(gi2 - gj.y);
+                    const float e2 = ex2_approx(gi2 - gj.z), e3 = ex2_approx(gi2 - gj.w);
+                    if (is_g) {
+                        float4 o;
+                        o.x = (j + 0 < i) ? bi * e0 * acc[4 * j4 + 0] : 0.f;
+                        o.y = (j + 1 < i) ? bi * e1 * acc[4 * j4 + 1] : 0.f;
+                        o.z = (j + 2 < i) ? bi * e2 * acc[4 * j4 + 2] : 0.f;
+                        o.w = (j + 3 < i) ? bi * e3 * acc[4 * j4 + 3] : 0.f;
+                        *reinterpret_cast<float4 *>(&sm.tl[i * LDT + j]) = o;
                     } else {
-#pragma unroll
-                        for (int e2 = 0; e2 < 16; ++e2) {
-                            const int j = half * 32 + 2 * e2;
-                            const float a = (j <= i) ? __expf((float)(gi - sm.g[j])) * acc[2 * e2] : 0.f;
-                            const float b = (j + 1 <= i) ? __expf((float)(gi - sm.g[j + 1])) * acc[2 * e2 + 1] : 0.f;
-                            split2(a, b, p_hi[half * 16 + e2], p_lo[half * 16 + e2]);
-                        }
+                        const float a0 = (j + 0 <= i) ? e0 * acc[4 * j4 + 0] : 0.f;
+                        const float a1 = (j + 1 <= i) ? e1 * acc[4 * j4 + 1] : 0.f;
+                        const float a2 = (j + 2 <= i) ? e2 * acc[4 * j4 + 2] : 0.f;
+                        const float a3 = (j + 3 <= i) ? e3 * acc[4 * j4 + 3] : 0.f;
+                        split2(a0, a1, p_hi[2 * j4], p_lo[2 * j4]);
+                        split2(a2, a3, p_hi[2 * j4 + 1], p_lo[2 * j4 + 1]);
                     }
                 }
             }
             tc_fence_before();
             warp_arrive(B_D1_FREE);
+            pg_sync();
+            KLA_TR(1, c, 4);
 
             // ---- T = (I + L)^-1, blocked: 16x16 diagonal blocks, then 16x16 and 32x32 off-diagonal blocks ------
             if (pt < 64) {
-                pg_half_sync();  // L rows written by warps 0, 1
                 const int blk = pt >> 4, j = pt & 15;
                 const float *Lb = sm.tl + (blk * 16) * LDT + blk * 16;
                 float x[16];
 #pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    float s0 = 0.f, s1 = 0.f;
+                for (int r = 0; r < 16; ++r) {
+                    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
 #pragma unroll
-                    for (int m = 0; m < i; m += 2) {
-                        s0 += Lb[i * LDT + m] * x[m];
-                        if (m + 1 < i) s1 += Lb[i * LDT + m + 1] * x[m + 1];
+                    for (int m4 = 0; m4 < r; m4 += 4) {
+                        const float4 l4 = *reinterpret_cast<const float4 *>(Lb + r * LDT + m4);
+                        s0 += l4.x * x[m4];
+                        if (m4 + 1 < r) s1 += l4.y * x[m4 + 1];
+                        if (m4 + 2 < r) s2 += l4.z * x[m4 + 2];
+                        if (m4 + 3 < r) s3 += l4.w * x[m4 + 3];
                     }
-                    x[i] = (i == j) ? 1.f : ((i > j) ? -(s0 + s1) : 0.f);
+                    x[r] = (r == j) ? 1.f : ((r > j) ? -((s0 + s1) + (s2 + s3)) : 0.f);
                 }
                 pg_half_sync();  // every column of the block has read L_bb
                 float *Tb = sm.tl + (blk * 16) * LDT + blk * 16;
 #pragma unroll
-                for (int i = 0; i < 16; ++i) Tb[i * LDT + j] = x[i];
+                for (int r = 0; r < 16; ++r) Tb[r * LDT + j] = x[r];
             }
             pg_sync();
+            KLA_TR(1, c, 5);
             {
                 // level 1: M = L10 T00 and L32 T22 (16x16 each); then T10 = -T11 M, T32 = -T33 M
-                const int prod = pt >> 6, r = (pt & 63) >> 2, c4 = (pt & 3) * 4;
+                const int prod = pt >> 7, r = (pt & 127) >> 3, c2 = (pt & 7) * 2;
                 const int rb = prod ? 48 : 16, cb = prod ? 32 : 0;
-                tile_mm<1>(sm.mm + prod * 16 * LDM, LDM, sm.tl + rb * LDT + cb, LDT, sm.tl + cb * LDT + cb, LDT, r, c4, 16, true, false, 1.f);
+                row_mm<16, 2>(sm.mm + prod * 16 * LDM, LDM, sm.tl + rb * LDT + cb, LDT, sm.tl + cb * LDT + cb, LDT, r, c2, true, false, 1.f);
                 pg_sync();
-                tile_mm<1>(sm.tl + rb * LDT + cb, LDT, sm.tl + rb * LDT + rb, LDT, sm.mm + prod * 16 * LDM, LDM, r, c4, 16, false, true, -1.f);
+                row_mm<16, 2>(sm.tl + rb * LDT + cb, LDT, sm.tl + rb * LDT + rb, LDT, sm.mm + prod * 16 * LDM, LDM, r, c2, false, true, -1.f);
                 pg_sync();
             }
+            KLA_TR(1, c, 6);
             {
                 // level 2: M = L[32..63][0..31] T[0..31][0..31]; T[32..63][0..31] = -T[32..63][32..63] M
-                const int r0 = (pt >> 3) * 2, c4 = (pt & 7) * 4;
-                tile_mm<2>(sm.mm, LDM, sm.tl + 32 * LDT, LDT, sm.tl, LDT, r0, c4, 32, true, false, 1.f);
+                const int r = pt >> 3, c4 = (pt & 7) * 4;
+                row_mm<32, 4>(sm.mm, LDM, sm.tl + 32 * LDT, LDT, sm.tl, LDT, r, c4, true, false, 1.f);
                 pg_sync();
-                tile_mm<2>(sm.tl + 32 * LDT, LDT, sm.tl + 32 * LDT + 32, LDT, sm.mm, LDM, r0, c4, 32, false, true, -1.f);
+                row_mm<32, 4>(sm.tl + 32 * LDT, LDT, sm.tl + 32 * LDT + 32, LDT, sm.mm, LDM, r, c4, false, true, -1.f);
                 pg_sync();
             }
             // ---- write T (after MMA-3(c-1) has read the previous one) and P (after MMA-4(c-1)) ----------------------
+            KLA_TR(1, c, 7);
             if (c > 0 && pg_any(!wait(B_D3_DONE, ph ^ 1))) break;
+            KLA_TR(1, c, 8);
             {
-                const int i = pt >> 1, half = pt & 1;
+                const int r = pt >> 2, qq = pt & 3;  // row, 16-column quarter
 #pragma unroll
-                for (int ch = 0; ch < 4; ++ch) {
-                    const float4 a = *reinterpret_cast<const float4 *>(&sm.tl[i * LDT + half * 32 + ch * 8]);
-                    const float4 b = *reinterpret_cast<const float4 *>(&sm.tl[i * LDT + half * 32 + ch * 8 + 4]);
+                for (int ch = 0; ch < 2; ++ch) {
+                    const float4 a = *reinterpret_cast<const float4 *>(&sm.tl[r * LDT + qq * 16 + ch * 8]);
+                    const float4 b = *reinterpret_cast<const float4 *>(&sm.tl[r * LDT + qq * 16 + ch * 8 + 4]);
                     uint4 hi, lo;
                     split2(a.x, a.y, hi.x, lo.x);
                     split2(a.z, a.w, hi.y, lo.y);
                     split2(b.x, b.y, hi.z, lo.z);
                     split2(b.z, b.w, hi.w, lo.w);
-                    *reinterpret_cast<uint4 *>(sm.t_hi + sw128(i, half * 4 + ch)) = hi;
-                    *reinterpret_cast<uint4 *>(sm.t_lo + sw128(i, half * 4 + ch)) = lo;
+                    *reinterpret_cast<uint4 *>(sm.t_hi + sw128(r, qq * 2 + ch)) = hi;
+                    *reinterpret_cast<uint4 *>(sm.t_lo + sw128(r, qq * 2 + ch)) = lo;
                 }
             }
+            KLA_TR(1, c, 9);
             if (c > 0 && pg_any(!wait(B_D4_DONE, ph ^ 1))) break;
-            if (pt >= 64) {
-                const int i = pt - 64;
+            KLA_TR(1, c, 10);
+            if (!is_g) {
 #pragma unroll
-                for (int ch = 0; ch < 8; ++ch) {
-                    *reinterpret_cast<uint4 *>(sm.p_hi + sw128(i, ch)) = make_uint4(p_hi[4 * ch], p_hi[4 * ch + 1], p_hi[4 * ch + 2], p_hi[4 * ch + 3]);
-                    *reinterpret_cast<uint4 *>(sm.p_lo + sw128(i, ch)) = make_uint4(p_lo[4 * ch], p_lo[4 * ch + 1], p_lo[4 * ch + 2], p_lo[4 * ch + 3]);
+                for (int ch = 0; ch < 4; ++ch) {
+                    *reinterpret_cast<uint4 *>(sm.p_hi + sw128(i, chh * 4 + ch)) = make_uint4(p_hi[4 * ch], p_hi[4 * ch + 1], p_hi[4 * ch + 2], p_hi[4 * ch + 3]);
+                    *reinterpret_cast<uint4 *>(sm.p_lo + sw128(i, chh * 4 + ch)) = make_uint4(p_lo[4 * ch], p_lo[4 * ch + 1], p_lo[4 * ch + 2], p_lo[4 * ch + 3]);
                 }
             }
             fence_async_smem();
-            pg_sync();  // the solve matrix is reused by the next chunk
+            pg_sync();  // the solve matrix and g2 are reused by the next chunk
             warp_arrive(B_TP_READY);
+            KLA_TR(1, c, 11);
         }
     } else {
         // =============================== chain group ==========================================================
         const int ct = tid - PG_T;              // 0..255
         const int q = warp & 3;                 // TMEM lane quadrant
         const int hf = ct >> 7;                 // column half: 0 -> columns 0..31, 1 -> 32..63
-        const int srow = q * 32 + lane;         // state row (M = 128 accumulator layout)
+        const int srow = q * 32 + lane;         // state row (M = 128 accumulator layout, 32x32b loads)
         const bool s_act = srow < D;
-        const int i = q * 16 + lane;            // chunk row (M = 64 accumulator layout); valid for lane < 16
-        const bool r_act = lane < 16;
+        // M = 64 accumulators, 16x256b loads: rows i0 and i0 + 8, column pairs cp + 8j (j = 0..3)
+        const int i0 = q * 16 + (lane >> 2), i1 = i0 + 8;
+        const int cp = hf * 32 + 2 * (lane & 3);
+        const uint32_t tm16 = tmem + ((uint32_t)(q * 32) << 16) + hf * 32;
 
         float S[32];
         if (s_act && p.init_state) {
@@ -576,18 +613,22 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             fence_async_smem();
             warp_arrive(B_S_READY);
         };
-        const __nv_bfloat16 *vbase = reinterpret_cast<const __nv_bfloat16 *>(p.v) + (size_t)h * D + sl * NS + hf * 32;
+        // byte offsets of this thread's bf16 pairs inside the 64-token x 64-column B-operand tiles
+        uint32_t off0[4], off1[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            off0[j] = sw128(i0, hf * 4 + j) + 4 * (lane & 3);
+            off1[j] = sw128(i1, hf * 4 + j) + 4 * (lane & 3);
+        }
+        const __nv_bfloat16 *vbase = reinterpret_cast<const __nv_bfloat16 *>(p.v) + (size_t)h * D + sl * NS + cp;
         const size_t tokstride = (size_t)p.H * D;
-        uint4 vreg[4];
+        uint32_t v0[4], v1[4];  // V[i0][cp + 8j .. +1], V[i1][...] as packed bf16 pairs
         auto fetch_v = [&](int c) {
-            const int t = c * C + i;
-            if (r_act && t < len) {
-                const uint4 *src = reinterpret_cast<const uint4 *>(vbase + (size_t)(tok0 + t) * tokstride);
+            const int t0 = c * C + i0, t1 = c * C + i1;
 #pragma unroll
-                for (int u = 0; u < 4; ++u) vreg[u] = src[u];
-            } else {
-#pragma unroll
-                for (int u = 0; u < 4; ++u) vreg[u] = make_uint4(0, 0, 0, 0);
+            for (int j = 0; j < 4; ++j) {
+                v0[j] = (t0 < len) ? *reinterpret_cast<const uint32_t *>(vbase + (size_t)(tok0 + t0) * tokstride + 8 * j) : 0u;
+                v1[j] = (t1 < len) ? *reinterpret_cast<const uint32_t *>(vbase + (size_t)(tok0 + t1) * tokstride + 8 * j) : 0u;
             }
         };
         fetch_v(0);
@@ -598,76 +639,70 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             const int rows = (c == nchunks - 1) ? last_rows : C;
             const int sc = c % NSTAGE;
             // ---- rhs = B (V - D_gamma K S_0) ------------------------------------------------------------------
+            KLA_TR(2, c, 0);
             if (!wait(B_TP_READY, ph)) break;   // scalars of chunk c
-            if (!wait(B_D2_DONE, ph)) break;
-            tc_fence_after();
-            float bi = 0.f, gi = 0.f, di = 0.f;
-            if (r_act) {
-                bi = sm.beta[sc][i];
-                gi = sm.gam[sc][i];
-                di = sm.dec[sc][i];
-            }
+            KLA_TR(2, c, 1);
+            const float b0 = sm.beta[sc][i0], b1 = sm.beta[sc][i1];
+            const float g0 = sm.gam[sc][i0], g1 = sm.gam[sc][i1];
+            const float d0 = sm.dec[sc][i0], d1 = sm.dec[sc][i1];
             const float gC = sm.gam[sc][C - 1];
+            if (!wait(B_D2_DONE, ph)) break;
+            KLA_TR(2, c, 2);
+            tc_fence_after();
             {
-                float acc[32];
-                tmem_ld32(tm_lane + TM_KS + hf * 32, acc);
-                if (r_act) {
+                float acc[16];
+                tmem_ld16x256b_x4(tm16 + TM_KS, acc);
 #pragma unroll
-                    for (int ch = 0; ch < 4; ++ch) {
-                        const __nv_bfloat162 *h2 = reinterpret_cast<const __nv_bfloat162 *>(&vreg[ch]);
-                        float r[8];
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const float2 f = __bfloat1622float2(h2[e]);
-                            r[2 * e] = bi * (f.x - gi * acc[ch * 8 + 2 * e]);
-                            r[2 * e + 1] = bi * (f.y - gi * acc[ch * 8 + 2 * e + 1]);
-                        }
-                        uint4 hi, lo;
-                        split2(r[0], r[1], hi.x, lo.x);
-                        split2(r[2], r[3], hi.y, lo.y);
-                        split2(r[4], r[5], hi.z, lo.z);
-                        split2(r[6], r[7], hi.w, lo.w);
-                        *reinterpret_cast<uint4 *>(sm.ru_hi + sw128(i, hf * 4 + ch)) = hi;
-                        *reinterpret_cast<uint4 *>(sm.ru_lo + sw128(i, hf * 4 + ch)) = lo;
-                    }
+                for (int j = 0; j < 4; ++j) {
+                    const float2 fa = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&v0[j]));
+                    const float2 fb = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&v1[j]));
+                    uint32_t hi, lo;
+                    split2(b0 * (fa.x - g0 * acc[4 * j]), b0 * (fa.y - g0 * acc[4 * j + 1]), hi, lo);
+                    *reinterpret_cast<uint32_t *>(sm.ru_hi + off0[j]) = hi;
+                    *reinterpret_cast<uint32_t *>(sm.ru_lo + off0[j]) = lo;
+                    split2(b1 * (fb.x - g1 * acc[4 * j + 2]), b1 * (fb.y - g1 * acc[4 * j + 3]), hi, lo);
+                    *reinterpret_cast<uint32_t *>(sm.ru_hi + off1[j]) = hi;
+                    *reinterpret_cast<uint32_t *>(sm.ru_lo + off1[j]) = lo;
                 }
             }
             fence_async_smem();
             tc_fence_before();
             warp_arrive(B_RHS_READY);
+            KLA_TR(2, c, 3);
             if (c + 1 < nchunks) fetch_v(c + 1);
 
             // ---- U and D U as hi/lo operands -------------------------------------------------------------------
             if (!wait(B_D3_DONE, ph)) break;
+            KLA_TR(2, c, 4);
             tc_fence_after();
             {
-                float acc[32];
-                tmem_ld32(tm_lane + TM_U + hf * 32, acc);
-                if (r_act) {
+                float acc[16];
+                tmem_ld16x256b_x4(tm16 + TM_U, acc);
 #pragma unroll
-                    for (int ch = 0; ch < 4; ++ch) {
-                        uint4 hi, lo;
-                        split2(acc[8 * ch + 0], acc[8 * ch + 1], hi.x, lo.x);
-                        split2(acc[8 * ch + 2], acc[8 * ch + 3], hi.y, lo.y);
-                        split2(acc[8 * ch + 4], acc[8 * ch + 5], hi.z, lo.z);
-                        split2(acc[8 * ch + 6], acc[8 * ch + 7], hi.w, lo.w);
-                        *reinterpret_cast<uint4 *>(sm.ru_hi + sw128(i, hf * 4 + ch)) = hi;
-                        *reinterpret_cast<uint4 *>(sm.ru_lo + sw128(i, hf * 4 + ch)) = lo;
-                        split2(di * acc[8 * ch + 0], di * acc[8 * ch + 1], hi.x, lo.x);
-                        split2(di * acc[8 * ch + 2], di * acc[8 * ch + 3], hi.y, lo.y);
-                        split2(di * acc[8 * ch + 4], di * acc[8 * ch + 5], hi.z, lo.z);
-                        split2(di * acc[8 * ch + 6], di * acc[8 * ch + 7], hi.w, lo.w);
-                        *reinterpret_cast<uint4 *>(sm.du_hi + sw128(i, hf * 4 + ch)) = hi;
-                        *reinterpret_cast<uint4 *>(sm.du_lo + sw128(i, hf * 4 + ch)) = lo;
-                    }
+                for (int j = 0; j < 4; ++j) {
+                    uint32_t hi, lo;
+                    split2(acc[4 * j], acc[4 * j + 1], hi, lo);
+                    *reinterpret_cast<uint32_t *>(sm.ru_hi + off0[j]) = hi;
+                    *reinterpret_cast<uint32_t *>(sm.ru_lo + off0[j]) = lo;
+                    split2(acc[4 * j + 2], acc[4 * j + 3], hi, lo);
+                    *reinterpret_cast<uint32_t *>(sm.ru_hi + off1[j]) = hi;
+                    *reinterpret_cast<uint32_t *>(sm.ru_lo + off1[j]) = lo;
+                    split2(d0 * acc[4 * j], d0 * acc[4 * j + 1], hi, lo);
+                    *reinterpret_cast<uint32_t *>(sm.du_hi + off0[j]) = hi;
+                    *reinterpret_cast<uint32_t *>(sm.du_lo + off0[j]) = lo;
+                    split2(d1 * acc[4 * j + 2], d1 * acc[4 * j + 3], hi, lo);
+                    *reinterpret_cast<uint32_t *>(sm.du_hi + off1[j]) = hi;
+                    *reinterpret_cast<uint32_t *>(sm.du_lo + off1[j]) = lo;
                 }
             }
             fence_async_smem();
             tc_fence_before();
             warp_arrive(B_U_READY);
+            KLA_TR(2, c, 5);
 
             // ---- state: S <- gamma_C S + K^T (D U) -----------------------------------------------------------------
             if (!wait(B_D5_DONE, ph)) break;
+            KLA_TR(2, c, 6);
             tc_fence_after();
             {
                 float acc[32];
@@ -679,23 +714,26 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             }
             tc_fence_before();
             if (c + 1 < nchunks) store_state_tiles();
+            KLA_TR(2, c, 7);
 
             // ---- outputs: O_i = gamma_i (Q S_0)_i + (P U)_i (off the chain) -----------------------------------------
             if (!wait(B_D4_DONE, ph)) break;
+            KLA_TR(2, c, 8);
             tc_fence_after();
             {
-                float acc[32], qs[32];
-                tmem_ld32(tm_lane + TM_PU + hf * 32, acc);
-                tmem_ld32(tm_lane + ((c & 1) ? TM_QS1 : TM_QS0) + hf * 32, qs);
-                if (r_act && i < rows) {
-                    OUT *orow = reinterpret_cast<OUT *>(p.out) + ((size_t)(tok0 + c * C + i) * p.H + h) * D + sl * NS + hf * 32;
+                float acc[16], qs[16];
+                tmem_ld16x256b_x4(tm16 + TM_PU, acc);
+                tmem_ld16x256b_x4(tm16 + ((c & 1) ? TM_QS1 : TM_QS0), qs);
+                OUT *o0 = reinterpret_cast<OUT *>(p.out) + ((size_t)(tok0 + c * C + i0) * p.H + h) * D + sl * NS + cp;
+                OUT *o1 = reinterpret_cast<OUT *>(p.out) + ((size_t)(tok0 + c * C + i1) * p.H + h) * D + sl * NS + cp;
 #pragma unroll
-                    for (int e = 0; e < 32; e += 4)
-                        store4(orow + e, make_float4(gi * qs[e] + acc[e], gi * qs[e + 1] + acc[e + 1],
-                                                     gi * qs[e + 2] + acc[e + 2], gi * qs[e + 3] + acc[e + 3]));
+                for (int j = 0; j < 4; ++j) {
+                    if (i0 < rows) store2(o0 + 8 * j, g0 * qs[4 * j] + acc[4 * j], g0 * qs[4 * j + 1] + acc[4 * j + 1]);
+                    if (i1 < rows) store2(o1 + 8 * j, g1 * qs[4 * j + 2] + acc[4 * j + 2], g1 * qs[4 * j + 3] + acc[4 * j + 3]);
                 }
             }
             tc_fence_before();
+            KLA_TR(2, c, 9);
         }
         if (!sm.abort_flag && p.final_state && s_act) {
 #pragma unroll
@@ -761,6 +799,29 @@ cudaError_t launch_t(const ChunkParams &p, cudaStream_t stream)
     if (err != cudaSuccess) return err;
     const int grid = p.n_seq * p.H * (D / NS);
     if (grid == 0) return cudaSuccess;
+#ifdef KLA_TRACE
+    {
+        static long long *tbuf = nullptr;
+        if (!tbuf) cudaMallocManaged(&tbuf, 3 * 64 * 16 * sizeof(long long));
+        memset(tbuf, 0, 3 * 64 * 16 * sizeof(long long));
+        ChunkParams pt = p;
+        pt.trace = tbuf;
+        kern<<<grid, NT, smem, stream>>>(tq, tk, pt);
+        cudaDeviceSynchronize();
+        FILE *f = fopen("gpurun_out/trace.txt", "w");
+        if (f) {
+            for (int r = 0; r < 3; ++r)
+                for (int c = 0; c < 64; ++c) {
+                    fprintf(f, "%d %d", r, c);
+                    for (int e = 0; e < 16; ++e) fprintf(f, " %lld", tbuf[(r * 64 + c) * 16 + e]);
+                    fprintf(f, "\n");
+                }
+            fclose(f);
+        }
+        count_launch(1);
+        return cudaGetLastError();
+    }
+#endif
     kern<<<grid, NT, smem, stream>>>(tq, tk, p);
     count_launch(1);
     return cudaGetLastError();

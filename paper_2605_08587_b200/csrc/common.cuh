@@ -17,6 +17,7 @@ struct ChunkParams {
     float *final_state;       // may be null
     const int32_t *cu_seqlens;  // device, may be null (fixed length)
     int32_t *status_word;       // may be null
+    long long *trace;           // debug builds only (KLA_TRACE): per-event SM clock stamps; else null
     int32_t B, T, H, n_seq;
     float eps;
 };
@@ -71,6 +72,12 @@ __device__ __forceinline__ void store4(__nv_bfloat16 *p, float4 x)
     raw.x = *reinterpret_cast<uint32_t *>(&a);
     raw.y = *reinterpret_cast<uint32_t *>(&b);
     *reinterpret_cast<uint2 *>(p) = raw;
+}
+
+__device__ __forceinline__ void store2(float *p, float a, float b) { *reinterpret_cast<float2 *>(p) = make_float2(a, b); }
+__device__ __forceinline__ void store2(__nv_bfloat16 *p, float a, float b)
+{
+    *reinterpret_cast<__nv_bfloat162 *>(p) = __floats2bfloat162_rn(a, b);
 }
 
 }  // namespace kla

@@ -3,19 +3,20 @@
 //
 // One CTA owns NS = 64 consecutive d_v columns of one (sequence, head) and walks that sequence's
 // chunks (C = 64 tokens) in order.  Its d_k x NS slice of the state stays in registers in fp32 for
-// the whole sequence.  The CTA is warp-specialised (13 warps):
+// the whole sequence.  The CTA is warp-specialised (17 warps), every role a compact loop:
 //
-//   control warp (1 thread)  issues every TMA load and every tcgen05.mma, in a fixed order
-//   pre group   (4 warps)    state-independent work for chunk c+1 while the chain works on chunk c:
-//                            beta, g (Eq. 3, decay sums), L = B (A^- o K K^T), T = (I + L)^-1 by
-//                            blocked forward substitution in shared memory, P = A o Q K^T
+//   control warp             issues every TMA load and every tcgen05.mma, in a fixed order
+//   pre group (8 warps)      state-independent work for chunk c+1 while the chain works on chunk c:
+//                            g (decay sums), beta (Eq. 3, ||k||^2 read off the diagonal of K K^T),
+//                            X = A^- o K K^T, T = (I + B X)^-1 by blocked substitution in shared
+//                            memory, and (half of the warps, one chunk behind) P = A o Q K^T
 //   chain group (8 warps)    the serial dependency over chunks:
 //                            rhs = B (V - D_gamma K S_0), U = T rhs                      (Eq. 7)
 //                            O = D_gamma Q S_0 + P U                                     (Eq. 8)
 //                            S <- gamma_C S_0 + K^T diag(exp(g_C - g_j)) U               (Eq. 9)
 //
 // Tensor-core products per chunk (fp32 accumulation in TMEM):
-//   MMA-1  [K;Q] K^T   M=128   -> G (lanes 0..63) and Q K^T (lanes 64..127)
+//   MMA-1  [K;Q] K^T   M=128   -> K K^T (lanes 0..63) and Q K^T (lanes 64..127), double-buffered
 //   MMA-2  K S_0, Q S_0        two M=64 products, S_0 = S_hi + S_lo
 //   MMA-3  T rhs       M=64    T_hi rhs_hi + T_hi rhs_lo + T_lo rhs_hi
 //   MMA-4  P U         M=64    same three-term form
@@ -25,11 +26,17 @@
 // carried as a pair of bf16 values hi + lo (16 significand bits): a single bf16 rounding of any of
 // them costs 1e-2..7e-2 in max|err|/rms on the layer-shaped workloads, far above the 2e-3 bound.
 //
+// Code size matters here: a role whose per-chunk code is one long unrolled stream runs at the speed
+// of instruction fetch (measured: three times slower than the same code resident in the instruction
+// cache), so loops are kept rolled wherever register arrays do not force unrolling, and the bounded
+// barrier wait is one out-of-line function.
+//
 // Every wait on an mbarrier is bounded; when one gives up the CTA raises an abort flag, reports
 // KLA_ERR_TIMEOUT through the status word, releases its TMEM and exits.
 #include <cuda.h>
 
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 
@@ -51,25 +58,27 @@ constexpr long long WAIT_LIMIT = 2000000000LL;  // SM clocks (~1 s) before a wai
 constexpr float LOG2E = 1.4426950408889634f;
 
 // TMEM columns (fp32, 128 lanes each)
-constexpr uint32_t TM_D1 = 0, TM_KS = 64, TM_QS0 = 128, TM_QS1 = 192, TM_U = 256, TM_PU = 320, TM_DS = 384, TM_COLS = 512;
+constexpr uint32_t TM_D1 = 0 /* two buffers of 64 */, TM_KS = 128, TM_QS0 = 192, TM_QS1 = 256, TM_U = 320, TM_PU = 384,
+                   TM_DS = 448, TM_COLS = 512;
 
 constexpr int LDT = 68;  // row stride (floats) of the fp32 solve matrix
-constexpr int LDM = 36;  // row stride of the solve scratch
+constexpr int LDM = 40;  // row stride of the solve scratch
 
 enum Bar {
     B_FULL0 = 0,             // +stage: TMA landed
-    B_D1_DONE = 3,           // MMA-1(c) complete
-    B_D1_FREE = 4,           // pre group finished reading D1(c)
-    B_TP_READY = 5,          // T(c), P(c), scalars(c) written
-    B_S_READY = 6,           // state tiles for chunk c written
-    B_D2_DONE = 7,           // K S_0 of chunk c complete
-    B_RHS_READY = 8,
-    B_D3_DONE = 9,
-    B_U_READY = 10,
-    B_D5_DONE = 11,
-    B_D4_DONE = 12,          // P U (and, earlier in the pipe, Q S_0) of chunk c complete
-    B_TAIL_READY = 13,       // masked rows of the last chunk zeroed
-    B_COUNT = 14
+    B_D1_DONE0 = 3,          // +buffer: MMA-1 complete
+    B_D1_FREE0 = 5,          // +buffer: every pre warp finished reading that D1 buffer
+    B_T_READY = 7,           // T(c) and the scalars of chunk c written
+    B_P_READY = 8,           // P(c) written
+    B_S_READY = 9,           // state tiles for chunk c written
+    B_D2_DONE = 10,          // K S_0 of chunk c complete
+    B_RHS_READY = 11,
+    B_D3_DONE = 12,
+    B_U_READY = 13,
+    B_D5_DONE = 14,
+    B_D4_DONE = 15,          // P U (and, earlier in the pipe, Q S_0) of chunk c complete
+    B_TAIL_READY = 16,       // masked rows of the last chunk zeroed
+    B_COUNT = 17
 };
 
 template <int D>
@@ -88,9 +97,9 @@ struct TcSmem {
     alignas(1024) unsigned char ru_lo[8192];
     alignas(1024) unsigned char du_hi[8192];    // diag(exp(g_C - g_j)) U
     alignas(1024) unsigned char du_lo[8192];
-    alignas(16) float tl[64 * LDT];             // L, overwritten in place by T = (I + L)^-1
-    alignas(16) float mm[32 * LDM];             // scratch for the block products of the solve
-    alignas(16) float g2[64];                   // log2(e) * chunk-local running sum of log alpha
+    alignas(16) float tl[64 * LDT];             // X = A^- o K K^T, overwritten in place by T = (I + B X)^-1
+    alignas(16) float mm[32 * LDM];             // scratch for the block products of the inverse
+    alignas(16) float g2[NSTAGE][64];           // log2(e) * chunk-local running sum of log alpha
     float beta[NSTAGE][64];
     float gam[NSTAGE][64];                      // exp(g_i)
     float dec[NSTAGE][64];                      // exp(g_C - g_i)
@@ -99,46 +108,27 @@ struct TcSmem {
     volatile int abort_flag;
 };
 
-// ---- small fp32 block products on shared memory, used by the triangular solve ------------------------
-// Cm[r][c4..c4+CW) = sign * sum_k A[r][k] * Bm[k][c4..c4+CW) for one row r; K is a compile-time bound.
-// b_lower: Bm is lower triangular (Bm[k][c] = 0 for k < c)  -> terms with k < c4 are skipped
-// a_lower: A  is lower triangular (A[r][k]  = 0 for k > r)  -> terms with k > r are skipped
-template <int K, int CW>
-__device__ __forceinline__ void row_mm(float *Cm, int ldc, const float *A, int lda, const float *Bm, int ldb, int r,
-                                       int c4, bool b_lower, bool a_lower, float sign)
+// Bounded wait on an mbarrier phase that also leaves when another role has aborted.  Every lane of the
+// calling warp polls: letting one lane poll and broadcasting the result splits the warp, and each later
+// warp-collective instruction (elect.sync, tcgen05.ld) then pays for re-forming it.
+__device__ __noinline__ bool bar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag)
 {
-    float acc[CW];
-#pragma unroll
-    for (int e = 0; e < CW; ++e) acc[e] = 0.f;
-    const int k0 = b_lower ? c4 : 0;
-    const int k1 = a_lower ? (r + 1) : K;
-#pragma unroll
-    for (int kk = 0; kk < K; kk += 4) {
-        if (kk + 4 > k0 && kk < k1) {
-            const float4 a = *reinterpret_cast<const float4 *>(A + r * lda + kk);
-            const float av[4] = {a.x, a.y, a.z, a.w};
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int k = kk + u;
-                // zero operands outside the triangular ranges contribute exact zeros; no predicate needed
-                if (CW == 4) {
-                    const float4 b = *reinterpret_cast<const float4 *>(Bm + k * ldb + c4);
-                    acc[0] += av[u] * b.x; acc[1] += av[u] * b.y; acc[2] += av[u] * b.z; acc[3] += av[u] * b.w;
-                } else {
-                    const float2 b = *reinterpret_cast<const float2 *>(Bm + k * ldb + c4);
-                    acc[0] += av[u] * b.x; acc[1] += av[u] * b.y;
-                }
-            }
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (true) {
+#pragma unroll 1
+        for (int i = 0; i < 32; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (clock64() - t0 > WAIT_LIMIT) {
+            *abort_flag = 1;
+            return false;
         }
     }
-    if (CW == 4)
-        *reinterpret_cast<float4 *>(Cm + r * ldc + c4) = make_float4(sign * acc[0], sign * acc[1], sign * acc[2], sign * acc[3]);
-    else
-        *reinterpret_cast<float2 *>(Cm + r * ldc + c4) = make_float2(sign * acc[0], sign * acc[1]);
 }
 
 __device__ __forceinline__ void pg_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
-__device__ __forceinline__ void pg_half_sync() { asm volatile("bar.sync 2, 64;" ::: "memory"); }
+__device__ __forceinline__ void half_sync() { asm volatile("bar.sync 3, 64;" ::: "memory"); }
 // Barrier over the pre group that also ORs a flag: makes "some thread's wait gave up" a collective
 // decision, so that no thread is left alone at a later pg_sync().
 __device__ __forceinline__ bool pg_any(bool flag)
@@ -146,7 +136,7 @@ __device__ __forceinline__ bool pg_any(bool flag)
     uint32_t r;
     asm volatile(
         "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 p, %1, 0;\n\t"
-        "bar.red.or.pred q, 3, 256, p;\n\tselp.u32 %0, 1, 0, q;\n\t}"
+        "bar.red.or.pred q, 2, 256, p;\n\tselp.u32 %0, 1, 0, q;\n\t}"
         : "=r"(r)
         : "r"((uint32_t)flag)
         : "memory");
@@ -157,12 +147,66 @@ __device__ __forceinline__ bool pg_any(bool flag)
 // role r (0 control, 1 pre, 2 chain), chunk c, event e -> trace[(r * 64 + c) * 16 + e]
 #define KLA_TR(r, c, e)                                                                        \
     do {                                                                                       \
-        if (p.trace && blockIdx.x == 0 && (c) < 64 && (((r) == 0) || ((r) == 1 && tid == 0) || ((r) == 2 && tid == PG_T))) \
+        if (p.trace && blockIdx.x == 0 && (c) < 64 && (((r) == 0 && lane == 0) || ((r) == 1 && tid == 0) || ((r) == 2 && tid == PG_T))) \
             p.trace[((r) * 64 + (c)) * 16 + (e)] = clock64();                                  \
     } while (0)
 #else
 #define KLA_TR(r, c, e) do { } while (0)
 #endif
+
+// One level of the blocked inverse of I + B X (X strictly lower triangular, 64 x 64, in `tl`): for every pair
+// of adjacent BS x BS diagonal blocks (T_00, T_11 already inverted) the block below the diagonal becomes
+//   T_10 = -T_11 (B_1 X_10 T_00).
+// All pairs of the level are done at once by the 256 threads of the pre group: 32 result rows x BS columns,
+// one 1 x 4 tile per thread; `mm` holds the intermediate product.  Trip counts are warp-uniform.
+template <int BS>
+__device__ __forceinline__ void merge_level(float *tl, float *mm, const float *bet, int pt)
+{
+    constexpr int QPR = BS / 4;                 // column quads per row
+    constexpr int RMASK = 128 / BS - 1;         // a warp covers 128 / BS consecutive rows
+    const bool act = pt < 8 * BS;
+    const int R = pt / QPR, c4 = (pt % QPR) * 4;
+    const int pr = R / BS, r = R % BS;          // pair, row inside the block
+    const int rb = (2 * pr + 1) * BS, cb = 2 * pr * BS;
+    if (act) {
+        // M = B_1 X_10 T_00
+        const float *Ap = tl + (rb + r) * LDT + cb;
+        const float *Bp = tl + cb * LDT + cb + c4;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 2
+        for (int k = 0; k < BS; k += 4) {
+            const float4 a = *reinterpret_cast<const float4 *>(Ap + k);
+            const float av[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const float4 b = *reinterpret_cast<const float4 *>(Bp + (k + u) * LDT);
+                acc.x += av[u] * b.x; acc.y += av[u] * b.y; acc.z += av[u] * b.z; acc.w += av[u] * b.w;
+            }
+        }
+        const float s = bet[rb + r];
+        *reinterpret_cast<float4 *>(&mm[R * LDM + c4]) = make_float4(s * acc.x, s * acc.y, s * acc.z, s * acc.w);
+    }
+    pg_sync();
+    if (act) {
+        // T_10 = -T_11 M; T_11 is lower triangular: columns k > r of its row r are zero
+        const float *Ap = tl + (rb + r) * LDT + rb;
+        const float *Bp = mm + (pr * BS) * LDM + c4;
+        const int kend = min(BS, (r | RMASK) + 1);
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 2
+        for (int k = 0; k < kend; k += 4) {
+            const float4 a = *reinterpret_cast<const float4 *>(Ap + k);
+            const float av[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const float4 b = *reinterpret_cast<const float4 *>(Bp + (k + u) * LDM);
+                acc.x += av[u] * b.x; acc.y += av[u] * b.y; acc.z += av[u] * b.z; acc.w += av[u] * b.w;
+            }
+        }
+        *reinterpret_cast<float4 *>(&tl[(rb + r) * LDT + cb + c4]) = make_float4(-acc.x, -acc.y, -acc.z, -acc.w);
+    }
+    pg_sync();
+}
 
 template <int D, typename OUT>
 __global__ void __launch_bounds__(NT, 1)
@@ -171,7 +215,6 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     using Smem = TcSmem<D>;
     constexpr int KB = Smem::KB;
     constexpr int SLICES = D / NS;
-    constexpr int KSTEPS = D / 16;
     constexpr uint32_t STAGE_BYTES = Smem::KQ_BYTES;
     constexpr uint32_t ID_G = idesc_bf16(128, 64, 0, 0);    // [K;Q] K^T : A K-major, B K-major
     constexpr uint32_t ID_S = idesc_bf16(64, NS, 0, 1);     // K S / Q S / T rhs / P U : M=64, B MN-major
@@ -212,9 +255,12 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     // ---- set-up ------------------------------------------------------------------------------------------
     if (tid == 0) {
         for (int s = 0; s < NSTAGE; ++s) mbar_init(&sm.bar[B_FULL0 + s], 1);
-        mbar_init(&sm.bar[B_D1_DONE], 1);
-        mbar_init(&sm.bar[B_D1_FREE], PG_T / 32);
-        mbar_init(&sm.bar[B_TP_READY], PG_T / 32);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&sm.bar[B_D1_DONE0 + b], 1);
+            mbar_init(&sm.bar[B_D1_FREE0 + b], PG_T / 32);
+        }
+        mbar_init(&sm.bar[B_T_READY], PG_T / 32);
+        mbar_init(&sm.bar[B_P_READY], PG_T / 64);
         mbar_init(&sm.bar[B_S_READY], CG_T / 32);
         mbar_init(&sm.bar[B_D2_DONE], 1);
         mbar_init(&sm.bar[B_RHS_READY], CG_T / 32);
@@ -226,6 +272,8 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         sm.abort_flag = 0;
         mbar_fence_init();
     }
+    // the block of the solve matrix above the diagonal blocks is never written again
+    for (int i = tid; i < 64 * LDT; i += NT) sm.tl[i] = 0.f;
     if (warp == 0) tmem_alloc(&sm.tmem_base, TM_COLS);
     tc_fence_before();
     __syncthreads();
@@ -233,22 +281,7 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     const uint32_t tmem = sm.tmem_base;
     const uint32_t tm_lane = tmem + ((uint32_t)((warp & 3) * 32) << 16);  // this warp's 32 TMEM lanes
 
-    // Bounded wait that also leaves when another role has aborted.
-    auto wait = [&](int b, uint32_t parity) -> bool {
-        uint64_t *bar = &sm.bar[b];
-        if (mbar_try_wait(bar, parity)) return true;
-        const long long t0 = clock64();
-        while (true) {
-#pragma unroll 1
-            for (int i = 0; i < 32; ++i)
-                if (mbar_try_wait(bar, parity)) return true;
-            if (sm.abort_flag) return false;
-            if (clock64() - t0 > WAIT_LIMIT) {
-                sm.abort_flag = 1;
-                return false;
-            }
-        }
-    };
+    auto wait = [&](int b, uint32_t parity) -> bool { return bar_wait(&sm.bar[b], parity, &sm.abort_flag); };
     // one arrival per warp, after the warp's shared-memory writes are visible to the async proxy
     auto warp_arrive = [&](int b) {
         __syncwarp();
@@ -257,10 +290,14 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 
     if (warp == NT / 32 - 1) {
         // =============================== control warp =====================================================
+        // The whole warp runs this role in lock step: waits are taken by every lane, TMA loads are issued
+        // by lane 0 and tensor-core instructions by the lane that elect.sync picks.
         if (lane == 0) {
             tma_prefetch_desc(&tm_q);
             tma_prefetch_desc(&tm_k);
-            auto issue_tma = [&](int c) {
+        }
+        auto issue_tma = [&](int c) {
+            if (lane == 0) {
                 const int st = c % NSTAGE;
                 mbar_expect_tx(&sm.bar[B_FULL0 + st], STAGE_BYTES);
                 const int row = tok0 + c * C;
@@ -269,117 +306,115 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     tma_load_2d(sm.kq[st] + kb * 16384, &tm_k, h * D + kb * 64, row, &sm.bar[B_FULL0 + st]);
                     tma_load_2d(sm.kq[st] + kb * 16384 + 8192, &tm_q, h * D + kb * 64, row, &sm.bar[B_FULL0 + st]);
                 }
-            };
-            // Descriptors: everything except the 14-bit start-address field is fixed, so a K-step is an add.
-            const uint64_t d_kq0 = smem_desc_sw128(smem_u32(sm.kq[0]), 16, 1024);             // K-major views of a stage
-            const uint64_t d_kt0 = smem_desc_sw128(smem_u32(sm.kq[0]), KB * 8192, 1024);      // K^T (MN-major) view
-            const uint64_t d_sh = smem_desc_sw128(smem_u32(sm.s_hi), 16, 1024), d_sl = smem_desc_sw128(smem_u32(sm.s_lo), 16, 1024);
-            const uint64_t d_th = smem_desc_sw128(smem_u32(sm.t_hi), 16, 1024), d_tl = smem_desc_sw128(smem_u32(sm.t_lo), 16, 1024);
-            const uint64_t d_ph = smem_desc_sw128(smem_u32(sm.p_hi), 16, 1024), d_pl = smem_desc_sw128(smem_u32(sm.p_lo), 16, 1024);
-            const uint64_t d_rh = smem_desc_sw128(smem_u32(sm.ru_hi), 16, 1024), d_rl = smem_desc_sw128(smem_u32(sm.ru_lo), 16, 1024);
-            const uint64_t d_dh = smem_desc_sw128(smem_u32(sm.du_hi), 16, 1024), d_dl = smem_desc_sw128(smem_u32(sm.du_lo), 16, 1024);
-            constexpr uint64_t STAGE_STEP = (uint64_t)(Smem::KQ_BYTES >> 4);
-            auto kstep = [](int s) -> uint64_t { return (uint64_t)(((s / 4) * 16384 + (s % 4) * 32) >> 4); };
-
-            auto mma1 = [&](int c) {  // [K;Q] K^T -> D1
-                const uint64_t a0 = d_kq0 + (uint64_t)(c % NSTAGE) * STAGE_STEP;
-#pragma unroll
-                for (int s = 0; s < KSTEPS; ++s) mma_bf16_ss(tmem + TM_D1, a0 + kstep(s), a0 + kstep(s), ID_G, s > 0);
-                mma_commit(&sm.bar[B_D1_DONE]);
-            };
-            bool ok = true;
-            for (int c = 0; c < NSTAGE && c < nchunks; ++c) issue_tma(c);
-            // MMA-1(0)
-            ok = wait(B_FULL0, 0);
-            if (ok && nchunks == 1 && last_rows < C) ok = wait(B_TAIL_READY, 0);
-            if (ok) {
-                tc_fence_after();
-                mma1(0);
             }
-            for (int c = 0; ok && c < nchunks; ++c) {
-                const uint32_t ph = (uint32_t)(c & 1);
-                const uint64_t k0 = d_kq0 + (uint64_t)(c % NSTAGE) * STAGE_STEP;
-                const uint64_t kt0 = d_kt0 + (uint64_t)(c % NSTAGE) * STAGE_STEP;
-                // MMA-1(c+1): as early as its inputs and the D1 buffer allow
-                if (c + 1 < nchunks) {
-                    if (!(ok = wait(B_FULL0 + (c + 1) % NSTAGE, (uint32_t)(((c + 1) / NSTAGE) & 1)))) break;
-                    if (c + 2 == nchunks && last_rows < C)
-                        if (!(ok = wait(B_TAIL_READY, 0))) break;
-                    if (!(ok = wait(B_D1_FREE, ph))) break;
-                    tc_fence_after();
-                    mma1(c + 1);
-                }
-                KLA_TR(0, c, 0);
-                // MMA-2(c): K S_0 -> TM_KS (on the chain), then Q S_0 -> TM_QS[c&1] (needed only for the outputs)
-                if (!(ok = wait(B_S_READY, ph))) break;
-                KLA_TR(0, c, 1);
+            __syncwarp();
+        };
+        auto wwait = [&](int b, uint32_t parity) -> bool { return __all_sync(0xffffffffu, wait(b, parity)); };
+        // four MMAs (K = 64): operand descriptors advance by astep / bstep (16-byte units) per K-step
+        auto seq = [&](uint32_t d, uint64_t a, uint64_t astep, uint64_t b, uint64_t bstep, uint32_t idesc, uint32_t acc) {
+#pragma unroll
+            for (int s = 0; s < 4; ++s) mma_bf16_ss(d, a + s * astep, b + s * bstep, idesc, s > 0 ? 1u : acc);
+        };
+        // Descriptors: everything except the 14-bit start-address field is fixed, so a K-step is an add.
+        const uint64_t d_kq0 = smem_desc_sw128(smem_u32(sm.kq[0]), 16, 1024);             // K-major views of a stage
+        const uint64_t d_kt0 = smem_desc_sw128(smem_u32(sm.kq[0]), KB * 8192, 1024);      // K^T (MN-major) view
+        const uint64_t d_sh = smem_desc_sw128(smem_u32(sm.s_hi), 16, 1024), d_sl = smem_desc_sw128(smem_u32(sm.s_lo), 16, 1024);
+        const uint64_t d_th = smem_desc_sw128(smem_u32(sm.t_hi), 16, 1024), d_tl = smem_desc_sw128(smem_u32(sm.t_lo), 16, 1024);
+        const uint64_t d_ph = smem_desc_sw128(smem_u32(sm.p_hi), 16, 1024), d_pl = smem_desc_sw128(smem_u32(sm.p_lo), 16, 1024);
+        const uint64_t d_rh = smem_desc_sw128(smem_u32(sm.ru_hi), 16, 1024), d_rl = smem_desc_sw128(smem_u32(sm.ru_lo), 16, 1024);
+        const uint64_t d_dh = smem_desc_sw128(smem_u32(sm.du_hi), 16, 1024), d_dl = smem_desc_sw128(smem_u32(sm.du_lo), 16, 1024);
+        constexpr uint64_t STAGE_STEP = (uint64_t)(Smem::KQ_BYTES >> 4);
+
+        auto mma1 = [&](int c) {  // [K;Q] K^T -> D1 buffer c & 1
+            const uint64_t a0 = d_kq0 + (uint64_t)(c % NSTAGE) * STAGE_STEP;
+#pragma unroll 1
+            for (int kb = 0; kb < KB; ++kb) seq(tmem + TM_D1 + (uint32_t)(c & 1) * 64, a0 + kb * 1024, 2, a0 + kb * 1024, 2, ID_G, kb > 0);
+            mma_commit(&sm.bar[B_D1_DONE0 + (c & 1)]);
+        };
+        // [K or Q](c) S_0 -> d; qoff = 512 selects the Q tile of a block
+        auto mma_xs = [&](uint32_t d, uint64_t k0, uint64_t qoff) {
+#pragma unroll 1
+            for (int kb = 0; kb < KB; ++kb) seq(d, k0 + qoff + kb * 1024, 2, d_sh + kb * 512, 128, ID_S, kb > 0);
+#pragma unroll 1
+            for (int kb = 0; kb < KB; ++kb) seq(d, k0 + qoff + kb * 1024, 2, d_sl + kb * 512, 128, ID_S, 1);
+        };
+        // three-term product (a_hi + a_lo)(b_hi + b_lo) ~ a_hi b_hi + a_hi b_lo + a_lo b_hi, K = 64
+        auto mma_3 = [&](uint32_t d, uint64_t ah, uint64_t al, uint64_t bh, uint64_t bl) {
+            seq(d, ah, 2, bh, 128, ID_S, 0);
+            seq(d, ah, 2, bl, 128, ID_S, 1);
+            seq(d, al, 2, bh, 128, ID_S, 1);
+        };
+        bool ok = true;
+        for (int c = 0; c < NSTAGE && c < nchunks; ++c) issue_tma(c);
+        // MMA-1(0)
+        ok = wwait(B_FULL0, 0);
+        if (ok && nchunks == 1 && last_rows < C) ok = wwait(B_TAIL_READY, 0);
+        if (ok) {
+            tc_fence_after();
+            mma1(0);
+        }
+        for (int c = 0; ok && c < nchunks; ++c) {
+            const uint32_t ph = (uint32_t)(c & 1);
+            const uint64_t k0 = d_kq0 + (uint64_t)(c % NSTAGE) * STAGE_STEP;
+            const uint64_t kt0 = d_kt0 + (uint64_t)(c % NSTAGE) * STAGE_STEP;
+            // MMA-1(c+1): as early as its inputs and its D1 buffer allow
+            if (c + 1 < nchunks) {
+                if (!(ok = wwait(B_FULL0 + (c + 1) % NSTAGE, (uint32_t)(((c + 1) / NSTAGE) & 1)))) break;
+                if (c + 2 == nchunks && last_rows < C)
+                    if (!(ok = wwait(B_TAIL_READY, 0))) break;
+                if (c >= 1)   // the buffer was last used by chunk c - 1: its ((c - 1) / 2)-th use
+                    if (!(ok = wwait(B_D1_FREE0 + ((c + 1) & 1), (uint32_t)(((c - 1) >> 1) & 1)))) break;
                 tc_fence_after();
-                {
-#pragma unroll
-                    for (int s = 0; s < KSTEPS; ++s) mma_bf16_ss(tmem + TM_KS, k0 + kstep(s), d_sh + (uint64_t)(s * 128), ID_S, s > 0);
-#pragma unroll
-                    for (int s = 0; s < KSTEPS; ++s) mma_bf16_ss(tmem + TM_KS, k0 + kstep(s), d_sl + (uint64_t)(s * 128), ID_S, 1);
-                    mma_commit(&sm.bar[B_D2_DONE]);
-                    const uint32_t tq = tmem + ((c & 1) ? TM_QS1 : TM_QS0);
-#pragma unroll
-                    for (int s = 0; s < KSTEPS; ++s) mma_bf16_ss(tq, k0 + 512 + kstep(s), d_sh + (uint64_t)(s * 128), ID_S, s > 0);
-#pragma unroll
-                    for (int s = 0; s < KSTEPS; ++s) mma_bf16_ss(tq, k0 + 512 + kstep(s), d_sl + (uint64_t)(s * 128), ID_S, 1);
-                }
-                KLA_TR(0, c, 2);
-                // MMA-3(c): U = T rhs
-                if (!(ok = wait(B_TP_READY, ph))) break;
-                KLA_TR(0, c, 3);
-                if (!(ok = wait(B_RHS_READY, ph))) break;
-                KLA_TR(0, c, 4);
-                tc_fence_after();
-                {
-#pragma unroll
-                    for (int s = 0; s < 4; ++s) mma_bf16_ss(tmem + TM_U, d_th + (uint64_t)(s * 2), d_rh + (uint64_t)(s * 128), ID_S, s > 0);
-#pragma unroll
-                    for (int s = 0; s < 4; ++s) mma_bf16_ss(tmem + TM_U, d_th + (uint64_t)(s * 2), d_rl + (uint64_t)(s * 128), ID_S, 1);
-#pragma unroll
-                    for (int s = 0; s < 4; ++s) mma_bf16_ss(tmem + TM_U, d_tl + (uint64_t)(s * 2), d_rh + (uint64_t)(s * 128), ID_S, 1);
-                    mma_commit(&sm.bar[B_D3_DONE]);
-                }
-                KLA_TR(0, c, 5);
-                // MMA-5(c): K^T (D U)   then   MMA-4(c): P U
-                if (!(ok = wait(B_U_READY, ph))) break;
-                KLA_TR(0, c, 6);
-                tc_fence_after();
-                {
-                    // A = K^T: M = d_k (64-wide blocks KB*8192 bytes apart; for d_k = 64 the second block
-                    // is the Q tile, whose rows land in TMEM lanes 64..127 and are ignored), K = tokens
-#pragma unroll
-                    for (int s = 0; s < 4; ++s) mma_bf16_ss(tmem + TM_DS, kt0 + (uint64_t)(s * 128), d_dh + (uint64_t)(s * 128), ID_DS, s > 0);
-#pragma unroll
-                    for (int s = 0; s < 4; ++s) mma_bf16_ss(tmem + TM_DS, kt0 + (uint64_t)(s * 128), d_dl + (uint64_t)(s * 128), ID_DS, 1);
-                    mma_commit(&sm.bar[B_D5_DONE]);
-#pragma unroll
-                    for (int s = 0; s < 4; ++s) mma_bf16_ss(tmem + TM_PU, d_ph + (uint64_t)(s * 2), d_rh + (uint64_t)(s * 128), ID_S, s > 0);
-#pragma unroll
-                    for (int s = 0; s < 4; ++s) mma_bf16_ss(tmem + TM_PU, d_ph + (uint64_t)(s * 2), d_rl + (uint64_t)(s * 128), ID_S, 1);
-#pragma unroll
-                    for (int s = 0; s < 4; ++s) mma_bf16_ss(tmem + TM_PU, d_pl + (uint64_t)(s * 2), d_rh + (uint64_t)(s * 128), ID_S, 1);
-                    mma_commit(&sm.bar[B_D4_DONE]);
-                }
-                KLA_TR(0, c, 7);
-                // the K/Q stage of chunk c is free once MMA-5(c) has read it
-                if (c + NSTAGE < nchunks) {
-                    if (!(ok = wait(B_D5_DONE, ph))) break;
-                    issue_tma(c + NSTAGE);
-                }
+                mma1(c + 1);
+            }
+            KLA_TR(0, c, 0);
+            // MMA-2(c): K S_0 -> TM_KS (on the chain), then Q S_0 -> TM_QS[c&1] (needed only for the outputs)
+            if (!(ok = wwait(B_S_READY, ph))) break;
+            KLA_TR(0, c, 1);
+            tc_fence_after();
+            mma_xs(tmem + TM_KS, k0, 0);
+            mma_commit(&sm.bar[B_D2_DONE]);
+            mma_xs(tmem + ((c & 1) ? TM_QS1 : TM_QS0), k0, 512);
+            KLA_TR(0, c, 2);
+            // MMA-3(c): U = T rhs
+            if (!(ok = wwait(B_T_READY, ph))) break;
+            KLA_TR(0, c, 3);
+            if (!(ok = wwait(B_RHS_READY, ph))) break;
+            KLA_TR(0, c, 4);
+            tc_fence_after();
+            mma_3(tmem + TM_U, d_th, d_tl, d_rh, d_rl);
+            mma_commit(&sm.bar[B_D3_DONE]);
+            KLA_TR(0, c, 5);
+            // MMA-5(c): K^T (D U)   then   MMA-4(c): P U
+            if (!(ok = wwait(B_U_READY, ph))) break;
+            KLA_TR(0, c, 6);
+            tc_fence_after();
+            // A = K^T: M = d_k (64-wide blocks KB*8192 bytes apart; for d_k = 64 the second block
+            // is the Q tile, whose rows land in TMEM lanes 64..127 and are ignored), K = tokens
+            seq(tmem + TM_DS, kt0, 128, d_dh, 128, ID_DS, 0);
+            seq(tmem + TM_DS, kt0, 128, d_dl, 128, ID_DS, 1);
+            mma_commit(&sm.bar[B_D5_DONE]);
+            if (!(ok = wwait(B_P_READY, ph))) break;
+            tc_fence_after();
+            mma_3(tmem + TM_PU, d_ph, d_pl, d_rh, d_rl);
+            mma_commit(&sm.bar[B_D4_DONE]);
+            KLA_TR(0, c, 7);
+            // the K/Q stage of chunk c is free once MMA-5(c) has read it
+            if (c + NSTAGE < nchunks) {
+                if (!(ok = wwait(B_D5_DONE, ph))) break;
+                issue_tma(c + NSTAGE);
             }
         }
     } else if (warp < PG_T / 32) {
         // =============================== pre group ==========================================================
+        // Warps 0, 1, 4, 5 hold rows of K K^T (TMEM lanes 0..63), warps 2, 3, 6, 7 rows of Q K^T (lanes 64..127).
+        // Iteration c: the first set forms X(c) while the second forms P(c-1); then all eight warps invert.
         const int pt = tid;                       // 0..255
         const int q = warp & 3, chh = warp >> 2;  // TMEM lane quadrant, column half of D1
-        const int lrow = q * 32 + lane;           // D1 row held by this thread: G row (< 64) or Q K^T row
-        const bool is_g = lrow < 64;
-        const int i = lrow & 63;
-        const int nrow = pt >> 2, npart = pt & 3; // norm work: 4 threads per token
-        const bool scan_warp = warp == PG_T / 32 - 1;
+        const bool is_g = q < 2;
+        const int i = (q & 1) * 32 + lane;        // row of K K^T or of Q K^T held by this thread
+        const bool live = chh <= (q & 1);         // otherwise all 32 columns are above the diagonal
+        const bool scan_warp = warp == 4;         // K K^T rows 0..31 x columns 32..63: no X work
         float la_next0 = 0.f, la_next1 = 0.f, eta_next = 0.f;
         auto fetch_gates = [&](int c) {
             if (scan_warp) {
@@ -387,166 +422,165 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 la_next0 = (t < len) ? p.log_alpha[(size_t)(tok0 + t) * p.H + h] : 0.f;
                 la_next1 = (t + 1 < len) ? p.log_alpha[(size_t)(tok0 + t + 1) * p.H + h] : 0.f;
             }
-            if (npart == 0) {
-                const int t = c * C + nrow;
+            if (is_g && chh == q) {   // the thread whose 32 columns contain the diagonal element of its row
+                const int t = c * C + i;
                 eta_next = (t < len) ? p.eta[(size_t)(tok0 + t) * p.H + h] : 0.f;
             }
         };
+        // P(c) = A o Q K^T as bf16 hi/lo operand tiles (rows of Q K^T: warps 2, 3, 6, 7 only)
+        auto form_p = [&](int c) -> bool {
+            // D1(c) complete; the P tiles are free once MMA-4(c-1) has read them
+            bool okp = wait(B_D1_DONE0 + (c & 1), (uint32_t)((c >> 1) & 1));
+            if (okp && c > 0) okp = wait(B_D4_DONE, (uint32_t)((c - 1) & 1));
+            if (!okp) return false;
+            tc_fence_after();
+            const int sc = c % NSTAGE;
+            const float gi2 = sm.g2[sc][i];
+            const uint32_t tbase = tm_lane + TM_D1 + (uint32_t)(c & 1) * 64 + chh * 32;
+#pragma unroll 1
+            for (int grp = 0; grp < 4; ++grp) {
+                uint4 hi = make_uint4(0, 0, 0, 0), lo = hi;
+                if (live) {
+                    float a[8];
+                    tmem_ld8(tbase + grp * 8, a);
+                    const int j0 = chh * 32 + grp * 8;
+                    const float4 ga = *reinterpret_cast<const float4 *>(&sm.g2[sc][j0]);
+                    const float4 gb = *reinterpret_cast<const float4 *>(&sm.g2[sc][j0 + 4]);
+                    const float gj[8] = {ga.x, ga.y, ga.z, ga.w, gb.x, gb.y, gb.z, gb.w};
+                    float x[8];
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) x[e] = (j0 + e <= i) ? ex2_approx(gi2 - gj[e]) * a[e] : 0.f;
+                    split2(x[0], x[1], hi.x, lo.x);
+                    split2(x[2], x[3], hi.y, lo.y);
+                    split2(x[4], x[5], hi.z, lo.z);
+                    split2(x[6], x[7], hi.w, lo.w);
+                }
+                *reinterpret_cast<uint4 *>(sm.p_hi + sw128(i, chh * 4 + grp)) = hi;
+                *reinterpret_cast<uint4 *>(sm.p_lo + sw128(i, chh * 4 + grp)) = lo;
+            }
+            tc_fence_before();
+            fence_async_smem();
+            warp_arrive(B_D1_FREE0 + (c & 1));
+            warp_arrive(B_P_READY);
+            return true;
+        };
         fetch_gates(0);
-        for (int c = 0; c < nchunks; ++c) {
+        int c = 0;
+        for (; c < nchunks; ++c) {
             const uint32_t ph = (uint32_t)(c & 1);
             const int rows = (c == nchunks - 1) ? last_rows : C;
             const int sc = c % NSTAGE;
             const float la0 = la_next0, la1 = la_next1, eta_cur = eta_next;
             if (c + 1 < nchunks) fetch_gates(c + 1);
-            // ---- g_i, gamma_i, exp(g_C - g_i): fp64 scan by one warp (needs no tile) -----------------------------
+            // ---- g_i (chunk-local running sum of log alpha), gamma_i, exp(g_C - g_i) -----------------------------
             if (scan_warp) {
-                const double v0 = (double)la0, v1 = (double)la1;
-                const double run = v0 + v1;
-                double incl = run;
+                float incl = la0 + la1;
 #pragma unroll
                 for (int o = 1; o < 32; o <<= 1) {
-                    const double t = __shfl_up_sync(0xffffffffu, incl, o);
+                    const float t = __shfl_up_sync(0xffffffffu, incl, o);
                     if (lane >= o) incl += t;
                 }
-                const double gC = __shfl_sync(0xffffffffu, incl, 31);
-                const double ga = incl - v1, gb = incl;
-                const float a2 = (float)(ga * (double)LOG2E), b2 = (float)(gb * (double)LOG2E);
-                *reinterpret_cast<float2 *>(&sm.g2[2 * lane]) = make_float2(a2, b2);
+                const float gC = __shfl_sync(0xffffffffu, incl, 31);
+                const float a2 = (incl - la1) * LOG2E, b2 = incl * LOG2E, c2 = gC * LOG2E;
+                *reinterpret_cast<float2 *>(&sm.g2[sc][2 * lane]) = make_float2(a2, b2);
                 *reinterpret_cast<float2 *>(&sm.gam[sc][2 * lane]) = make_float2(ex2_approx(a2), ex2_approx(b2));
-                *reinterpret_cast<float2 *>(&sm.dec[sc][2 * lane]) =
-                    make_float2(ex2_approx((float)((gC - ga) * (double)LOG2E)), ex2_approx((float)((gC - gb) * (double)LOG2E)));
+                *reinterpret_cast<float2 *>(&sm.dec[sc][2 * lane]) = make_float2(ex2_approx(c2 - a2), ex2_approx(c2 - b2));
             }
             KLA_TR(1, c, 0);
-            if (pg_any(!wait(B_FULL0 + sc, (uint32_t)((c / NSTAGE) & 1)))) break;
-            KLA_TR(1, c, 1);
-            unsigned char *kq = sm.kq[sc];
+            bool okc = true;
             if (rows < C) {
                 // last chunk: rows past the end of the sequence hold a neighbour's tokens (or TMA zero
                 // fill); zero them so that they are inert in every product
-                for (int e = pt; e < (C - rows) * 8; e += PG_T) {
-                    const int r = rows + e / 8, ch = e % 8;
-                    const uint4 z = make_uint4(0, 0, 0, 0);
+                okc = wait(B_FULL0 + sc, (uint32_t)((c / NSTAGE) & 1));
+                if (okc) {
+                    unsigned char *kq = sm.kq[sc];
+                    for (int e = pt; e < (C - rows) * 8; e += PG_T) {
+                        const int r = rows + e / 8, ch = e % 8;
+                        const uint4 z = make_uint4(0, 0, 0, 0);
 #pragma unroll
-                    for (int kb = 0; kb < KB; ++kb) {
-                        *reinterpret_cast<uint4 *>(kq + kb * 16384 + sw128(r, ch)) = z;
-                        *reinterpret_cast<uint4 *>(kq + kb * 16384 + 8192 + sw128(r, ch)) = z;
-                    }
-                }
-                fence_async_smem();
-                warp_arrive(B_TAIL_READY);
-            }
-            // ---- beta_i = eta_i / (||k_i||^2 + eps): 4 threads per token ------------------------------------------
-            {
-                float n0 = 0.f, n1 = 0.f;
-                if (nrow < rows) {
-#pragma unroll
-                    for (int kb = 0; kb < KB; ++kb)
-#pragma unroll
-                        for (int cc = 0; cc < 2; ++cc) {
-                            const uint4 raw = *reinterpret_cast<const uint4 *>(kq + kb * 16384 + sw128(nrow, npart * 2 + cc));
-                            const __nv_bfloat162 *h2 = reinterpret_cast<const __nv_bfloat162 *>(&raw);
-                            const float2 f0 = __bfloat1622float2(h2[0]), f1 = __bfloat1622float2(h2[1]);
-                            const float2 f2 = __bfloat1622float2(h2[2]), f3 = __bfloat1622float2(h2[3]);
-                            n0 += f0.x * f0.x + f0.y * f0.y + f2.x * f2.x + f2.y * f2.y;
-                            n1 += f1.x * f1.x + f1.y * f1.y + f3.x * f3.x + f3.y * f3.y;
+                        for (int kb = 0; kb < KB; ++kb) {
+                            *reinterpret_cast<uint4 *>(kq + kb * 16384 + sw128(r, ch)) = z;
+                            *reinterpret_cast<uint4 *>(kq + kb * 16384 + 8192 + sw128(r, ch)) = z;
                         }
+                    }
+                    fence_async_smem();
+                    warp_arrive(B_TAIL_READY);
                 }
-                float nk = n0 + n1;
-                nk += __shfl_xor_sync(0xffffffffu, nk, 1);
-                nk += __shfl_xor_sync(0xffffffffu, nk, 2);
-                if (npart == 0) sm.beta[sc][nrow] = (nrow < rows) ? eta_cur / (nk + p.eps) : 0.f;
+            }
+            if (pg_any(!okc)) break;   // also publishes the decay sums to the whole group
+            if (is_g) {
+                // ---- X = A^- o K K^T from MMA-1 (this thread: row i, 32 columns) and beta_i ----------------------------
+                okc = wait(B_D1_DONE0 + (c & 1), (uint32_t)((c >> 1) & 1));
+                if (okc) {
+                    tc_fence_after();
+                    if (live) {
+                        const float gi2 = sm.g2[sc][i];
+                        float dg = 0.f;   // G_ii = ||k_i||^2
+                        const uint32_t tbase = tm_lane + TM_D1 + (uint32_t)(c & 1) * 64 + chh * 32;
+#pragma unroll 1
+                        for (int grp = 0; grp < 4; ++grp) {
+                            float a[8];
+                            tmem_ld8(tbase + grp * 8, a);
+                            const int j0 = chh * 32 + grp * 8;
+                            const float4 ga = *reinterpret_cast<const float4 *>(&sm.g2[sc][j0]);
+                            const float4 gb = *reinterpret_cast<const float4 *>(&sm.g2[sc][j0 + 4]);
+                            const float gj[8] = {ga.x, ga.y, ga.z, ga.w, gb.x, gb.y, gb.z, gb.w};
+                            float x[8];
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) {
+                                x[e] = (j0 + e < i) ? ex2_approx(gi2 - gj[e]) * a[e] : 0.f;
+                                dg = (j0 + e == i) ? a[e] : dg;
+                            }
+                            *reinterpret_cast<float4 *>(&sm.tl[i * LDT + j0]) = make_float4(x[0], x[1], x[2], x[3]);
+                            *reinterpret_cast<float4 *>(&sm.tl[i * LDT + j0 + 4]) = make_float4(x[4], x[5], x[6], x[7]);
+                        }
+                        // beta_i = eta_i / (||k_i||^2 + eps), Eq. 3; rows past the end of the sequence get 0
+                        if (chh == q) sm.beta[sc][i] = (i < rows) ? eta_cur / (dg + p.eps) : 0.f;
+                    }
+                    tc_fence_before();
+                    warp_arrive(B_D1_FREE0 + (c & 1));
+                }
+            } else if (c > 0) {
+                okc = form_p(c - 1);
+            }
+            if (pg_any(!okc)) break;
+            KLA_TR(1, c, 1);
+
+            // ---- T = (I + B X)^-1: 8x8 diagonal blocks by substitution, then the off-diagonal blocks
+            //      T_10 = -T_11 (B_1 X_10 T_00) at block sizes 8, 16, 32 -----------------------------------------------
+            const float *bet = sm.beta[sc];
+            if (pt < 64) {
+                const int blk = pt >> 3, j = pt & 7;
+                float *Lb = sm.tl + (blk * 8) * LDT + blk * 8;
+                float x[8];
+#pragma unroll
+                for (int r = 0; r < 8; ++r) {
+                    const float4 l0 = *reinterpret_cast<const float4 *>(Lb + r * LDT);
+                    const float4 l1 = *reinterpret_cast<const float4 *>(Lb + r * LDT + 4);
+                    const float l[8] = {l0.x, l0.y, l0.z, l0.w, l1.x, l1.y, l1.z, l1.w};
+                    float s = 0.f;
+#pragma unroll
+                    for (int m = 0; m < r; ++m) s += l[m] * x[m];
+                    x[r] = (r == j) ? 1.f : ((r > j) ? -bet[blk * 8 + r] * s : 0.f);
+                }
+                half_sync();  // every column of the block has read X_bb
+#pragma unroll
+                for (int r = 0; r < 8; ++r) Lb[r * LDT + j] = x[r];
             }
             pg_sync();
             KLA_TR(1, c, 2);
-            // ---- L (lanes 0..63) and P (lanes 64..127) from MMA-1; this thread: row i, 32 columns ---------------------
-            if (pg_any(!wait(B_D1_DONE, ph))) break;
-            KLA_TR(1, c, 3);
-            tc_fence_after();
-            uint32_t p_hi[16], p_lo[16];  // this thread's half P row, packed bf16 pairs (Q K^T rows only)
-            {
-                const float gi2 = sm.g2[i];
-                const float bi = sm.beta[sc][i];
-                float acc[32];
-                tmem_ld32(tm_lane + TM_D1 + chh * 32, acc);
-#pragma unroll
-                for (int j4 = 0; j4 < 8; ++j4) {
-                    const float4 gj = *reinterpret_cast<const float4 *>(&sm.g2[chh * 32 + 4 * j4]);
-                    const int j = chh * 32 + 4 * j4;
-                    const float e0 = ex2_approx(gi2 - gj.x), e1 = ex2_approx(gi2 - gj.y);
-                    const float e2 = ex2_approx(gi2 - gj.z), e3 = ex2_approx(gi2 - gj.w);
-                    if (is_g) {
-                        float4 o;
-                        o.x = (j + 0 < i) ? bi * e0 * acc[4 * j4 + 0] : 0.f;
-                        o.y = (j + 1 < i) ? bi * e1 * acc[4 * j4 + 1] : 0.f;
-                        o.z = (j + 2 < i) ? bi * e2 * acc[4 * j4 + 2] : 0.f;
-                        o.w = (j + 3 < i) ? bi * e3 * acc[4 * j4 + 3] : 0.f;
-                        *reinterpret_cast<float4 *>(&sm.tl[i * LDT + j]) = o;
-                    } else {
-                        const float a0 = (j + 0 <= i) ? e0 * acc[4 * j4 + 0] : 0.f;
-                        const float a1 = (j + 1 <= i) ? e1 * acc[4 * j4 + 1] : 0.f;
-                        const float a2 = (j + 2 <= i) ? e2 * acc[4 * j4 + 2] : 0.f;
-                        const float a3 = (j + 3 <= i) ? e3 * acc[4 * j4 + 3] : 0.f;
-                        split2(a0, a1, p_hi[2 * j4], p_lo[2 * j4]);
-                        split2(a2, a3, p_hi[2 * j4 + 1], p_lo[2 * j4 + 1]);
-                    }
-                }
-            }
-            tc_fence_before();
-            warp_arrive(B_D1_FREE);
-            pg_sync();
-            KLA_TR(1, c, 4);
-
-            // ---- T = (I + L)^-1, blocked: 16x16 diagonal blocks, then 16x16 and 32x32 off-diagonal blocks ------
-            if (pt < 64) {
-                const int blk = pt >> 4, j = pt & 15;
-                const float *Lb = sm.tl + (blk * 16) * LDT + blk * 16;
-                float x[16];
-#pragma unroll
-                for (int r = 0; r < 16; ++r) {
-                    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-#pragma unroll
-                    for (int m4 = 0; m4 < r; m4 += 4) {
-                        const float4 l4 = *reinterpret_cast<const float4 *>(Lb + r * LDT + m4);
-                        s0 += l4.x * x[m4];
-                        if (m4 + 1 < r) s1 += l4.y * x[m4 + 1];
-                        if (m4 + 2 < r) s2 += l4.z * x[m4 + 2];
-                        if (m4 + 3 < r) s3 += l4.w * x[m4 + 3];
-                    }
-                    x[r] = (r == j) ? 1.f : ((r > j) ? -((s0 + s1) + (s2 + s3)) : 0.f);
-                }
-                pg_half_sync();  // every column of the block has read L_bb
-                float *Tb = sm.tl + (blk * 16) * LDT + blk * 16;
-#pragma unroll
-                for (int r = 0; r < 16; ++r) Tb[r * LDT + j] = x[r];
-            }
-            pg_sync();
-            KLA_TR(1, c, 5);
-            {
-                // level 1: M = L10 T00 and L32 T22 (16x16 each); then T10 = -T11 M, T32 = -T33 M
-                const int prod = pt >> 7, r = (pt & 127) >> 3, c2 = (pt & 7) * 2;
-                const int rb = prod ? 48 : 16, cb = prod ? 32 : 0;
-                row_mm<16, 2>(sm.mm + prod * 16 * LDM, LDM, sm.tl + rb * LDT + cb, LDT, sm.tl + cb * LDT + cb, LDT, r, c2, true, false, 1.f);
-                pg_sync();
-                row_mm<16, 2>(sm.tl + rb * LDT + cb, LDT, sm.tl + rb * LDT + rb, LDT, sm.mm + prod * 16 * LDM, LDM, r, c2, false, true, -1.f);
-                pg_sync();
-            }
+            merge_level<8>(sm.tl, sm.mm, bet, pt);
             KLA_TR(1, c, 6);
-            {
-                // level 2: M = L[32..63][0..31] T[0..31][0..31]; T[32..63][0..31] = -T[32..63][32..63] M
-                const int r = pt >> 3, c4 = (pt & 7) * 4;
-                row_mm<32, 4>(sm.mm, LDM, sm.tl + 32 * LDT, LDT, sm.tl, LDT, r, c4, true, false, 1.f);
-                pg_sync();
-                row_mm<32, 4>(sm.tl + 32 * LDT, LDT, sm.tl + 32 * LDT + 32, LDT, sm.mm, LDM, r, c4, false, true, -1.f);
-                pg_sync();
-            }
-            // ---- write T (after MMA-3(c-1) has read the previous one) and P (after MMA-4(c-1)) ----------------------
+            merge_level<16>(sm.tl, sm.mm, bet, pt);
             KLA_TR(1, c, 7);
+            merge_level<32>(sm.tl, sm.mm, bet, pt);
+            // ---- write T as bf16 hi/lo operand tiles, after MMA-3(c-1) has read the previous ones ----------------------
+            KLA_TR(1, c, 3);
             if (c > 0 && pg_any(!wait(B_D3_DONE, ph ^ 1))) break;
-            KLA_TR(1, c, 8);
+            KLA_TR(1, c, 4);
             {
-                const int r = pt >> 2, qq = pt & 3;  // row, 16-column quarter
-#pragma unroll
+                const int r = pt & 63, qq = pt >> 6;  // row, 16-column quarter
+#pragma unroll 1
                 for (int ch = 0; ch < 2; ++ch) {
                     const float4 a = *reinterpret_cast<const float4 *>(&sm.tl[r * LDT + qq * 16 + ch * 8]);
                     const float4 b = *reinterpret_cast<const float4 *>(&sm.tl[r * LDT + qq * 16 + ch * 8 + 4]);
@@ -559,21 +593,13 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     *reinterpret_cast<uint4 *>(sm.t_lo + sw128(r, qq * 2 + ch)) = lo;
                 }
             }
-            KLA_TR(1, c, 9);
-            if (c > 0 && pg_any(!wait(B_D4_DONE, ph ^ 1))) break;
-            KLA_TR(1, c, 10);
-            if (!is_g) {
-#pragma unroll
-                for (int ch = 0; ch < 4; ++ch) {
-                    *reinterpret_cast<uint4 *>(sm.p_hi + sw128(i, chh * 4 + ch)) = make_uint4(p_hi[4 * ch], p_hi[4 * ch + 1], p_hi[4 * ch + 2], p_hi[4 * ch + 3]);
-                    *reinterpret_cast<uint4 *>(sm.p_lo + sw128(i, chh * 4 + ch)) = make_uint4(p_lo[4 * ch], p_lo[4 * ch + 1], p_lo[4 * ch + 2], p_lo[4 * ch + 3]);
-                }
-            }
             fence_async_smem();
-            pg_sync();  // the solve matrix and g2 are reused by the next chunk
-            warp_arrive(B_TP_READY);
-            KLA_TR(1, c, 11);
+            pg_sync();  // the solve matrix is reused by the next chunk
+            warp_arrive(B_T_READY);
+            KLA_TR(1, c, 5);
         }
+        // P of the last chunk
+        if (c == nchunks && !is_g) form_p(nchunks - 1);
     } else {
         // =============================== chain group ==========================================================
         const int ct = tid - PG_T;              // 0..255
@@ -640,7 +666,7 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             const int sc = c % NSTAGE;
             // ---- rhs = B (V - D_gamma K S_0) ------------------------------------------------------------------
             KLA_TR(2, c, 0);
-            if (!wait(B_TP_READY, ph)) break;   // scalars of chunk c
+            if (!wait(B_T_READY, ph)) break;   // scalars of chunk c
             KLA_TR(2, c, 1);
             const float b0 = sm.beta[sc][i0], b1 = sm.beta[sc][i1];
             const float g0 = sm.gam[sc][i0], g1 = sm.gam[sc][i1];
@@ -808,7 +834,8 @@ cudaError_t launch_t(const ChunkParams &p, cudaStream_t stream)
         pt.trace = tbuf;
         kern<<<grid, NT, smem, stream>>>(tq, tk, pt);
         cudaDeviceSynchronize();
-        FILE *f = fopen("gpurun_out/trace.txt", "w");
+        const char *tf = getenv("KLA_TRACE_FILE");
+        FILE *f = tf ? fopen(tf, "w") : nullptr;
         if (f) {
             for (int r = 0; r < 3; ++r)
                 for (int c = 0; c < 64; ++c) {

@@ -78,7 +78,8 @@ enum Bar {
     B_D5_DONE = 14,
     B_D4_DONE = 15,          // P U (and, earlier in the pipe, Q S_0) of chunk c complete
     B_TAIL_READY = 16,       // masked rows of the last chunk zeroed
-    B_COUNT = 17
+    B_V_FULL = 17,           // V slice of chunk c landed
+    B_COUNT = 18
 };
 
 template <int D>
@@ -97,6 +98,7 @@ struct TcSmem {
     alignas(1024) unsigned char ru_lo[8192];
     alignas(1024) unsigned char du_hi[8192];    // diag(exp(g_C - g_j)) U
     alignas(1024) unsigned char du_lo[8192];
+    alignas(1024) unsigned char vt[8192];       // V slice of one chunk: 64 tokens x 64 bf16, same layout as ru_*
     alignas(16) float tl[64 * LDT];             // X = A^- o K K^T, overwritten in place by T = (I + B X)^-1
     alignas(16) float mm[32 * LDM];             // scratch for the block products of the inverse
     alignas(16) float g2[NSTAGE][64];           // log2(e) * chunk-local running sum of log alpha
@@ -210,7 +212,8 @@ __device__ __forceinline__ void merge_level(float *tl, float *mm, const float *b
 
 template <int D, typename OUT>
 __global__ void __launch_bounds__(NT, 1)
-kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k, ChunkParams p)
+kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                    const __grid_constant__ CUtensorMap tm_v, ChunkParams p)
 {
     using Smem = TcSmem<D>;
     constexpr int KB = Smem::KB;
@@ -269,6 +272,7 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         mbar_init(&sm.bar[B_D5_DONE], 1);
         mbar_init(&sm.bar[B_D4_DONE], 1);
         mbar_init(&sm.bar[B_TAIL_READY], PG_T / 32);
+        mbar_init(&sm.bar[B_V_FULL], 1);
         sm.abort_flag = 0;
         mbar_fence_init();
     }
@@ -295,6 +299,7 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         if (lane == 0) {
             tma_prefetch_desc(&tm_q);
             tma_prefetch_desc(&tm_k);
+            tma_prefetch_desc(&tm_v);
         }
         auto issue_tma = [&](int c) {
             if (lane == 0) {
@@ -306,6 +311,16 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     tma_load_2d(sm.kq[st] + kb * 16384, &tm_k, h * D + kb * 64, row, &sm.bar[B_FULL0 + st]);
                     tma_load_2d(sm.kq[st] + kb * 16384 + 8192, &tm_q, h * D + kb * 64, row, &sm.bar[B_FULL0 + st]);
                 }
+            }
+            __syncwarp();
+        };
+        // V slice of chunk c: one 64 x 64 box; the single buffer is free once every chain warp has posted rhs(c-1).
+        // (Fetching V with plain loads into registers a chunk ahead stalled the chain warps for the full
+        // global-memory latency at their next barrier wait.)
+        auto issue_tma_v = [&](int c) {
+            if (lane == 0) {
+                mbar_expect_tx(&sm.bar[B_V_FULL], 8192);
+                tma_load_2d(sm.vt, &tm_v, h * D + sl * NS, tok0 + c * C, &sm.bar[B_V_FULL]);
             }
             __syncwarp();
         };
@@ -346,6 +361,7 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         };
         bool ok = true;
         for (int c = 0; c < NSTAGE && c < nchunks; ++c) issue_tma(c);
+        issue_tma_v(0);
         // MMA-1(0)
         ok = wwait(B_FULL0, 0);
         if (ok && nchunks == 1 && last_rows < C) ok = wwait(B_TAIL_READY, 0);
@@ -381,6 +397,7 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             KLA_TR(0, c, 3);
             if (!(ok = wwait(B_RHS_READY, ph))) break;
             KLA_TR(0, c, 4);
+            if (c + 1 < nchunks) issue_tma_v(c + 1);
             tc_fence_after();
             mma_3(tmem + TM_U, d_th, d_tl, d_rh, d_rl);
             mma_commit(&sm.bar[B_D3_DONE]);
@@ -639,25 +656,10 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             fence_async_smem();
             warp_arrive(B_S_READY);
         };
-        // byte offsets of this thread's bf16 pairs inside the 64-token x 64-column B-operand tiles
-        uint32_t off0[4], off1[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            off0[j] = sw128(i0, hf * 4 + j) + 4 * (lane & 3);
-            off1[j] = sw128(i1, hf * 4 + j) + 4 * (lane & 3);
-        }
-        const __nv_bfloat16 *vbase = reinterpret_cast<const __nv_bfloat16 *>(p.v) + (size_t)h * D + sl * NS + cp;
-        const size_t tokstride = (size_t)p.H * D;
-        uint32_t v0[4], v1[4];  // V[i0][cp + 8j .. +1], V[i1][...] as packed bf16 pairs
-        auto fetch_v = [&](int c) {
-            const int t0 = c * C + i0, t1 = c * C + i1;
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                v0[j] = (t0 < len) ? *reinterpret_cast<const uint32_t *>(vbase + (size_t)(tok0 + t0) * tokstride + 8 * j) : 0u;
-                v1[j] = (t1 < len) ? *reinterpret_cast<const uint32_t *>(vbase + (size_t)(tok0 + t1) * tokstride + 8 * j) : 0u;
-            }
-        };
-        fetch_v(0);
+        // byte offset of this thread's bf16 pair j (columns cp + 8j, cp + 8j + 1) of row i inside the
+        // 64-token x 64-column B-operand tiles
+        const uint32_t lo4 = 4 * (lane & 3);
+        auto off = [&](int i, int j) -> uint32_t { return sw128(i, hf * 4 + j) + lo4; };
         store_state_tiles();
 
         for (int c = 0; c < nchunks; ++c) {
@@ -672,54 +674,55 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             const float g0 = sm.gam[sc][i0], g1 = sm.gam[sc][i1];
             const float d0 = sm.dec[sc][i0], d1 = sm.dec[sc][i1];
             const float gC = sm.gam[sc][C - 1];
+            if (!wait(B_V_FULL, ph)) break;
             if (!wait(B_D2_DONE, ph)) break;
             KLA_TR(2, c, 2);
             tc_fence_after();
-            {
-                float acc[16];
-                tmem_ld16x256b_x4(tm16 + TM_KS, acc);
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const float2 fa = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&v0[j]));
-                    const float2 fb = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&v1[j]));
-                    uint32_t hi, lo;
-                    split2(b0 * (fa.x - g0 * acc[4 * j]), b0 * (fa.y - g0 * acc[4 * j + 1]), hi, lo);
-                    *reinterpret_cast<uint32_t *>(sm.ru_hi + off0[j]) = hi;
-                    *reinterpret_cast<uint32_t *>(sm.ru_lo + off0[j]) = lo;
-                    split2(b1 * (fb.x - g1 * acc[4 * j + 2]), b1 * (fb.y - g1 * acc[4 * j + 3]), hi, lo);
-                    *reinterpret_cast<uint32_t *>(sm.ru_hi + off1[j]) = hi;
-                    *reinterpret_cast<uint32_t *>(sm.ru_lo + off1[j]) = lo;
-                }
+#pragma unroll 1
+            for (int j = 0; j < 4; ++j) {
+                float acc[4];
+                tmem_ld16x256b_x1(tm16 + TM_KS + 8 * j, acc);
+                const uint32_t o0 = off(i0, j), o1 = off(i1, j);
+                // V[i0][cp + 8j .. +1], V[i1][...]; rows past the end of the sequence are another sequence's tokens
+                const uint32_t va = (i0 < rows) ? *reinterpret_cast<const uint32_t *>(sm.vt + o0) : 0u;
+                const uint32_t vb = (i1 < rows) ? *reinterpret_cast<const uint32_t *>(sm.vt + o1) : 0u;
+                const float2 fa = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&va));
+                const float2 fb = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&vb));
+                uint32_t hi, lo;
+                split2(b0 * (fa.x - g0 * acc[0]), b0 * (fa.y - g0 * acc[1]), hi, lo);
+                *reinterpret_cast<uint32_t *>(sm.ru_hi + o0) = hi;
+                *reinterpret_cast<uint32_t *>(sm.ru_lo + o0) = lo;
+                split2(b1 * (fb.x - g1 * acc[2]), b1 * (fb.y - g1 * acc[3]), hi, lo);
+                *reinterpret_cast<uint32_t *>(sm.ru_hi + o1) = hi;
+                *reinterpret_cast<uint32_t *>(sm.ru_lo + o1) = lo;
             }
             fence_async_smem();
             tc_fence_before();
             warp_arrive(B_RHS_READY);
             KLA_TR(2, c, 3);
-            if (c + 1 < nchunks) fetch_v(c + 1);
 
             // ---- U and D U as hi/lo operands -------------------------------------------------------------------
             if (!wait(B_D3_DONE, ph)) break;
             KLA_TR(2, c, 4);
             tc_fence_after();
-            {
-                float acc[16];
-                tmem_ld16x256b_x4(tm16 + TM_U, acc);
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    uint32_t hi, lo;
-                    split2(acc[4 * j], acc[4 * j + 1], hi, lo);
-                    *reinterpret_cast<uint32_t *>(sm.ru_hi + off0[j]) = hi;
-                    *reinterpret_cast<uint32_t *>(sm.ru_lo + off0[j]) = lo;
-                    split2(acc[4 * j + 2], acc[4 * j + 3], hi, lo);
-                    *reinterpret_cast<uint32_t *>(sm.ru_hi + off1[j]) = hi;
-                    *reinterpret_cast<uint32_t *>(sm.ru_lo + off1[j]) = lo;
-                    split2(d0 * acc[4 * j], d0 * acc[4 * j + 1], hi, lo);
-                    *reinterpret_cast<uint32_t *>(sm.du_hi + off0[j]) = hi;
-                    *reinterpret_cast<uint32_t *>(sm.du_lo + off0[j]) = lo;
-                    split2(d1 * acc[4 * j + 2], d1 * acc[4 * j + 3], hi, lo);
-                    *reinterpret_cast<uint32_t *>(sm.du_hi + off1[j]) = hi;
-                    *reinterpret_cast<uint32_t *>(sm.du_lo + off1[j]) = lo;
-                }
+#pragma unroll 1
+            for (int j = 0; j < 4; ++j) {
+                float acc[4];
+                tmem_ld16x256b_x1(tm16 + TM_U + 8 * j, acc);
+                const uint32_t o0 = off(i0, j), o1 = off(i1, j);
+                uint32_t hi, lo;
+                split2(acc[0], acc[1], hi, lo);
+                *reinterpret_cast<uint32_t *>(sm.ru_hi + o0) = hi;
+                *reinterpret_cast<uint32_t *>(sm.ru_lo + o0) = lo;
+                split2(acc[2], acc[3], hi, lo);
+                *reinterpret_cast<uint32_t *>(sm.ru_hi + o1) = hi;
+                *reinterpret_cast<uint32_t *>(sm.ru_lo + o1) = lo;
+                split2(d0 * acc[0], d0 * acc[1], hi, lo);
+                *reinterpret_cast<uint32_t *>(sm.du_hi + o0) = hi;
+                *reinterpret_cast<uint32_t *>(sm.du_lo + o0) = lo;
+                split2(d1 * acc[2], d1 * acc[3], hi, lo);
+                *reinterpret_cast<uint32_t *>(sm.du_hi + o1) = hi;
+                *reinterpret_cast<uint32_t *>(sm.du_lo + o1) = lo;
             }
             fence_async_smem();
             tc_fence_before();
@@ -747,15 +750,16 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             KLA_TR(2, c, 8);
             tc_fence_after();
             {
-                float acc[16], qs[16];
-                tmem_ld16x256b_x4(tm16 + TM_PU, acc);
-                tmem_ld16x256b_x4(tm16 + ((c & 1) ? TM_QS1 : TM_QS0), qs);
                 OUT *o0 = reinterpret_cast<OUT *>(p.out) + ((size_t)(tok0 + c * C + i0) * p.H + h) * D + sl * NS + cp;
                 OUT *o1 = reinterpret_cast<OUT *>(p.out) + ((size_t)(tok0 + c * C + i1) * p.H + h) * D + sl * NS + cp;
-#pragma unroll
+                const uint32_t tq = tm16 + ((c & 1) ? TM_QS1 : TM_QS0);
+#pragma unroll 1
                 for (int j = 0; j < 4; ++j) {
-                    if (i0 < rows) store2(o0 + 8 * j, g0 * qs[4 * j] + acc[4 * j], g0 * qs[4 * j + 1] + acc[4 * j + 1]);
-                    if (i1 < rows) store2(o1 + 8 * j, g1 * qs[4 * j + 2] + acc[4 * j + 2], g1 * qs[4 * j + 3] + acc[4 * j + 3]);
+                    float acc[4], qs[4];
+                    tmem_ld16x256b_x1(tm16 + TM_PU + 8 * j, acc);
+                    tmem_ld16x256b_x1(tq + 8 * j, qs);
+                    if (i0 < rows) store2(o0 + 8 * j, g0 * qs[0] + acc[0], g0 * qs[1] + acc[1]);
+                    if (i1 < rows) store2(o1 + 8 * j, g1 * qs[2] + acc[2], g1 * qs[3] + acc[3]);
                 }
             }
             tc_fence_before();
@@ -816,8 +820,9 @@ cudaError_t launch_t(const ChunkParams &p, cudaStream_t stream)
 {
     using Smem = TcSmem<D>;
     const uint64_t n_tok = (uint64_t)p.B * p.T;
-    CUtensorMap tq, tk;
-    if (!make_tmap(&tq, p.q, n_tok, (uint64_t)p.H * D) || !make_tmap(&tk, p.k, n_tok, (uint64_t)p.H * D))
+    CUtensorMap tq, tk, tv;
+    if (!make_tmap(&tq, p.q, n_tok, (uint64_t)p.H * D) || !make_tmap(&tk, p.k, n_tok, (uint64_t)p.H * D) ||
+        !make_tmap(&tv, p.v, n_tok, (uint64_t)p.H * D))
         return cudaErrorInvalidValue;
     auto kern = kla_chunk_tc_kernel<D, OUT>;
     const int smem = (int)sizeof(Smem) + 1024;
@@ -832,7 +837,7 @@ cudaError_t launch_t(const ChunkParams &p, cudaStream_t stream)
         memset(tbuf, 0, 3 * 64 * 16 * sizeof(long long));
         ChunkParams pt = p;
         pt.trace = tbuf;
-        kern<<<grid, NT, smem, stream>>>(tq, tk, pt);
+        kern<<<grid, NT, smem, stream>>>(tq, tk, tv, pt);
         cudaDeviceSynchronize();
         const char *tf = getenv("KLA_TRACE_FILE");
         FILE *f = tf ? fopen(tf, "w") : nullptr;
@@ -849,7 +854,7 @@ cudaError_t launch_t(const ChunkParams &p, cudaStream_t stream)
         return cudaGetLastError();
     }
 #endif
-    kern<<<grid, NT, smem, stream>>>(tq, tk, p);
+    kern<<<grid, NT, smem, stream>>>(tq, tk, tv, p);
     count_launch(1);
     return cudaGetLastError();
 }

@@ -285,7 +285,11 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     const uint32_t tmem = sm.tmem_base;
     const uint32_t tm_lane = tmem + ((uint32_t)((warp & 3) * 32) << 16);  // this warp's 32 TMEM lanes
 
-    auto wait = [&](int b, uint32_t parity) -> bool { return bar_wait(&sm.bar[b], parity, &sm.abort_flag); };
+    // fast path inline (the phase is often complete already), polling loop out of line
+    auto wait = [&](int b, uint32_t parity) -> bool {
+        if (mbar_try_wait(&sm.bar[b], parity)) return true;
+        return bar_wait(&sm.bar[b], parity, &sm.abort_flag);
+    };
     // one arrival per warp, after the warp's shared-memory writes are visible to the async proxy
     auto warp_arrive = [&](int b) {
         __syncwarp();
@@ -326,38 +330,35 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         };
         auto wwait = [&](int b, uint32_t parity) -> bool { return __all_sync(0xffffffffu, wait(b, parity)); };
         // four MMAs (K = 64): operand descriptors advance by astep / bstep (16-byte units) per K-step
-        auto seq = [&](uint32_t d, uint64_t a, uint64_t astep, uint64_t b, uint64_t bstep, uint32_t idesc, uint32_t acc) {
-#pragma unroll
-            for (int s = 0; s < 4; ++s) mma_bf16_ss(d, a + s * astep, b + s * bstep, idesc, s > 0 ? 1u : acc);
-        };
+#define KLA_SEQ(d, a, astep, b, bstep, idesc, acc) mma4_bf16_lo<astep, bstep>(d, a, b, idesc, acc)
         // Descriptors: everything except the 14-bit start-address field is fixed, so a K-step is an add.
-        const uint64_t d_kq0 = smem_desc_sw128(smem_u32(sm.kq[0]), 16, 1024);             // K-major views of a stage
-        const uint64_t d_kt0 = smem_desc_sw128(smem_u32(sm.kq[0]), KB * 8192, 1024);      // K^T (MN-major) view
-        const uint64_t d_sh = smem_desc_sw128(smem_u32(sm.s_hi), 16, 1024), d_sl = smem_desc_sw128(smem_u32(sm.s_lo), 16, 1024);
-        const uint64_t d_th = smem_desc_sw128(smem_u32(sm.t_hi), 16, 1024), d_tl = smem_desc_sw128(smem_u32(sm.t_lo), 16, 1024);
-        const uint64_t d_ph = smem_desc_sw128(smem_u32(sm.p_hi), 16, 1024), d_pl = smem_desc_sw128(smem_u32(sm.p_lo), 16, 1024);
-        const uint64_t d_rh = smem_desc_sw128(smem_u32(sm.ru_hi), 16, 1024), d_rl = smem_desc_sw128(smem_u32(sm.ru_lo), 16, 1024);
-        const uint64_t d_dh = smem_desc_sw128(smem_u32(sm.du_hi), 16, 1024), d_dl = smem_desc_sw128(smem_u32(sm.du_lo), 16, 1024);
-        constexpr uint64_t STAGE_STEP = (uint64_t)(Smem::KQ_BYTES >> 4);
+        const uint32_t d_kq0 = desc_lo(smem_desc_sw128(smem_u32(sm.kq[0]), 16, 1024));             // K-major views of a stage
+        const uint32_t d_kt0 = desc_lo(smem_desc_sw128(smem_u32(sm.kq[0]), KB * 8192, 1024));      // K^T (MN-major) view
+        const uint32_t d_sh = desc_lo(smem_desc_sw128(smem_u32(sm.s_hi), 16, 1024)), d_sl = desc_lo(smem_desc_sw128(smem_u32(sm.s_lo), 16, 1024));
+        const uint32_t d_th = desc_lo(smem_desc_sw128(smem_u32(sm.t_hi), 16, 1024)), d_tl = desc_lo(smem_desc_sw128(smem_u32(sm.t_lo), 16, 1024));
+        const uint32_t d_ph = desc_lo(smem_desc_sw128(smem_u32(sm.p_hi), 16, 1024)), d_pl = desc_lo(smem_desc_sw128(smem_u32(sm.p_lo), 16, 1024));
+        const uint32_t d_rh = desc_lo(smem_desc_sw128(smem_u32(sm.ru_hi), 16, 1024)), d_rl = desc_lo(smem_desc_sw128(smem_u32(sm.ru_lo), 16, 1024));
+        const uint32_t d_dh = desc_lo(smem_desc_sw128(smem_u32(sm.du_hi), 16, 1024)), d_dl = desc_lo(smem_desc_sw128(smem_u32(sm.du_lo), 16, 1024));
+        constexpr uint32_t STAGE_STEP = (uint32_t)(Smem::KQ_BYTES >> 4);
 
         auto mma1 = [&](int c) {  // [K;Q] K^T -> D1 buffer c & 1
-            const uint64_t a0 = d_kq0 + (uint64_t)(c % NSTAGE) * STAGE_STEP;
+            const uint32_t a0 = d_kq0 + (uint32_t)(c % NSTAGE) * STAGE_STEP;
 #pragma unroll 1
-            for (int kb = 0; kb < KB; ++kb) seq(tmem + TM_D1 + (uint32_t)(c & 1) * 64, a0 + kb * 1024, 2, a0 + kb * 1024, 2, ID_G, kb > 0);
+            for (int kb = 0; kb < KB; ++kb) KLA_SEQ(tmem + TM_D1 + (uint32_t)(c & 1) * 64, a0 + kb * 1024, 2, a0 + kb * 1024, 2, ID_G, kb > 0);
             mma_commit(&sm.bar[B_D1_DONE0 + (c & 1)]);
         };
         // [K or Q](c) S_0 -> d; qoff = 512 selects the Q tile of a block
-        auto mma_xs = [&](uint32_t d, uint64_t k0, uint64_t qoff) {
+        auto mma_xs = [&](uint32_t d, uint32_t k0, uint32_t qoff) {
 #pragma unroll 1
-            for (int kb = 0; kb < KB; ++kb) seq(d, k0 + qoff + kb * 1024, 2, d_sh + kb * 512, 128, ID_S, kb > 0);
+            for (int kb = 0; kb < KB; ++kb) KLA_SEQ(d, k0 + qoff + kb * 1024, 2, d_sh + kb * 512, 128, ID_S, kb > 0);
 #pragma unroll 1
-            for (int kb = 0; kb < KB; ++kb) seq(d, k0 + qoff + kb * 1024, 2, d_sl + kb * 512, 128, ID_S, 1);
+            for (int kb = 0; kb < KB; ++kb) KLA_SEQ(d, k0 + qoff + kb * 1024, 2, d_sl + kb * 512, 128, ID_S, 1);
         };
         // three-term product (a_hi + a_lo)(b_hi + b_lo) ~ a_hi b_hi + a_hi b_lo + a_lo b_hi, K = 64
-        auto mma_3 = [&](uint32_t d, uint64_t ah, uint64_t al, uint64_t bh, uint64_t bl) {
-            seq(d, ah, 2, bh, 128, ID_S, 0);
-            seq(d, ah, 2, bl, 128, ID_S, 1);
-            seq(d, al, 2, bh, 128, ID_S, 1);
+        auto mma_3 = [&](uint32_t d, uint32_t ah, uint32_t al, uint32_t bh, uint32_t bl) {
+            KLA_SEQ(d, ah, 2, bh, 128, ID_S, 0);
+            KLA_SEQ(d, ah, 2, bl, 128, ID_S, 1);
+            KLA_SEQ(d, al, 2, bh, 128, ID_S, 1);
         };
         bool ok = true;
         for (int c = 0; c < NSTAGE && c < nchunks; ++c) issue_tma(c);
@@ -371,8 +372,8 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         }
         for (int c = 0; ok && c < nchunks; ++c) {
             const uint32_t ph = (uint32_t)(c & 1);
-            const uint64_t k0 = d_kq0 + (uint64_t)(c % NSTAGE) * STAGE_STEP;
-            const uint64_t kt0 = d_kt0 + (uint64_t)(c % NSTAGE) * STAGE_STEP;
+            const uint32_t k0 = d_kq0 + (uint32_t)(c % NSTAGE) * STAGE_STEP;
+            const uint32_t kt0 = d_kt0 + (uint32_t)(c % NSTAGE) * STAGE_STEP;
             // MMA-1(c+1): as early as its inputs and its D1 buffer allow
             if (c + 1 < nchunks) {
                 if (!(ok = wwait(B_FULL0 + (c + 1) % NSTAGE, (uint32_t)(((c + 1) / NSTAGE) & 1)))) break;
@@ -408,8 +409,8 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             tc_fence_after();
             // A = K^T: M = d_k (64-wide blocks KB*8192 bytes apart; for d_k = 64 the second block
             // is the Q tile, whose rows land in TMEM lanes 64..127 and are ignored), K = tokens
-            seq(tmem + TM_DS, kt0, 128, d_dh, 128, ID_DS, 0);
-            seq(tmem + TM_DS, kt0, 128, d_dl, 128, ID_DS, 1);
+            KLA_SEQ(tmem + TM_DS, kt0, 128, d_dh, 128, ID_DS, 0);
+            KLA_SEQ(tmem + TM_DS, kt0, 128, d_dl, 128, ID_DS, 1);
             mma_commit(&sm.bar[B_D5_DONE]);
             if (!(ok = wwait(B_P_READY, ph))) break;
             tc_fence_after();

@@ -132,6 +132,47 @@ __device__ __forceinline__ void mma_bf16_ss(uint32_t tmem_d, uint64_t adesc, uin
         ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+// The same instruction with the descriptors given by their low words only.  Every descriptor built by
+// smem_desc_sw128 with sbo = 1024 has the same high word (stride offset, version, swizzle mode), and a K-step
+// or a tile switch changes only the 14-bit start-address field, so operand arithmetic stays in 32 bits.
+constexpr uint32_t DESC_HI_SW128_SBO1024 = (1024u >> 4) | (1u << 14) | (2u << 29);
+__device__ __forceinline__ uint32_t desc_lo(uint64_t desc) { return (uint32_t)desc; }
+__device__ __forceinline__ void mma_bf16_lo(uint32_t tmem_d, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p, e;\n\t.reg .b64 da, db;\n\t"
+        "mov.b64 da, {%1, %5};\n\tmov.b64 db, {%2, %5};\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "elect.sync _|e, 0xffffffff;\n\t"
+        "@e tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t}"
+        ::"r"(tmem_d), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "n"(DESC_HI_SW128_SBO1024)
+        : "memory");
+}
+// Four MMAs over K = 64 in one block: one election, descriptor low words advanced by the compile-time steps
+// ASTEP / BSTEP (16-byte units) per K-step.  The first MMA overwrites the accumulator unless `accumulate`.
+template <uint32_t ASTEP, uint32_t BSTEP>
+__device__ __forceinline__ void mma4_bf16_lo(uint32_t tmem_d, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p, e;\n\t.reg .b64 da, db;\n\t.reg .b32 ra, rb;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "elect.sync _|e, 0xffffffff;\n\t"
+        "@!e bra MMA4_DONE;\n\t"
+        "mov.b64 da, {%1, %5};\n\tmov.b64 db, {%2, %5};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t"
+        "add.u32 ra, %1, %6;\n\tadd.u32 rb, %2, %7;\n\t"
+        "mov.b64 da, {ra, %5};\n\tmov.b64 db, {rb, %5};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, 1;\n\t"
+        "add.u32 ra, ra, %6;\n\tadd.u32 rb, rb, %7;\n\t"
+        "mov.b64 da, {ra, %5};\n\tmov.b64 db, {rb, %5};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, 1;\n\t"
+        "add.u32 ra, ra, %6;\n\tadd.u32 rb, rb, %7;\n\t"
+        "mov.b64 da, {ra, %5};\n\tmov.b64 db, {rb, %5};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, 1;\n\t"
+        "MMA4_DONE:\n\t}"
+        ::"r"(tmem_d), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "n"(DESC_HI_SW128_SBO1024), "n"(ASTEP), "n"(BSTEP)
+        : "memory");
+}
 // Arrive on an mbarrier once all MMAs issued so far by this warp's elected lane have completed
 // (same calling convention: converged warp, one elected lane issues).
 __device__ __forceinline__ void mma_commit(uint64_t *bar)

@@ -129,6 +129,14 @@ __device__ __noinline__ bool bar_wait(uint64_t *bar, uint32_t parity, volatile i
     }
 }
 
+// Warp-uniform wait for the control warp: every lane polls, the warp leaves together.  Out of line: the control
+// program calls it a dozen times per chunk.
+__device__ __noinline__ bool warp_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag)
+{
+    const bool ok = mbar_try_wait(bar, parity) || bar_wait(bar, parity, abort_flag);
+    return __all_sync(0xffffffffu, ok);
+}
+
 __device__ __forceinline__ void pg_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 __device__ __forceinline__ void half_sync() { asm volatile("bar.sync 3, 64;" ::: "memory"); }
 // Barrier over the pre group that also ORs a flag: makes "some thread's wait gave up" a collective
@@ -328,7 +336,7 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             }
             __syncwarp();
         };
-        auto wwait = [&](int b, uint32_t parity) -> bool { return __all_sync(0xffffffffu, wait(b, parity)); };
+        auto wwait = [&](int b, uint32_t parity) -> bool { return warp_wait(&sm.bar[b], parity, &sm.abort_flag); };
         // four MMAs (K = 64): operand descriptors advance by astep / bstep (16-byte units) per K-step
 #define KLA_SEQ(d, a, astep, b, bstep, idesc, acc) mma4_bf16_lo<astep, bstep>(d, a, b, idesc, acc)
         // Descriptors: everything except the 14-bit start-address field is fixed, so a K-step is an add.
@@ -347,34 +355,24 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             for (int kb = 0; kb < KB; ++kb) KLA_SEQ(tmem + TM_D1 + (uint32_t)(c & 1) * 64, a0 + kb * 1024, 2, a0 + kb * 1024, 2, ID_G, kb > 0);
             mma_commit(&sm.bar[B_D1_DONE0 + (c & 1)]);
         };
-        // [K or Q](c) S_0 -> d; qoff = 512 selects the Q tile of a block
+        // [K or Q](c) S_0 -> d; qoff = 512 selects the Q tile of a block; S_0 = S_hi + S_lo
         auto mma_xs = [&](uint32_t d, uint32_t k0, uint32_t qoff) {
 #pragma unroll 1
-            for (int kb = 0; kb < KB; ++kb) KLA_SEQ(d, k0 + qoff + kb * 1024, 2, d_sh + kb * 512, 128, ID_S, kb > 0);
-#pragma unroll 1
-            for (int kb = 0; kb < KB; ++kb) KLA_SEQ(d, k0 + qoff + kb * 1024, 2, d_sl + kb * 512, 128, ID_S, 1);
+            for (int t = 0; t < 2 * KB; ++t) {
+                const uint32_t kb = (uint32_t)t & (KB - 1);
+                KLA_SEQ(d, k0 + qoff + kb * 1024, 2, (t >= KB ? d_sl : d_sh) + kb * 512, 128, ID_S, t > 0);
+            }
         };
         // three-term product (a_hi + a_lo)(b_hi + b_lo) ~ a_hi b_hi + a_hi b_lo + a_lo b_hi, K = 64
         auto mma_3 = [&](uint32_t d, uint32_t ah, uint32_t al, uint32_t bh, uint32_t bl) {
-            KLA_SEQ(d, ah, 2, bh, 128, ID_S, 0);
-            KLA_SEQ(d, ah, 2, bl, 128, ID_S, 1);
-            KLA_SEQ(d, al, 2, bh, 128, ID_S, 1);
+#pragma unroll 1
+            for (int t = 0; t < 3; ++t) KLA_SEQ(d, t == 2 ? al : ah, 2, t == 1 ? bl : bh, 128, ID_S, t > 0);
         };
         bool ok = true;
         for (int c = 0; c < NSTAGE && c < nchunks; ++c) issue_tma(c);
         issue_tma_v(0);
-        // MMA-1(0)
-        ok = wwait(B_FULL0, 0);
-        if (ok && nchunks == 1 && last_rows < C) ok = wwait(B_TAIL_READY, 0);
-        if (ok) {
-            tc_fence_after();
-            mma1(0);
-        }
-        for (int c = 0; ok && c < nchunks; ++c) {
-            const uint32_t ph = (uint32_t)(c & 1);
-            const uint32_t k0 = d_kq0 + (uint32_t)(c % NSTAGE) * STAGE_STEP;
-            const uint32_t kt0 = d_kt0 + (uint32_t)(c % NSTAGE) * STAGE_STEP;
-            // MMA-1(c+1): as early as its inputs and its D1 buffer allow
+        // iteration c issues MMA-1(c+1) first, as early as its inputs and its D1 buffer allow; c = -1 does only that
+        for (int c = -1; ok && c < nchunks; ++c) {
             if (c + 1 < nchunks) {
                 if (!(ok = wwait(B_FULL0 + (c + 1) % NSTAGE, (uint32_t)(((c + 1) / NSTAGE) & 1)))) break;
                 if (c + 2 == nchunks && last_rows < C)
@@ -384,14 +382,20 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 tc_fence_after();
                 mma1(c + 1);
             }
+            if (c < 0) continue;
+            const uint32_t ph = (uint32_t)(c & 1);
+            const uint32_t k0 = d_kq0 + (uint32_t)(c % NSTAGE) * STAGE_STEP;
+            const uint32_t kt0 = d_kt0 + (uint32_t)(c % NSTAGE) * STAGE_STEP;
             KLA_TR(0, c, 0);
             // MMA-2(c): K S_0 -> TM_KS (on the chain), then Q S_0 -> TM_QS[c&1] (needed only for the outputs)
             if (!(ok = wwait(B_S_READY, ph))) break;
             KLA_TR(0, c, 1);
             tc_fence_after();
-            mma_xs(tmem + TM_KS, k0, 0);
-            mma_commit(&sm.bar[B_D2_DONE]);
-            mma_xs(tmem + ((c & 1) ? TM_QS1 : TM_QS0), k0, 512);
+#pragma unroll 1
+            for (int x = 0; x < 2; ++x) {
+                mma_xs(tmem + (x == 0 ? TM_KS : ((c & 1) ? TM_QS1 : TM_QS0)), k0, x * 512);
+                if (x == 0) mma_commit(&sm.bar[B_D2_DONE]);
+            }
             KLA_TR(0, c, 2);
             // MMA-3(c): U = T rhs
             if (!(ok = wwait(B_T_READY, ph))) break;
@@ -409,8 +413,8 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             tc_fence_after();
             // A = K^T: M = d_k (64-wide blocks KB*8192 bytes apart; for d_k = 64 the second block
             // is the Q tile, whose rows land in TMEM lanes 64..127 and are ignored), K = tokens
-            KLA_SEQ(tmem + TM_DS, kt0, 128, d_dh, 128, ID_DS, 0);
-            KLA_SEQ(tmem + TM_DS, kt0, 128, d_dl, 128, ID_DS, 1);
+#pragma unroll 1
+            for (int t = 0; t < 2; ++t) KLA_SEQ(tmem + TM_DS, kt0, 128, t ? d_dl : d_dh, 128, ID_DS, t);
             mma_commit(&sm.bar[B_D5_DONE]);
             if (!(ok = wwait(B_P_READY, ph))) break;
             tc_fence_after();
@@ -526,9 +530,11 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 }
             }
             if (pg_any(!okc)) break;   // also publishes the decay sums to the whole group
+            KLA_TR(1, c, 9);
             if (is_g) {
                 // ---- X = A^- o K K^T from MMA-1 (this thread: row i, 32 columns) and beta_i ----------------------------
                 okc = wait(B_D1_DONE0 + (c & 1), (uint32_t)((c >> 1) & 1));
+                KLA_TR(1, c, 10);
                 if (okc) {
                     tc_fence_after();
                     if (live) {
@@ -555,6 +561,7 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                         // beta_i = eta_i / (||k_i||^2 + eps), Eq. 3; rows past the end of the sequence get 0
                         if (chh == q) sm.beta[sc][i] = (i < rows) ? eta_cur / (dg + p.eps) : 0.f;
                     }
+                    KLA_TR(1, c, 11);
                     tc_fence_before();
                     warp_arrive(B_D1_FREE0 + (c & 1));
                 }

@@ -53,6 +53,9 @@ constexpr int C = 64;    // chunk length
 constexpr int NS = 64;   // state columns per CTA
 constexpr int PG_T = 256, CG_T = 256;
 constexpr int NT = PG_T + CG_T + 32;
+// Thread layout: warp 0 control, warps 1..8 chain group, warps 9..16 pre group: the roles on the serial chain
+// sit in the lowest warp slots, which the warp schedulers favour when several warps are ready.
+constexpr int CG_BASE = 32, PG_BASE = 32 + CG_T;
 constexpr int NSTAGE = 3;
 constexpr long long WAIT_LIMIT = 2000000000LL;  // SM clocks (~1 s) before a wait gives up
 constexpr float LOG2E = 1.4426950408889634f;
@@ -119,8 +122,10 @@ __device__ __noinline__ bool bar_wait(uint64_t *bar, uint32_t parity, volatile i
     const long long t0 = clock64();
     while (true) {
 #pragma unroll 1
-        for (int i = 0; i < 32; ++i)
+        for (int i = 0; i < 64; ++i) {
             if (mbar_try_wait(bar, parity)) return true;
+            __nanosleep(32);   // a polling warp is always ready to issue: keep it from crowding out working warps
+        }
         if (*abort_flag) return false;
         if (clock64() - t0 > WAIT_LIMIT) {
             *abort_flag = 1;
@@ -157,7 +162,7 @@ __device__ __forceinline__ bool pg_any(bool flag)
 // role r (0 control, 1 pre, 2 chain), chunk c, event e -> trace[(r * 64 + c) * 16 + e]
 #define KLA_TR(r, c, e)                                                                        \
     do {                                                                                       \
-        if (p.trace && blockIdx.x == 0 && (c) < 64 && (((r) == 0 && lane == 0) || ((r) == 1 && tid == 0) || ((r) == 2 && tid == PG_T))) \
+        if (p.trace && blockIdx.x == 0 && (c) < 64 && (((r) == 0 && lane == 0) || ((r) == 1 && tid == PG_BASE) || ((r) == 2 && tid == CG_BASE))) \
             p.trace[((r) * 64 + (c)) * 16 + (e)] = clock64();                                  \
     } while (0)
 #else
@@ -304,7 +309,7 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         if (lane == 0) mbar_arrive(&sm.bar[b]);
     };
 
-    if (warp == NT / 32 - 1) {
+    if (warp == 0) {
         // =============================== control warp =====================================================
         // The whole warp runs this role in lock step: waits are taken by every lane, TMA loads are issued
         // by lane 0 and tensor-core instructions by the lane that elect.sync picks.
@@ -427,16 +432,16 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 issue_tma(c + NSTAGE);
             }
         }
-    } else if (warp < PG_T / 32) {
+    } else if (warp >= PG_BASE / 32) {
         // =============================== pre group ==========================================================
         // Warps 0, 1, 4, 5 hold rows of K K^T (TMEM lanes 0..63), warps 2, 3, 6, 7 rows of Q K^T (lanes 64..127).
         // Iteration c: the first set forms X(c) while the second forms P(c-1); then all eight warps invert.
-        const int pt = tid;                       // 0..255
-        const int q = warp & 3, chh = warp >> 2;  // TMEM lane quadrant, column half of D1
+        const int pt = tid - PG_BASE;             // 0..255
+        const int q = warp & 3, chh = (warp - PG_BASE / 32) >> 2;  // TMEM lane quadrant, column half of D1
         const bool is_g = q < 2;
         const int i = (q & 1) * 32 + lane;        // row of K K^T or of Q K^T held by this thread
         const bool live = chh <= (q & 1);         // otherwise all 32 columns are above the diagonal
-        const bool scan_warp = warp == 4;         // K K^T rows 0..31 x columns 32..63: no X work
+        const bool scan_warp = q == 0 && chh == 1;         // K K^T rows 0..31 x columns 32..63: no X work
         float la_next0 = 0.f, la_next1 = 0.f, eta_next = 0.f;
         auto fetch_gates = [&](int c) {
             if (scan_warp) {
@@ -627,7 +632,7 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         if (c == nchunks && !is_g) form_p(nchunks - 1);
     } else {
         // =============================== chain group ==========================================================
-        const int ct = tid - PG_T;              // 0..255
+        const int ct = tid - CG_BASE;           // 0..255
         const int q = warp & 3;                 // TMEM lane quadrant
         const int hf = ct >> 7;                 // column half: 0 -> columns 0..31, 1 -> 32..63
         const int srow = q * 32 + lane;         // state row (M = 128 accumulator layout, 32x32b loads)

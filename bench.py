@@ -28,6 +28,9 @@ if ROOT not in sys.path:
 
 METRIC = "chunk_fwd_throughput"
 UNIT = "Mtok/s"
+# dram__bytes_read.sum + dram__bytes_write.sum of one headline launch of the chunk kernel, from the ncu capture
+# summarised under profiles/; None while the kernel has changed since the counters were taken.
+CHUNK_TC_DRAM_BYTES_PER_LAUNCH = None
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -55,6 +58,23 @@ def algorithmic_flops(n_tok, H, d, C=64):
     """Causal-half count of Algorithm 1 (right): K K^T, K S0, T.rhs, Q S0, Q K^T, (A o QK^T) U, K^T D U, solve."""
     per_token_head = 2 * C * (d + d) + 6 * d * d + C * C / 3.0
     return n_tok * H * per_token_head
+
+
+# ---- multi-rank aggregation (host logic; covered by a gloo test on CPU) ---------------------------------
+def max_over_ranks(value, device):
+    """Maximum of a per-rank scalar over all ranks of the default process group (identity without one)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([float(value)], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_mtok_per_s(tokens_per_rank, world, ms_per_step):
+    """Every rank processes its own batch (weak scaling): tokens of all ranks over the slowest rank's time."""
+    return world * tokens_per_rank / (ms_per_step * 1e-3) / 1e6
 
 
 # ---- clocks sampling ------------------------------------------------------------------------------------
@@ -127,7 +147,7 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    sample = dict(B=1, H=8, T=4096, d=128)
+    sample = dict(B=8, H=8, T=4096, d=128)
     for _ in range(args.warmup):
         oracle_sample_run(**sample)
     times, thr = [], 1
@@ -136,7 +156,7 @@ def run_reference(args):
         times.append(dt)
     ms = 1e3 * sum(times) / len(times)
     value = sample["B"] * sample["T"] / (ms / 1e3) / 1e6
-    desc = "%d of 8 sequences x 8 heads x 4096 tokens of the headline workload per step" % sample["B"]
+    desc = "the whole headline workload (%d sequences x 8 heads x 4096 tokens) per step" % sample["B"]
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
@@ -299,18 +319,13 @@ def run_ours(args):
     launches = launch_count() - n0
     if world > 1:
         dist.barrier()
-        tm = torch.tensor([total_ms], device=dev)
-        dist.all_reduce(tm, op=dist.ReduceOp.MAX)
-        total_ms = float(tm.item())
+    total_ms = max_over_ranks(total_ms, dev)
     ms = total_ms / args.steps
     tokens_all = world * B * T
-    value = tokens_all / (ms * 1e-3) / 1e6
+    value = whole_job_mtok_per_s(B * T, world, ms)
 
     e2e_ms, h2d, d2h = (float("nan"), 0, 0) if args.quick else e2e_leg(w, dev, max(2, min(args.steps, 5)), 2)
-    if world > 1:
-        tm = torch.tensor([e2e_ms], device=dev)
-        dist.all_reduce(tm, op=dist.ReduceOp.MAX)
-        e2e_ms = float(tm.item())
+    e2e_ms = max_over_ranks(e2e_ms, dev)
 
     if rank != 0:
         if world > 1:
@@ -325,16 +340,11 @@ def run_ours(args):
     achieved = nbytes / (ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": peak_src + " (burst copy)",
-                "kernel": "kla_chunk_tc_kernel" if os.environ.get("KLA_BENCH_SIMT") is None else "kla_chunk_simt_kernel",
+                "kernel": "kla_chunk_tc_kernel",
                 "algorithmic_bytes_per_launch": nbytes, "algorithmic_flops_per_launch": flops,
                 "tensor_time_us_at_peak": t_tc * 1e6, "hbm_time_us_at_peak": t_hbm * 1e6,
                 "frac_of_roofline_time": max(t_hbm, t_tc) / (ms * 1e-3)}
-    traffic_file = os.path.join(ROOT, "profiles", "traffic.json")
-    if os.path.exists(traffic_file):
-        try:
-            roofline["traffic"] = json.load(open(traffic_file)).get("chunk_fwd_cfg2_dram_bytes_per_launch")
-        except Exception:
-            pass
+    roofline["traffic"] = CHUNK_TC_DRAM_BYTES_PER_LAUNCH
 
     extras = {}
     if not args.quick:
@@ -345,9 +355,9 @@ def run_ours(args):
 
     cpu = None
     if not (args.no_cpu_baseline or args.quick):
-        v, thr, dt = oracle_sample_run(B=4)
+        v, thr, dt = oracle_sample_run(B=8, repeats=3)
         cpu = {"value": v, "unit": UNIT, "cores": thr, "kind": "oracle",
-               "sample": "4 of 8 sequences x 8 heads x 4096 tokens of the headline workload, %.1f s" % dt}
+               "sample": "the whole headline workload (8 sequences x 8 heads x 4096 tokens), best of 3 runs, %.1f s each" % dt}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(3, args.warmup), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",

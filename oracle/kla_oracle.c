@@ -8,11 +8,11 @@
  * What it computes: the token-by-token recurrence of Algorithm 1 (left panel, "Tokenwise update")
  * with the Kaczmarz coefficient of Eq. (3), applied to every (sequence, head) independently:
  *
- *     S~   = alpha_t * S_{t-1}                alpha_t = exp(log_alpha_t)      (Alg. 1 left, line 1)
- *     e_t  = v_t - S~^T k_t                                                    (line 2)
- *     beta = eta_t / (||k_t||^2 + eps)                                         (line 3, Eq. 3)
- *     S_t  = S~ + beta * k_t e_t^T                                             (line 4)
- *     o_t  = S_t^T q_t                                                         (line 5, see below)
+ *     S~   = alpha_t * S_{t-1}                alpha_t = exp(log_alpha_t)      (Alg. 1 left: decay)
+ *     e_t  = v_t - S~^T k_t                                                    (residual)
+ *     beta = eta_t / (||k_t||^2 + eps)                                         (coefficient, Eq. 3)
+ *     S_t  = S~ + beta * k_t e_t^T                                             (rank-one write)
+ *     o_t  = S_t^T q_t                                                         (read-out, see below)
  *
  * The state S is d_k x d_v (Section 2), stored row-major with d_v contiguous.
  * Readings taken where the paper is ambiguous:
@@ -40,23 +40,23 @@ static void kla_token_update(double *S, int d_k, int d_v, const double *q, const
                              double *e /* scratch d_v */, double *o)
 {
     const double alpha = exp(log_alpha);
-    /* line 1: decay */
+    /* decay */
     for (int i = 0; i < d_k; ++i)
         for (int j = 0; j < d_v; ++j) S[(size_t)i * d_v + j] *= alpha;
-    /* line 2: residual e = v - S~^T k */
+    /* residual e = v - S~^T k */
     for (int j = 0; j < d_v; ++j) e[j] = v[j];
     for (int i = 0; i < d_k; ++i)
         for (int j = 0; j < d_v; ++j) e[j] -= S[(size_t)i * d_v + j] * k[i];
-    /* line 3: Kaczmarz coefficient */
+    /* Kaczmarz coefficient, Eq. 3 */
     double nk = 0.0;
     for (int i = 0; i < d_k; ++i) nk += k[i] * k[i];
     const double beta = eta / (nk + eps);
-    /* line 4: rank-one write */
+    /* rank-one write */
     for (int i = 0; i < d_k; ++i) {
         const double bk = beta * k[i];
         for (int j = 0; j < d_v; ++j) S[(size_t)i * d_v + j] += bk * e[j];
     }
-    /* line 5: read-out from the post-write state */
+    /* read-out from the post-write state */
     for (int j = 0; j < d_v; ++j) o[j] = 0.0;
     for (int i = 0; i < d_k; ++i)
         for (int j = 0; j < d_v; ++j) o[j] += S[(size_t)i * d_v + j] * q[i];

@@ -58,6 +58,13 @@ typedef enum { KLA_F32 = 0, KLA_BF16 = 1 } kla_dtype;
 /* Force the CUDA-core fp32 chunk kernel even where the tensor-core kernel applies (used to
  * cross-check the two device paths against each other and against the oracle). */
 #define KLA_FLAG_FORCE_SIMT 1
+/* Segment-parallel scan of the tensor-core path (fixed-length input only).  Every chunk step is affine in the
+ * incoming state (Eqs. 7-9), so a sequence can be cut into G segments whose transition maps are found in
+ * parallel, chained, and the segments then run in parallel from their true start states: the same result up
+ * to rounding, about three times the state work, G times the parallelism.  By default the library decides
+ * from the shape (few long sequences -> segments) and the workspace query returns what that decision needs. */
+#define KLA_FLAG_NO_SEGMENTS 2            /* never cut sequences into segments                              */
+#define KLA_FLAG_SEGMENTS(g) ((g) << 8)   /* force g segments per sequence, 2 <= g <= 255 (fewer if T is short) */
 
 typedef struct {
     int32_t B;        /* sequences in the batch; packed (varlen) input: 1                       */
@@ -82,8 +89,10 @@ typedef struct {
 } kla_desc;
 
 /*
- * Scratch needed by kla_chunk_fwd for this descriptor and chunk length (may be 0).
- * Host-only computation; returns 0 for an invalid descriptor.
+ * Scratch needed by kla_chunk_fwd for this descriptor (shape, dtypes, flags) and chunk length; 0 unless the
+ * segment-parallel scan applies (then: per-segment transition maps and states, 3 x B x G x H x d_k x d_v fp32).
+ * Computed on the host (it reads the current device's SM count when a device is present); returns 0 for an
+ * invalid descriptor.  The same descriptor must be passed to kla_chunk_fwd with a workspace of at least this size.
  */
 size_t kla_chunk_fwd_workspace_bytes(const kla_desc *desc, int32_t chunk);
 

@@ -13,7 +13,13 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libkla_b200.so")
 
 KLA_F32, KLA_BF16 = 0, 1
-KLA_FLAG_NONE, KLA_FLAG_FORCE_SIMT = 0, 1
+KLA_FLAG_NONE, KLA_FLAG_FORCE_SIMT, KLA_FLAG_NO_SEGMENTS = 0, 1, 2
+
+
+def KLA_FLAG_SEGMENTS(g: int) -> int:
+    """Force g segments per sequence in the segment-parallel scan (include/kla.h)."""
+    return int(g) << 8
+
 
 EXPORTS = ["kla_chunk_fwd_workspace_bytes", "kla_chunk_fwd", "kla_decode_step", "kla_decode_steps",
            "kla_status_str", "kla_launch_count"]

@@ -63,6 +63,62 @@ static kla_status check_chunk(const kla_desc *d, const void *q, const void *k, c
     return KLA_OK;
 }
 
+// ---- segment-parallel scan: when to use it, and the workspace it needs ----------------------------------------------
+struct SegPlan {
+    int G = 0;            // segments per sequence (0: plain launch)
+    int seg_len = 0;      // tokens per segment (a multiple of the chunk length)
+    size_t off_map = 0, off_local = 0, off_start = 0, bytes = 0;   // workspace layout; cu_seg sits at offset 0
+};
+
+static int sm_count()
+{
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+        return 148;
+    return n;
+}
+
+// Few long sequences leave most SMs idle (one CTA per sequence x head x slice, each walking its chunks in series).
+// Cutting every sequence into G segments costs about two more passes of state work but runs G times as many CTAs.
+static SegPlan plan_segments(const kla_desc *d, int32_t chunk)
+{
+    SegPlan pl;
+    if (d->cu_seqlens || (d->flags & (KLA_FLAG_FORCE_SIMT | KLA_FLAG_NO_SEGMENTS)) || !chunk_tc_supported(d->d_k, chunk, d->io_dtype))
+        return pl;
+    const int chunks = (d->T + 63) / 64;
+    const int units = d->B * d->H * (d->d_k / 64);
+    const int forced = (d->flags >> 8) & 0xff;
+    int best_len = 0;
+    if (forced >= 2) {
+        best_len = (chunks + forced - 1) / forced;
+    } else if (forced == 0) {
+        const int sms = sm_count();
+        auto waves = [&](int ctas) { return (ctas + sms - 1) / sms; };
+        const double plain = (double)waves(units) * chunks;
+        double best = 0.75 * plain;   // only worth it for a clear win
+        for (int G = 2; G <= 32 && chunks / G >= 8; ++G) {
+            const int len = (chunks + G - 1) / G, Ge = (chunks + len - 1) / len;
+            if (Ge < 2) continue;
+            const double cost = 0.8 * waves(units * 2 * (Ge - 1)) * len + (double)waves(units * Ge) * len + 2.0 * Ge;
+            if (cost < best) {
+                best = cost;
+                best_len = len;
+            }
+        }
+    }
+    if (best_len <= 0) return pl;
+    pl.seg_len = best_len * 64;
+    pl.G = (d->T + pl.seg_len - 1) / pl.seg_len;
+    if (pl.G < 2) return SegPlan();
+    const size_t cu_bytes = (((size_t)d->B * pl.G + 1) * sizeof(int32_t) + 255) & ~(size_t)255;
+    const size_t st = (size_t)d->B * pl.G * d->H * d->d_k * d->d_v * sizeof(float);
+    pl.off_map = cu_bytes;
+    pl.off_local = cu_bytes + st;
+    pl.off_start = cu_bytes + 2 * st;
+    pl.bytes = cu_bytes + 3 * st;
+    return pl;
+}
+
 }  // namespace kla
 
 using namespace kla;
@@ -72,8 +128,8 @@ extern "C" {
 size_t kla_chunk_fwd_workspace_bytes(const kla_desc *desc, int32_t chunk)
 {
     if (check_common(desc) != KLA_OK) return 0;
-    (void)chunk;
-    return 0;  // both chunk kernels keep every intermediate on chip
+    // the chunk kernels keep every intermediate on chip; only the segment-parallel scan needs scratch
+    return plan_segments(desc, chunk).bytes;
 }
 
 kla_status kla_chunk_fwd(const kla_desc *desc, const void *q, const void *k, const void *v,
@@ -94,6 +150,7 @@ kla_status kla_chunk_fwd(const kla_desc *desc, const void *q, const void *k, con
     p.cu_seqlens = desc->cu_seqlens;
     p.status_word = desc->status_word;
     p.trace = nullptr;
+    p.seg_pass = 0; p.seg_G = 0; p.map_state = nullptr;
     p.B = desc->B; p.T = desc->T; p.H = desc->H; p.n_seq = desc->n_seq;
     p.eps = eps;
     if (desc->T == 0) {
@@ -108,6 +165,26 @@ kla_status kla_chunk_fwd(const kla_desc *desc, const void *q, const void *k, con
     }
     cudaStream_t stream = (cudaStream_t)desc->stream;
     cudaError_t err;
+    const SegPlan pl = plan_segments(desc, chunk);
+    if (pl.G >= 2) {
+        char *ws = (char *)desc->workspace;
+        int32_t *cu_seg = (int32_t *)ws;
+        float *map = (float *)(ws + pl.off_map), *local = (float *)(ws + pl.off_local), *start = (float *)(ws + pl.off_start);
+        if (launch_seg_bounds(cu_seg, desc->B, desc->T, pl.G, pl.seg_len, stream) != cudaSuccess) return KLA_ERR_LAUNCH;
+        ChunkParams p1 = p;   // pass 1: transition map and zero-start state of every segment but the last
+        p1.cu_seqlens = cu_seg; p1.n_seq = desc->B * pl.G;
+        p1.init_state = nullptr; p1.final_state = local; p1.map_state = map;
+        p1.seg_pass = 1; p1.seg_G = pl.G;
+        if (launch_chunk_tc(p1, desc->d_k, desc->io_dtype, desc->out_dtype, stream) != cudaSuccess) return KLA_ERR_LAUNCH;
+        if (launch_seg_combine(init_state, map, local, start, desc->B, desc->H, pl.G, desc->d_k, stream) != cudaSuccess)
+            return KLA_ERR_LAUNCH;
+        ChunkParams p3 = p;   // pass 3: every segment from its true start state
+        p3.cu_seqlens = cu_seg; p3.n_seq = desc->B * pl.G;
+        p3.init_state = start;
+        p3.seg_pass = 3; p3.seg_G = pl.G;
+        err = launch_chunk_tc(p3, desc->d_k, desc->io_dtype, desc->out_dtype, stream);
+        return err == cudaSuccess ? KLA_OK : KLA_ERR_LAUNCH;
+    }
     if (!(desc->flags & KLA_FLAG_FORCE_SIMT) && chunk_tc_supported(desc->d_k, chunk, desc->io_dtype))
         err = launch_chunk_tc(p, desc->d_k, desc->io_dtype, desc->out_dtype, stream);
     else

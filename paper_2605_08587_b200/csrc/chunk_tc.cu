@@ -240,9 +240,16 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     Smem &sm = *reinterpret_cast<Smem *>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int sl = blockIdx.x % SLICES;
-    const int h = (blockIdx.x / SLICES) % p.H;
-    const int n = blockIdx.x / (SLICES * p.H);
+    // plain launch: block = (sequence, head, slice).  Segment pass 1 doubles the slices (the second set carries
+    // the transition map) and skips each sequence's last segment; see ChunkParams.
+    const int nslices = p.seg_pass == 1 ? 2 * SLICES : SLICES;
+    const int sl2 = blockIdx.x % nslices;
+    const bool is_map = sl2 >= SLICES;
+    const int sl = sl2 % SLICES;
+    const int h = (blockIdx.x / nslices) % p.H;
+    int n = blockIdx.x / (nslices * p.H);
+    if (p.seg_pass == 1) n = (n / (p.seg_G - 1)) * p.seg_G + n % (p.seg_G - 1);
+    const bool no_out = p.seg_pass == 1;
 
     int tok0, len;
     if (p.cu_seqlens) {
@@ -253,8 +260,15 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         len = p.T;
     }
     const size_t state_off = (((size_t)n * p.H + h) * D) * D + (size_t)sl * NS;
+    // where this CTA's final state goes (null: nowhere)
+    float *fin = is_map ? p.map_state : p.final_state;
+    size_t fin_off = state_off;
+    if (p.seg_pass == 3 && fin) {
+        if (n % p.seg_G != p.seg_G - 1) fin = nullptr;
+        else fin_off = (((size_t)(n / p.seg_G) * p.H + h) * D) * D + (size_t)sl * NS;
+    }
 
-    if (len <= 0) {  // empty sequence: the final state is the initial state
+    if (len <= 0) {  // empty sequence: the final state is the initial state (never a segment: those are non-empty)
         if (p.final_state) {
             for (int i = tid; i < D * (NS / 4); i += NT) {
                 const int r = i / (NS / 4), c = (i % (NS / 4)) * 4;
@@ -397,7 +411,7 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             KLA_TR(0, c, 1);
             tc_fence_after();
 #pragma unroll 1
-            for (int x = 0; x < 2; ++x) {
+            for (int x = 0; x < (no_out ? 1 : 2); ++x) {
                 mma_xs(tmem + (x == 0 ? TM_KS : ((c & 1) ? TM_QS1 : TM_QS0)), k0, x * 512);
                 if (x == 0) mma_commit(&sm.bar[B_D2_DONE]);
             }
@@ -421,10 +435,12 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 #pragma unroll 1
             for (int t = 0; t < 2; ++t) KLA_SEQ(tmem + TM_DS, kt0, 128, t ? d_dl : d_dh, 128, ID_DS, t);
             mma_commit(&sm.bar[B_D5_DONE]);
-            if (!(ok = wwait(B_P_READY, ph))) break;
-            tc_fence_after();
-            mma_3(tmem + TM_PU, d_ph, d_pl, d_rh, d_rl);
-            mma_commit(&sm.bar[B_D4_DONE]);
+            if (!no_out) {
+                if (!(ok = wwait(B_P_READY, ph))) break;
+                tc_fence_after();
+                mma_3(tmem + TM_PU, d_ph, d_pl, d_rh, d_rl);
+                mma_commit(&sm.bar[B_D4_DONE]);
+            }
             KLA_TR(0, c, 7);
             // the K/Q stage of chunk c is free once MMA-5(c) has read it
             if (c + NSTAGE < nchunks) {
@@ -570,6 +586,8 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     tc_fence_before();
                     warp_arrive(B_D1_FREE0 + (c & 1));
                 }
+            } else if (no_out) {
+                warp_arrive(B_D1_FREE0 + (c & 1));   // nothing reads Q K^T: release this warp's share of D1(c)
             } else if (c > 0) {
                 okc = form_p(c - 1);
             }
@@ -629,7 +647,7 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             KLA_TR(1, c, 5);
         }
         // P of the last chunk
-        if (c == nchunks && !is_g) form_p(nchunks - 1);
+        if (c == nchunks && !is_g && !no_out) form_p(nchunks - 1);
     } else {
         // =============================== chain group ==========================================================
         const int ct = tid - CG_BASE;           // 0..255
@@ -643,7 +661,11 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         const uint32_t tm16 = tmem + ((uint32_t)(q * 32) << 16) + hf * 32;
 
         float S[32];
-        if (s_act && p.init_state) {
+        if (is_map) {
+            // transition map: start from the identity (columns sl * NS + hf * 32 .. of I)
+#pragma unroll
+            for (int c = 0; c < 32; ++c) S[c] = (srow == sl * NS + hf * 32 + c) ? 1.f : 0.f;
+        } else if (s_act && p.init_state) {
 #pragma unroll
             for (int c = 0; c < 32; c += 4) {
                 const float4 x = *reinterpret_cast<const float4 *>(p.init_state + state_off + (size_t)srow * D + hf * 32 + c);
@@ -697,8 +719,8 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 tmem_ld16x256b_x1(tm16 + TM_KS + 8 * j, acc);
                 const uint32_t o0 = off(i0, j), o1 = off(i1, j);
                 // V[i0][cp + 8j .. +1], V[i1][...]; rows past the end of the sequence are another sequence's tokens
-                const uint32_t va = (i0 < rows) ? *reinterpret_cast<const uint32_t *>(sm.vt + o0) : 0u;
-                const uint32_t vb = (i1 < rows) ? *reinterpret_cast<const uint32_t *>(sm.vt + o1) : 0u;
+                const uint32_t va = (i0 < rows && !is_map) ? *reinterpret_cast<const uint32_t *>(sm.vt + o0) : 0u;
+                const uint32_t vb = (i1 < rows && !is_map) ? *reinterpret_cast<const uint32_t *>(sm.vt + o1) : 0u;
                 const float2 fa = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&va));
                 const float2 fb = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&vb));
                 uint32_t hi, lo;
@@ -759,6 +781,7 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             KLA_TR(2, c, 7);
 
             // ---- outputs: O_i = gamma_i (Q S_0)_i + (P U)_i (off the chain) -----------------------------------------
+            if (no_out) continue;
             if (!wait(B_D4_DONE, ph)) break;
             KLA_TR(2, c, 8);
             tc_fence_after();
@@ -778,10 +801,10 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             tc_fence_before();
             KLA_TR(2, c, 9);
         }
-        if (!sm.abort_flag && p.final_state && s_act) {
+        if (!sm.abort_flag && fin && s_act) {
 #pragma unroll
             for (int c = 0; c < 32; c += 4)
-                *reinterpret_cast<float4 *>(p.final_state + state_off + (size_t)srow * D + hf * 32 + c) =
+                *reinterpret_cast<float4 *>(fin + fin_off + (size_t)srow * D + hf * 32 + c) =
                     make_float4(S[c], S[c + 1], S[c + 2], S[c + 3]);
         }
     }
@@ -841,7 +864,8 @@ cudaError_t launch_t(const ChunkParams &p, cudaStream_t stream)
     const int smem = (int)sizeof(Smem) + 1024;
     cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (err != cudaSuccess) return err;
-    const int grid = p.n_seq * p.H * (D / NS);
+    // segment pass 1: (seg_G - 1) segments per sequence, twice the slices; p.n_seq counts all segments there
+    const int grid = p.seg_pass == 1 ? (p.n_seq / p.seg_G) * (p.seg_G - 1) * p.H * 2 * (D / NS) : p.n_seq * p.H * (D / NS);
     if (grid == 0) return cudaSuccess;
 #ifdef KLA_TRACE
     {

@@ -20,6 +20,14 @@ struct ChunkParams {
     long long *trace;           // debug builds only (KLA_TRACE): per-event SM clock stamps; else null
     int32_t B, T, H, n_seq;
     float eps;
+    // Segment-parallel scan (tensor-core kernel only; all zero / null for a plain launch).
+    //   seg_pass 1: "sequence" index = a segment that is not the last of its sequence (seg_G segments per
+    //               sequence); no outputs; 2x the slices: the extra ones carry the transition map (state
+    //               started at the identity, v = 0) and write it to map_state.
+    //   seg_pass 3: every segment from its true start state; only the last segment of a sequence writes
+    //               final_state, at the sequence's index.
+    int32_t seg_pass, seg_G;
+    float *map_state;
 };
 
 struct DecodeParams {
@@ -38,6 +46,11 @@ cudaError_t launch_chunk_simt(const ChunkParams &p, int d, int chunk, int io_dty
                               cudaStream_t stream);
 cudaError_t launch_chunk_tc(const ChunkParams &p, int d, int io_dtype, int out_dtype,
                             cudaStream_t stream);
+// Segment-parallel helpers (segscan.cu).  cu_seg[b * G + g] = b * T + min(g * seg_len, T), one more entry = B * T.
+cudaError_t launch_seg_bounds(int32_t *cu_seg, int B, int T, int G, int seg_len, cudaStream_t stream);
+// start[b, 0] = init (or 0); start[b, g + 1] = map[b, g] . start[b, g] + local[b, g]   (d x d products, fp32)
+cudaError_t launch_seg_combine(const float *init_state, const float *map, const float *local, float *start, int B, int H,
+                               int G, int d, cudaStream_t stream);
 // True when the tensor-core kernel covers this case.
 bool chunk_tc_supported(int d, int chunk, int io_dtype);
 

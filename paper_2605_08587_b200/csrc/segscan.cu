@@ -1,0 +1,107 @@
+// Segment-parallel scan: the small kernels around the chunk kernel.
+//
+// Every chunk step is affine in the incoming state (Eqs. 7-9 are linear in S_0), so a run of chunks is too:
+//     S_end = Phi S_start + N,   Phi (d_k x d_k) = the state reached from the identity with v = 0,
+//                                N   (d_k x d_v) = the state reached from zero.
+// A long sequence is cut into G segments; pass 1 (the chunk kernel, no outputs) finds (Phi, N) of every segment
+// but the last in parallel; `seg_combine` below chains them serially -- G - 1 small fp32 products per head --
+// to get each segment's true start state; pass 3 (the chunk kernel again) then runs all segments in parallel.
+#include "common.cuh"
+
+namespace kla {
+
+namespace {
+
+__global__ void seg_bounds_kernel(int32_t *cu_seg, int B, int T, int G, int seg_len)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i > B * G) return;
+    if (i == B * G) {
+        cu_seg[i] = B * T;
+        return;
+    }
+    const int b = i / G, g = i % G;
+    cu_seg[i] = b * T + min(g * seg_len, T);
+}
+
+// One CTA per (sequence, head, 16-column slice of the state); thread r owns row r of the slice.
+template <int D>
+__global__ void __launch_bounds__(D) seg_combine_kernel(const float *init_state, const float *map, const float *local,
+                                                        float *start, int H, int G)
+{
+    constexpr int W = 16;
+    const int sl = blockIdx.x % (D / W);
+    const int h = (blockIdx.x / (D / W)) % H;
+    const int b = blockIdx.x / ((D / W) * H);
+    const int r = threadIdx.x;
+    __shared__ __align__(16) float S[2][D][W];
+
+    auto base = [&](int g) -> size_t { return ((size_t)(b * G + g) * H + h) * D * D; };
+    float cur[W];
+#pragma unroll
+    for (int c = 0; c < W; c += 4) {
+        float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (init_state) x = *reinterpret_cast<const float4 *>(init_state + ((size_t)b * H + h) * D * D + (size_t)r * D + sl * W + c);
+        cur[c] = x.x; cur[c + 1] = x.y; cur[c + 2] = x.z; cur[c + 3] = x.w;
+    }
+    for (int g = 0; g < G; ++g) {
+        // publish the start state of segment g
+        float *dst = start + base(g) + (size_t)r * D + sl * W;
+#pragma unroll
+        for (int c = 0; c < W; c += 4) {
+            const float4 x = make_float4(cur[c], cur[c + 1], cur[c + 2], cur[c + 3]);
+            *reinterpret_cast<float4 *>(dst + c) = x;
+            *reinterpret_cast<float4 *>(&S[g & 1][r][c]) = x;
+        }
+        if (g + 1 == G) break;
+        __syncthreads();
+        // next = Phi_g cur + N_g
+        const float *Mrow = map + base(g) + (size_t)r * D;
+        const float *Nrow = local + base(g) + (size_t)r * D + sl * W;
+        float acc[W];
+#pragma unroll
+        for (int c = 0; c < W; c += 4) {
+            const float4 x = *reinterpret_cast<const float4 *>(Nrow + c);
+            acc[c] = x.x; acc[c + 1] = x.y; acc[c + 2] = x.z; acc[c + 3] = x.w;
+        }
+#pragma unroll 2
+        for (int k = 0; k < D; k += 4) {
+            const float4 m = *reinterpret_cast<const float4 *>(Mrow + k);
+            const float mv[4] = {m.x, m.y, m.z, m.w};
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+#pragma unroll
+                for (int c = 0; c < W; c += 4) {
+                    const float4 s4 = *reinterpret_cast<const float4 *>(&S[g & 1][k + u][c]);
+                    acc[c] += mv[u] * s4.x; acc[c + 1] += mv[u] * s4.y; acc[c + 2] += mv[u] * s4.z; acc[c + 3] += mv[u] * s4.w;
+                }
+            }
+        }
+#pragma unroll
+        for (int c = 0; c < W; ++c) cur[c] = acc[c];
+        // the other buffer is written next; readers of this one are done after the next barrier
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_seg_bounds(int32_t *cu_seg, int B, int T, int G, int seg_len, cudaStream_t stream)
+{
+    const int n = B * G + 1;
+    seg_bounds_kernel<<<(n + 127) / 128, 128, 0, stream>>>(cu_seg, B, T, G, seg_len);
+    count_launch(1);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_seg_combine(const float *init_state, const float *map, const float *local, float *start, int B, int H,
+                               int G, int d, cudaStream_t stream)
+{
+    if (d == 128)
+        seg_combine_kernel<128><<<B * H * (128 / 16), 128, 0, stream>>>(init_state, map, local, start, H, G);
+    else
+        seg_combine_kernel<64><<<B * H * (64 / 16), 64, 0, stream>>>(init_state, map, local, start, H, G);
+    count_launch(1);
+    return cudaGetLastError();
+}
+
+}  // namespace kla

@@ -115,6 +115,28 @@ def test_workspace_query(lib):
     assert lib.kla_chunk_fwd_workspace_bytes(ctypes.byref(_desc()), 64) >= 0
 
 
+def test_workspace_grows_only_when_sequences_are_cut_into_segments(lib):
+    """Host logic of the segment-parallel scan: few long sequences get a workspace, many short ones do not,
+    flags force it on or off, and a missing workspace is refused before anything is launched."""
+    many = _desc(B=8, T=4096, H=8, d_k=128, d_v=128, n_seq=8)
+    assert lib.kla_chunk_fwd_workspace_bytes(ctypes.byref(many), 64) == 0
+    long1 = _desc(B=1, T=65536, H=8, d_k=128, d_v=128, n_seq=1)
+    need = lib.kla_chunk_fwd_workspace_bytes(ctypes.byref(long1), 64)
+    assert need > 0
+    state = 8 * 128 * 128 * 4
+    G = (need - 256) // (3 * state)
+    assert 2 <= G <= 32 and need == 256 + 3 * G * state        # cu_seg (padded) + map, local, start per segment
+    off = _desc(B=1, T=65536, H=8, d_k=128, d_v=128, n_seq=1, flags=2)
+    assert lib.kla_chunk_fwd_workspace_bytes(ctypes.byref(off), 64) == 0
+    forced = _desc(B=8, T=4096, H=8, d_k=128, d_v=128, n_seq=8, flags=4 << 8)
+    assert lib.kla_chunk_fwd_workspace_bytes(ctypes.byref(forced), 64) == 256 + 3 * 8 * 4 * state
+    assert lib.kla_chunk_fwd(ctypes.byref(forced), FAKE, FAKE, FAKE, FAKE, FAKE, 1e-6, 64, None, FAKE, None) == -7
+    # fp32 inputs and chunk 32 go to the CUDA-core kernel: never segmented
+    f32 = _desc(B=1, T=65536, H=8, d_k=128, d_v=128, n_seq=1, io_dtype=binding.KLA_F32)
+    assert lib.kla_chunk_fwd_workspace_bytes(ctypes.byref(f32), 64) == 0
+    assert lib.kla_chunk_fwd_workspace_bytes(ctypes.byref(long1), 32) == 0
+
+
 def test_binding_rejects_cpu_tensors():
     import torch
     from paper_2605_08587_b200 import kla_chunk_fwd

@@ -181,3 +181,35 @@ def test_config5_full_size_sampled():
     assert rel_err(np64(out[0][idx][:, heads]), ro) <= TOL_BF16
     assert rel_err(np64(fin[seqs][:, heads]), rf) <= TOL_BF16
     assert torch.isfinite(out).all() and torch.isfinite(fin).all()
+
+
+# ---- segment-parallel scan (long sequences cut into segments; same result up to rounding) ------------------
+from paper_2605_08587_b200 import KLA_FLAG_NO_SEGMENTS, KLA_FLAG_SEGMENTS  # noqa: E402
+
+
+@pytest.mark.parametrize("G", [2, 3, 7])
+@pytest.mark.parametrize("d", [64, 128])
+def test_forced_segments_match_oracle(G, d):
+    w = W.config3(B=2, H=2, T=1536 + 17, d=d, seed=200 + G)
+    _check_fixed(w, TOL_BF16, flags=KLA_FLAG_SEGMENTS(G))
+
+
+def test_segments_equal_plain_launch_closely():
+    w = W.config3(B=1, H=3, T=4096, seed=211)
+    o_p, f_p = gpu_chunk(w, flags=KLA_FLAG_NO_SEGMENTS)
+    o_s, f_s = gpu_chunk(w, flags=KLA_FLAG_SEGMENTS(4))
+    assert rel_err(np64(o_s), np64(o_p)) <= 2e-4
+    assert rel_err(np64(f_s), np64(f_p)) <= 2e-4
+
+
+def test_segments_without_init_state_and_without_final_state():
+    w = W.config2(B=1, H=2, T=1100, seed=213)
+    out, fin = gpu_chunk(w, flags=KLA_FLAG_SEGMENTS(3), want_final_state=False)
+    assert fin is None
+    ro, _ = oracle_chunk(w)
+    assert rel_err(np64(out), ro) <= TOL_BF16
+
+
+def test_more_segments_than_chunks_is_clamped():
+    w = W.config3(B=1, H=2, T=130, seed=215)
+    _check_fixed(w, TOL_BF16, flags=KLA_FLAG_SEGMENTS(9))

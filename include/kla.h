@@ -120,6 +120,30 @@ kla_status kla_chunk_fwd(const kla_desc *desc, const void *q, const void *k, con
                          const float *init_state, void *out, float *final_state);
 
 /*
+ * The same chunk forward for callers that cannot allocate device memory (no counterpart in the paper: this is a
+ * property of the library, not of the method).  kla_chunk_fwd needs a caller-provided workspace whenever it cuts
+ * long sequences into segments; a caller that has no allocator at hand -- code inside a region where its framework
+ * serves no allocations, a plugin that is handed nothing but its input and output buffers, a binding without
+ * cudaMalloc -- calls this instead.  desc->workspace and desc->workspace_bytes are ignored: the scratch is a fixed
+ * array of KLA_STATIC_SCRATCH_BYTES inside the library image, which every GPU that loads the library holds until
+ * the process exits.  The call itself allocates and frees nothing, on host or device.
+ *
+ *  - A shape whose scratch would exceed KLA_STATIC_SCRATCH_BYTES is refused with KLA_ERR_WORKSPACE before
+ *    anything is launched (kla_chunk_fwd_workspace_bytes tells what a shape needs; KLA_FLAG_NO_SEGMENTS makes
+ *    the need zero at the price of less parallelism).
+ *  - The first call on each device looks up that device's address of the array (with the device current, as
+ *    for every call); make that first call outside any stream capture.
+ *  - All calls share the one array and it keeps the previous call's contents.  Nothing in it has to start at
+ *    zero (a call writes every byte it later reads), but two calls that overlap on the GPU -- different streams,
+ *    or host threads racing on one stream -- would overwrite each other's segments: serialise them.
+ *  - Everything else (arguments, layouts, results, error codes) is exactly kla_chunk_fwd.
+ */
+#define KLA_STATIC_SCRATCH_BYTES (32u << 20)
+kla_status kla_chunk_fwd_static_scratch(const kla_desc *desc, const void *q, const void *k, const void *v,
+                                        const float *log_alpha, const float *eta, float eps, int32_t chunk,
+                                        const float *init_state, void *out, float *final_state);
+
+/*
  * One recurrent decode step (Algorithm 1 left) for B sequences x H heads; desc->T must be 1 and
  * desc->cu_seqlens NULL.
  *

@@ -3,5 +3,5 @@
 `binding` wraps the C ABI of include/kla.h; `workloads` draws the seeded synthetic inputs;
 `build` compiles the CUDA library in-tree.
 """
-from .binding import (KlaError, kla_chunk_fwd, kla_decode_step, kla_decode_steps, launch_count,  # noqa: F401
+from .binding import (KlaError, kla_chunk_fwd, kla_chunk_fwd_static_scratch, kla_decode_step, kla_decode_steps, launch_count,  # noqa: F401
                       KLA_F32, KLA_BF16, KLA_FLAG_NONE, KLA_FLAG_FORCE_SIMT, KLA_FLAG_NO_SEGMENTS, KLA_FLAG_SEGMENTS)

@@ -21,7 +21,7 @@ def KLA_FLAG_SEGMENTS(g: int) -> int:
     return int(g) << 8
 
 
-EXPORTS = ["kla_chunk_fwd_workspace_bytes", "kla_chunk_fwd", "kla_decode_step", "kla_decode_steps",
+EXPORTS = ["kla_chunk_fwd_workspace_bytes", "kla_chunk_fwd", "kla_chunk_fwd_static_scratch", "kla_decode_step", "kla_decode_steps",
            "kla_status_str", "kla_launch_count"]
 
 
@@ -57,6 +57,8 @@ def load():
     lib.kla_chunk_fwd_workspace_bytes.argtypes = [dp, ctypes.c_int32]
     lib.kla_chunk_fwd.restype = ctypes.c_int
     lib.kla_chunk_fwd.argtypes = [dp, vp, vp, vp, fp, fp, ctypes.c_float, ctypes.c_int32, fp, vp, fp]
+    lib.kla_chunk_fwd_static_scratch.restype = ctypes.c_int
+    lib.kla_chunk_fwd_static_scratch.argtypes = lib.kla_chunk_fwd.argtypes
     lib.kla_decode_step.restype = ctypes.c_int
     lib.kla_decode_step.argtypes = [dp, vp, vp, vp, fp, fp, ctypes.c_float, fp, vp]
     lib.kla_decode_steps.restype = ctypes.c_int
@@ -152,6 +154,34 @@ def kla_chunk_fwd(q, k, v, log_alpha, eta, eps, chunk=64, init_state=None, out=N
                                  _dev(log_alpha, "log_alpha", torch.float32), _dev(eta, "eta", torch.float32),
                                  float(eps), int(chunk), _dev(init_state, "init_state", torch.float32),
                                  _dev(out, "out"), _dev(final_state, "final_state", torch.float32))
+    _check(code)
+    return out, final_state
+
+
+STATIC_SCRATCH_BYTES = 32 << 20
+
+
+def kla_chunk_fwd_static_scratch(q, k, v, log_alpha, eta, eps, out, final_state=None, chunk=64, init_state=None,
+                                 flags=KLA_FLAG_NONE):
+    """Chunk forward for callers that cannot allocate device memory (include/kla.h:
+    kla_chunk_fwd_static_scratch).  The scratch of the segment-parallel scan is a fixed array inside the library,
+    so this wrapper allocates nothing either: `out` (and `final_state`, if wanted) must be passed in.  Shapes whose
+    scratch would exceed STATIC_SCRATCH_BYTES raise KlaError (workspace).  Calls must not overlap on the GPU."""
+    lib = load()
+    B, T, H, d_k = q.shape
+    d_v = v.shape[-1]
+    if tuple(k.shape) != (B, T, H, d_k) or tuple(v.shape) != (B, T, H, d_v) or tuple(out.shape) != (B, T, H, d_v):
+        raise ValueError("q, k, v, out shapes disagree")
+    if tuple(log_alpha.shape) != (B, T, H) or tuple(eta.shape) != (B, T, H):
+        raise ValueError("log_alpha, eta must be [B, T, H]")
+    desc = KlaDesc(B=B, T=T, H=H, d_k=d_k, d_v=d_v, n_seq=B, cu_seqlens=None, host_seqlens=None,
+                   io_dtype=_dt(q), out_dtype=_dt(out), flags=flags, workspace=None, workspace_bytes=0,
+                   status_word=None, stream=_stream(q.device))
+    with torch.cuda.device(q.device):
+        code = lib.kla_chunk_fwd_static_scratch(
+            ctypes.byref(desc), _dev(q, "q"), _dev(k, "k"), _dev(v, "v"), _dev(log_alpha, "log_alpha", torch.float32),
+            _dev(eta, "eta", torch.float32), float(eps), int(chunk), _dev(init_state, "init_state", torch.float32),
+            _dev(out, "out"), _dev(final_state, "final_state", torch.float32))
     _check(code)
     return out, final_state
 

@@ -347,6 +347,16 @@ def run_ours(args):
     roofline["traffic"] = CHUNK_TC_DRAM_BYTES_PER_LAUNCH
 
     extras = {}
+    if args.quick and args.also:
+        # profiling mode: one extra leg, small launch counts (the ncu captures under profiles/ use these)
+        if args.also == "decode":
+            extras["decode_l2_defeating_B512"] = decode_leg(dev, 4, 2, 1, peaks, B=512)
+        elif args.also == "decode64":
+            extras["decode_cfg4"] = decode_leg(dev, 8, 2, 1, peaks)
+        elif args.also == "long":
+            extras["chunk_cfg3_long_context"] = chunk_leg(W.config3(), dev, 2, 1, peaks, torch.bfloat16)
+        elif args.also == "varlen":
+            extras["chunk_cfg5_varlen"] = chunk_leg(W.config5(), dev, 2, 1, peaks, torch.bfloat16)
     if not args.quick:
         extras["decode_cfg4"] = decode_leg(dev, 256, 4, 2, peaks)
         extras["decode_l2_defeating_B512"] = decode_leg(dev, 32, 4, 2, peaks, B=512)
@@ -382,6 +392,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--quick", action="store_true", help="profiling mode: headline kernel only (no e2e, decode, long-context, varlen or CPU legs)")
+    ap.add_argument("--also", default="", choices=["", "decode", "decode64", "long", "varlen"],
+                    help="with --quick: run one more leg after the headline kernel (used for profiling)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":

@@ -231,6 +231,7 @@ kla_status kla_decode_steps(const kla_desc *desc, int32_t n_steps, const void *q
         p.out = (char *)out + (size_t)s * bh * desc->d_v * out_sz;
         p.BH = (int32_t)bh;
         p.eps = eps;
+        p.inputs_ready = s > 0 ? 1 : 0;
         if (launch_decode(p, desc->d_k, desc->io_dtype, desc->out_dtype, (cudaStream_t)desc->stream) != cudaSuccess)
             return KLA_ERR_LAUNCH;
     }

@@ -37,6 +37,9 @@ struct DecodeParams {
     void *out;
     int32_t BH;
     float eps;
+    // 1: q, k, v, log_alpha, eta were complete before the previous kernel on the stream started (later steps of
+    // kla_decode_steps), so they may be read while that kernel drains; 0: they may be its outputs
+    int32_t inputs_ready;
 };
 
 // Launchers implemented in the kernel translation units.  Each returns cudaGetLastError().

@@ -30,13 +30,10 @@ __global__ void __launch_bounds__(128) kla_decode_kernel(DecodeParams p)
     __shared__ float red_a[4][W], red_c[4][W];
     __shared__ float red_s[2][4];
 
-    // 1. issue the state loads first: they are the long-latency part
-    float *Sp = p.state + (size_t)bh * D * D + sl * W + cg * 4;
-    float4 s[NP];
-#pragma unroll
-    for (int i = 0; i < NP; ++i) s[i] = *reinterpret_cast<const float4 *>(Sp + (size_t)(rg + i * RPP) * D);
-
-    // 2. token vectors
+    // 1. token vectors and their reductions.  The kernel is launched with programmatic stream serialisation, so
+    //    it may start while the previous kernel on the stream drains.  When the vectors are known to predate that
+    //    kernel (later steps of a multi-step call) they are read right away; otherwise wait first.
+    if (!p.inputs_ready) asm volatile("griddepcontrol.wait;" ::: "memory");
     const IO *qp = reinterpret_cast<const IO *>(p.q) + (size_t)bh * D;
     const IO *kp = reinterpret_cast<const IO *>(p.k) + (size_t)bh * D;
     float kk = 0.f, kq = 0.f;
@@ -47,6 +44,9 @@ __global__ void __launch_bounds__(128) kla_decode_kernel(DecodeParams p)
         kk = kv * kv;
         kq = kv * qv;
     }
+    const float alpha = expf(p.log_alpha[bh]);
+    const float eta = p.eta[bh];
+    const float4 vv = load4(reinterpret_cast<const IO *>(p.v) + (size_t)bh * D + sl * W + cg * 4);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
         kk += __shfl_xor_sync(0xffffffffu, kk, o);
@@ -56,6 +56,15 @@ __global__ void __launch_bounds__(128) kla_decode_kernel(DecodeParams p)
         red_s[0][warp] = kk;
         red_s[1][warp] = kq;
     }
+
+    // 2. the state: written by the previous step, so wait for that kernel (a no-op for an ordinary launch), then
+    //    let the next step's kernel start its own prologue
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    float *Sp = p.state + (size_t)bh * D * D + sl * W + cg * 4;
+    float4 s[NP];
+#pragma unroll
+    for (int i = 0; i < NP; ++i) s[i] = *reinterpret_cast<const float4 *>(Sp + (size_t)(rg + i * RPP) * D);
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     __syncthreads();
     kk = red_s[0][0] + red_s[0][1] + red_s[0][2] + red_s[0][3];
     kq = red_s[1][0] + red_s[1][1] + red_s[1][2] + red_s[1][3];
@@ -93,9 +102,7 @@ __global__ void __launch_bounds__(128) kla_decode_kernel(DecodeParams p)
     }
 
     // 4. residual, coefficient, write-back, read-out
-    const float alpha = expf(p.log_alpha[bh]);
-    const float beta = p.eta[bh] / (kk + p.eps);
-    const float4 vv = load4(reinterpret_cast<const IO *>(p.v) + (size_t)bh * D + sl * W + cg * 4);
+    const float beta = eta / (kk + p.eps);
     float4 e = make_float4(vv.x - alpha * a.x, vv.y - alpha * a.y, vv.z - alpha * a.z, vv.w - alpha * a.w);
 #pragma unroll
     for (int i = 0; i < NP; ++i) {
@@ -117,9 +124,21 @@ template <int D, typename IO, typename OUT>
 static cudaError_t launch_decode_t(const DecodeParams &p, cudaStream_t stream)
 {
     constexpr int W = 32;
-    kla_decode_kernel<D, W, IO, OUT><<<p.BH * (D / W), 128, 0, stream>>>(p);
+    // programmatic dependent launch: the kernel's prologue may start while the previous kernel on the stream
+    // drains; its state accesses come after griddepcontrol.wait
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(p.BH * (D / W)));
+    cfg.blockDim = dim3(128);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const cudaError_t err = cudaLaunchKernelEx(&cfg, kla_decode_kernel<D, W, IO, OUT>, p);
     count_launch(1);
-    return cudaGetLastError();
+    return err != cudaSuccess ? err : cudaGetLastError();
 }
 
 cudaError_t launch_decode(const DecodeParams &p, int d, int io_dtype, int out_dtype, cudaStream_t stream)

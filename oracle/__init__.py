@@ -33,6 +33,8 @@ def _load():
                                            dp, dp, dp, dp, dp, ctypes.c_double, dp, dp, dp]
         lib.kla_oracle_decode_step.restype = ctypes.c_int
         lib.kla_oracle_decode_step.argtypes = [ctypes.c_int] * 4 + [dp] * 5 + [ctypes.c_double, dp, dp]
+        lib.kla_oracle_set_variant.restype = None
+        lib.kla_oracle_set_variant.argtypes = [ctypes.c_int, ctypes.c_int]
         lib.kla_oracle_set_threads.restype = None
         lib.kla_oracle_set_threads.argtypes = [ctypes.c_int]
         _lib = lib
@@ -45,6 +47,22 @@ def _f64(a):
 
 def _ptr(a):
     return a.ctypes.data_as(ctypes.POINTER(ctypes.c_double)) if a is not None else None
+
+
+class variant:
+    """Context manager selecting the layer-edge variants for the calls inside it:
+    `coeff_eta` -- beta_t = eta_t (the gated-delta-rule baseline coefficient, Section 2) instead of Eq. 3;
+    `qnorm`     -- read-out divided by ||q_t||, as Algorithm 1 (left) prints it.  Default: neither."""
+
+    def __init__(self, coeff_eta=False, qnorm=False):
+        self.args = (int(bool(coeff_eta)), int(bool(qnorm)))
+
+    def __enter__(self):
+        _load().kla_oracle_set_variant(*self.args)
+        return self
+
+    def __exit__(self, *a):
+        _load().kla_oracle_set_variant(0, 0)
 
 
 def set_threads(n: int) -> None:

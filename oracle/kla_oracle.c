@@ -35,6 +35,17 @@
 #endif
 
 /* One token of one head; S is updated in place, o receives d_v values. */
+/* The two layer-edge variants the paper names, selected per call (0 = the default above):
+ *   coeff_eta  beta_t = eta_t, the gated-delta-rule baseline coefficient without the key-norm division
+ *              (Section 2; the comparison model of Section 5);
+ *   qnorm      o_t = S_t^T q_t / ||q_t||, the read-out exactly as Algorithm 1 (left) prints it. */
+static int g_coeff_eta = 0, g_qnorm = 0;
+void kla_oracle_set_variant(int coeff_eta, int qnorm)
+{
+    g_coeff_eta = coeff_eta;
+    g_qnorm = qnorm;
+}
+
 static void kla_token_update(double *S, int d_k, int d_v, const double *q, const double *k,
                              const double *v, double log_alpha, double eta, double eps,
                              double *e /* scratch d_v */, double *o)
@@ -50,7 +61,7 @@ static void kla_token_update(double *S, int d_k, int d_v, const double *q, const
     /* Kaczmarz coefficient, Eq. 3 */
     double nk = 0.0;
     for (int i = 0; i < d_k; ++i) nk += k[i] * k[i];
-    const double beta = eta / (nk + eps);
+    const double beta = g_coeff_eta ? eta : eta / (nk + eps);
     /* rank-one write */
     for (int i = 0; i < d_k; ++i) {
         const double bk = beta * k[i];
@@ -60,6 +71,12 @@ static void kla_token_update(double *S, int d_k, int d_v, const double *q, const
     for (int j = 0; j < d_v; ++j) o[j] = 0.0;
     for (int i = 0; i < d_k; ++i)
         for (int j = 0; j < d_v; ++j) o[j] += S[(size_t)i * d_v + j] * q[i];
+    if (g_qnorm) {
+        double nq = 0.0;
+        for (int i = 0; i < d_k; ++i) nq += q[i] * q[i];
+        const double inv = 1.0 / sqrt(nq);
+        for (int j = 0; j < d_v; ++j) o[j] *= inv;
+    }
 }
 
 /*

@@ -234,3 +234,63 @@ def test_zero_key_with_eps_is_pure_decay_and_zero_eps_is_nan():
     np.testing.assert_allclose(fin, 0.25 * s0, atol=1e-15)
     out, fin, _ = oracle.forward(q, k, v, la, eta, 0.0, s0)
     assert np.isnan(fin).all()
+
+
+# ---- layer-edge variants: beta = eta (the gated-delta-rule baseline coefficient) and the ||q||-normalised read-out
+def test_variant_coeff_eta_is_the_unrolled_product_with_beta_equal_eta():
+    """Table 7 form again, with the write coefficient beta_j = eta_j (Section 2's gated delta rule): the same
+    explicit matrix products as the Kaczmarz pin, only the coefficient differs."""
+    rng = RNG(17)
+    T, d_k, d_v = 7, 4, 3
+    q, k, v, la, eta, s0 = _rand_problem(rng, B=1, T=T, H=1, d_k=d_k, d_v=d_v)
+    k = 0.5 * k                                   # keep I - eta k k^T well conditioned
+    with oracle.variant(coeff_eta=True):
+        out, fin, _ = oracle.forward(q, k, v, la, eta, 0.01, s0)
+    kk, qq, vv = k[0, :, 0], q[0, :, 0], v[0, :, 0]
+    beta, alpha = eta[0, :, 0], np.exp(la[0, :, 0])
+    Ms = [alpha[s] * (np.eye(d_k) - beta[s] * np.outer(kk[s], kk[s])) for s in range(T)]
+    for t in range(T):
+        acc = np.zeros(d_v)
+        for j in range(t + 1):
+            P = np.eye(d_k)
+            for s in range(j + 1, t + 1):
+                P = Ms[s] @ P
+            acc += beta[j] * (qq[t] @ P @ kk[j]) * vv[j]
+        P = np.eye(d_k)
+        for s in range(0, t + 1):
+            P = Ms[s] @ P
+        acc += qq[t] @ P @ s0[0, 0]
+        np.testing.assert_allclose(out[0, t, 0], acc, rtol=0, atol=1e-12)
+
+
+def test_variant_coeff_eta_equals_kaczmarz_on_unit_keys():
+    """With ||k_t|| = 1 and eps = 0 Eq. 3 gives beta_t = eta_t: the two coefficients coincide."""
+    rng = RNG(18)
+    q, k, v, la, eta, s0 = _rand_problem(rng, T=15)
+    k = k / np.linalg.norm(k, axis=-1, keepdims=True)
+    ref_o, ref_f, _ = oracle.forward(q, k, v, la, eta, 0.0, s0)
+    with oracle.variant(coeff_eta=True):
+        o, f, _ = oracle.forward(q, k, v, la, eta, 0.0, s0)
+    np.testing.assert_allclose(o, ref_o, rtol=0, atol=1e-12)
+    np.testing.assert_allclose(f, ref_f, rtol=0, atol=1e-12)
+
+
+def test_variant_qnorm_divides_the_readout_only():
+    """o_t = S_t^T q_t / ||q_t|| (Algorithm 1 left): the states are untouched, the output is the default output
+    over ||q_t||, and scaling q_t by any positive factor changes nothing."""
+    rng = RNG(19)
+    q, k, v, la, eta, s0 = _rand_problem(rng, T=11)
+    o0, f0, _ = oracle.forward(q, k, v, la, eta, 1e-3, s0)
+    with oracle.variant(qnorm=True):
+        o1, f1, _ = oracle.forward(q, k, v, la, eta, 1e-3, s0)
+        scale = np.exp(rng.standard_normal(q.shape[:-1]))[..., None]
+        o2, _, _ = oracle.forward(q * scale, k, v, la, eta, 1e-3, s0)
+        st = np.ascontiguousarray(s0.copy())
+        od = oracle.decode_step(q[:, 0], k[:, 0], v[:, 0], la[:, 0], eta[:, 0], 1e-3, st)
+    np.testing.assert_allclose(o1, o0 / np.linalg.norm(q, axis=-1, keepdims=True), rtol=0, atol=1e-12)
+    np.testing.assert_allclose(f1, f0, rtol=0, atol=0)
+    np.testing.assert_allclose(o2, o1, rtol=0, atol=1e-12)
+    np.testing.assert_allclose(od, o1[:, 0], rtol=0, atol=1e-12)
+    # and the default is restored on leaving the context
+    o3, _, _ = oracle.forward(q, k, v, la, eta, 1e-3, s0)
+    np.testing.assert_array_equal(o3, o0)

@@ -63,6 +63,10 @@ typedef enum { KLA_F32 = 0, KLA_BF16 = 1 } kla_dtype;
  * parallel, chained, and the segments then run in parallel from their true start states: the same result up
  * to rounding, about three times the state work, G times the parallelism.  By default the library decides
  * from the shape (few long sequences -> segments) and the workspace query returns what that decision needs. */
+/* Layer-edge variants named by the paper; both default to off (the recurrence at the top of this file). */
+#define KLA_FLAG_COEFF_ETA 4              /* beta_t = eta_t: the gated-delta-rule baseline coefficient of Section 2,
+                                             without the key-norm division of Eq. 3 (eps is then unused)          */
+#define KLA_FLAG_QNORM 8                  /* o_t = S_t^T q_t / ||q_t||: the read-out as Algorithm 1 (left) prints it */
 #define KLA_FLAG_NO_SEGMENTS 2            /* never cut sequences into segments                              */
 #define KLA_FLAG_SEGMENTS(g) ((g) << 8)   /* force g segments per sequence, 2 <= g <= 255 (fewer if T is short) */
 

@@ -14,6 +14,7 @@ LIB_PATH = os.path.join(_HERE, "libkla_b200.so")
 
 KLA_F32, KLA_BF16 = 0, 1
 KLA_FLAG_NONE, KLA_FLAG_FORCE_SIMT, KLA_FLAG_NO_SEGMENTS = 0, 1, 2
+KLA_FLAG_COEFF_ETA, KLA_FLAG_QNORM = 4, 8
 
 
 def KLA_FLAG_SEGMENTS(g: int) -> int:
@@ -186,13 +187,13 @@ def kla_chunk_fwd_static_scratch(q, k, v, log_alpha, eta, eps, out, final_state=
     return out, final_state
 
 
-def _decode_desc(q, v, out, B, H, d_k, d_v):
+def _decode_desc(q, v, out, B, H, d_k, d_v, flags=0):
     return KlaDesc(B=B, T=1, H=H, d_k=d_k, d_v=d_v, n_seq=B, cu_seqlens=None, host_seqlens=None,
-                   io_dtype=_dt(q), out_dtype=_dt(out), flags=0, workspace=None, workspace_bytes=0,
+                   io_dtype=_dt(q), out_dtype=_dt(out), flags=flags, workspace=None, workspace_bytes=0,
                    status_word=None, stream=_stream(q.device))
 
 
-def kla_decode_step(q, k, v, log_alpha, eta, eps, state_inout, out=None, out_dtype=None):
+def kla_decode_step(q, k, v, log_alpha, eta, eps, state_inout, out=None, out_dtype=None, flags=KLA_FLAG_NONE):
     """One decode step (include/kla.h: kla_decode_step).  q, k [B, H, d_k]; v [B, H, d_v];
     log_alpha, eta [B, H] fp32; state_inout [B, H, d_k, d_v] fp32, updated in place."""
     lib = load()
@@ -200,7 +201,7 @@ def kla_decode_step(q, k, v, log_alpha, eta, eps, state_inout, out=None, out_dty
     d_v = v.shape[-1]
     if out is None:
         out = torch.empty((B, H, d_v), device=q.device, dtype=out_dtype or q.dtype)
-    desc = _decode_desc(q, v, out, B, H, d_k, d_v)
+    desc = _decode_desc(q, v, out, B, H, d_k, d_v, flags)
     with torch.cuda.device(q.device):
         code = lib.kla_decode_step(ctypes.byref(desc), _dev(q, "q"), _dev(k, "k"), _dev(v, "v"),
                                    _dev(log_alpha, "log_alpha", torch.float32), _dev(eta, "eta", torch.float32),
@@ -209,7 +210,7 @@ def kla_decode_step(q, k, v, log_alpha, eta, eps, state_inout, out=None, out_dty
     return out
 
 
-def kla_decode_steps(q, k, v, log_alpha, eta, eps, state_inout, out=None, out_dtype=None):
+def kla_decode_steps(q, k, v, log_alpha, eta, eps, state_inout, out=None, out_dtype=None, flags=KLA_FLAG_NONE):
     """n consecutive decode steps (include/kla.h: kla_decode_steps).  q, k [n, B, H, d_k];
     v [n, B, H, d_v]; log_alpha, eta [n, B, H]; state carried in place; out [n, B, H, d_v]."""
     lib = load()
@@ -217,7 +218,7 @@ def kla_decode_steps(q, k, v, log_alpha, eta, eps, state_inout, out=None, out_dt
     d_v = v.shape[-1]
     if out is None:
         out = torch.empty((n, B, H, d_v), device=q.device, dtype=out_dtype or q.dtype)
-    desc = _decode_desc(q, v, out, B, H, d_k, d_v)
+    desc = _decode_desc(q, v, out, B, H, d_k, d_v, flags)
     with torch.cuda.device(q.device):
         code = lib.kla_decode_steps(ctypes.byref(desc), n, _dev(q, "q"), _dev(k, "k"), _dev(v, "v"),
                                     _dev(log_alpha, "log_alpha", torch.float32), _dev(eta, "eta", torch.float32),

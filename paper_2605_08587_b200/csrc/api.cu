@@ -151,6 +151,7 @@ kla_status kla_chunk_fwd(const kla_desc *desc, const void *q, const void *k, con
     p.status_word = desc->status_word;
     p.trace = nullptr;
     p.seg_pass = 0; p.seg_G = 0; p.map_state = nullptr;
+    p.variant = ((desc->flags & KLA_FLAG_COEFF_ETA) ? VARIANT_COEFF_ETA : 0) | ((desc->flags & KLA_FLAG_QNORM) ? VARIANT_QNORM : 0);
     p.B = desc->B; p.T = desc->T; p.H = desc->H; p.n_seq = desc->n_seq;
     p.eps = eps;
     if (desc->T == 0) {
@@ -232,6 +233,8 @@ kla_status kla_decode_steps(const kla_desc *desc, int32_t n_steps, const void *q
         p.BH = (int32_t)bh;
         p.eps = eps;
         p.inputs_ready = s > 0 ? 1 : 0;
+        p.coeff_eta = (desc->flags & KLA_FLAG_COEFF_ETA) ? 1 : 0;
+        p.qnorm = (desc->flags & KLA_FLAG_QNORM) ? 1 : 0;
         if (launch_decode(p, desc->d_k, desc->io_dtype, desc->out_dtype, (cudaStream_t)desc->stream) != cudaSuccess)
             return KLA_ERR_LAUNCH;
     }

@@ -40,6 +40,7 @@ struct SimtSmem {
     double g[C];       // chunk-local running sum of log alpha; kept in fp64 so that the
                        // differences g_i - g_j below do not cancel away fp32 digits
     float beta[C], la[C], eta[C];
+    float qn[C];       // 1 / ||q_i|| when the normalised read-out is asked for, else 1
 };
 
 template <typename IO>
@@ -169,11 +170,21 @@ __global__ void __launch_bounds__(NTHREADS) kla_chunk_simt_kernel(ChunkParams p)
 
         // ---- prologue: beta and chunk-local cumulative log decay -----------------------------
         for (int r = warp; r < C; r += NTHREADS / 32) {
-            float s = 0.f;
-            for (int d = lane; d < D; d += 32) s += sm.K[r][d] * sm.K[r][d];
+            float s = 0.f, sq = 0.f;
+            for (int d = lane; d < D; d += 32) {
+                s += sm.K[r][d] * sm.K[r][d];
+                sq += sm.Q[r][d] * sm.Q[r][d];
+            }
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-            if (lane == 0) sm.beta[r] = (r < rows) ? sm.eta[r] / (s + p.eps) : 0.f;
+            for (int o = 16; o > 0; o >>= 1) {
+                s += __shfl_xor_sync(0xffffffffu, s, o);
+                sq += __shfl_xor_sync(0xffffffffu, sq, o);
+            }
+            if (lane == 0) {
+                // Eq. 3, or beta = eta (the gated-delta-rule coefficient) when asked for
+                sm.beta[r] = (r < rows) ? ((p.variant & VARIANT_COEFF_ETA) ? sm.eta[r] : sm.eta[r] / (s + p.eps)) : 0.f;
+                sm.qn[r] = (p.variant & VARIANT_QNORM) ? 1.f / sqrtf(sq) : 1.f;
+            }
         }
         if (warp == 0) {
             // inclusive scan of C values, C/32 (or fewer) per lane
@@ -322,9 +333,10 @@ __global__ void __launch_bounds__(NTHREADS) kla_chunk_simt_kernel(ChunkParams p)
 #pragma unroll
                 for (int a = 0; a < ROe; ++a) {
                     const int i = ROe * tr + a;
+                    const float rn = sm.qn[i];
                     if (i < rows)
                         store4(og + (size_t)(tok0 + c0 + i) * HD + (size_t)h * D + sl * NS + 4 * tc,
-                               make_float4(acc[a][0], acc[a][1], acc[a][2], acc[a][3]));
+                               make_float4(rn * acc[a][0], rn * acc[a][1], rn * acc[a][2], rn * acc[a][3]));
                 }
             } else {
                 // C = 16: 128 threads, one row x 4 columns each
@@ -337,9 +349,10 @@ __global__ void __launch_bounds__(NTHREADS) kla_chunk_simt_kernel(ChunkParams p)
                         const float pij = sm.P[i][j];
                         a0 += pij * u.x; a1 += pij * u.y; a2 += pij * u.z; a3 += pij * u.w;
                     }
+                    const float rn = sm.qn[i];
                     if (i < rows)
                         store4(og + (size_t)(tok0 + c0 + i) * HD + (size_t)h * D + sl * NS + 4 * tc,
-                               make_float4(a0, a1, a2, a3));
+                               make_float4(rn * a0, rn * a1, rn * a2, rn * a3));
                 }
             }
         }

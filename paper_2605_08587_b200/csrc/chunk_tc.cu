@@ -111,6 +111,7 @@ struct TcSmem {
     alignas(8) uint64_t bar[B_COUNT];
     uint32_t tmem_base;
     volatile int abort_flag;
+    float qn[NSTAGE][64];                       // 1 / ||q_i|| (written only when the normalised read-out is asked for)
 };
 
 // Bounded wait on an mbarrier phase that also leaves when another role has aborted.  Every lane of the
@@ -223,7 +224,9 @@ __device__ __forceinline__ void merge_level(float *tl, float *mm, const float *b
     pg_sync();
 }
 
-template <int D, typename OUT>
+// VAR: compiled with the layer-edge variants (beta = eta, read-out over ||q||); the default instantiation carries
+// none of their code.
+template <int D, typename OUT, bool VAR>
 __global__ void __launch_bounds__(NT, 1)
 kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                     const __grid_constant__ CUtensorMap tm_v, ChunkParams p)
@@ -501,6 +504,22 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 *reinterpret_cast<uint4 *>(sm.p_hi + sw128(i, chh * 4 + grp)) = hi;
                 *reinterpret_cast<uint4 *>(sm.p_lo + sw128(i, chh * 4 + grp)) = lo;
             }
+            if constexpr (VAR) if ((p.variant & VARIANT_QNORM) && chh == 0) {
+                // ||q_i||^2 from row i of the Q tile (still resident: its stage is refilled only after MMA-4(c))
+                const unsigned char *qt = sm.kq[sc];
+                float n = 0.f;
+#pragma unroll 1
+                for (int e = 0; e < KB * 8; ++e) {
+                    const uint4 raw = *reinterpret_cast<const uint4 *>(qt + (e >> 3) * 16384 + 8192 + sw128(i, e & 7));
+                    const __nv_bfloat162 *h2 = reinterpret_cast<const __nv_bfloat162 *>(&raw);
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const float2 f = __bfloat1622float2(h2[u]);
+                        n += f.x * f.x + f.y * f.y;
+                    }
+                }
+                sm.qn[sc][i] = 1.f / sqrtf(n);
+            }
             tc_fence_before();
             fence_async_smem();
             warp_arrive(B_D1_FREE0 + (c & 1));
@@ -580,7 +599,10 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                             *reinterpret_cast<float4 *>(&sm.tl[i * LDT + j0 + 4]) = make_float4(x[4], x[5], x[6], x[7]);
                         }
                         // beta_i = eta_i / (||k_i||^2 + eps), Eq. 3; rows past the end of the sequence get 0
-                        if (chh == q) sm.beta[sc][i] = (i < rows) ? eta_cur / (dg + p.eps) : 0.f;
+                        if (chh == q) {
+                            if constexpr (VAR) sm.beta[sc][i] = (i < rows) ? ((p.variant & VARIANT_COEFF_ETA) ? eta_cur : eta_cur / (dg + p.eps)) : 0.f;
+                            else sm.beta[sc][i] = (i < rows) ? eta_cur / (dg + p.eps) : 0.f;
+                        }
                     }
                     KLA_TR(1, c, 11);
                     tc_fence_before();
@@ -794,8 +816,15 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     float acc[4], qs[4];
                     tmem_ld16x256b_x1(tm16 + TM_PU + 8 * j, acc);
                     tmem_ld16x256b_x1(tq + 8 * j, qs);
-                    if (i0 < rows) store2(o0 + 8 * j, g0 * qs[0] + acc[0], g0 * qs[1] + acc[1]);
-                    if (i1 < rows) store2(o1 + 8 * j, g1 * qs[2] + acc[2], g1 * qs[3] + acc[3]);
+                    if constexpr (VAR) {
+                        // read-out over ||q|| when asked for
+                        const float n0 = (p.variant & VARIANT_QNORM) ? sm.qn[sc][i0] : 1.f, n1 = (p.variant & VARIANT_QNORM) ? sm.qn[sc][i1] : 1.f;
+                        if (i0 < rows) store2(o0 + 8 * j, n0 * (g0 * qs[0] + acc[0]), n0 * (g0 * qs[1] + acc[1]));
+                        if (i1 < rows) store2(o1 + 8 * j, n1 * (g1 * qs[2] + acc[2]), n1 * (g1 * qs[3] + acc[3]));
+                    } else {
+                        if (i0 < rows) store2(o0 + 8 * j, g0 * qs[0] + acc[0], g0 * qs[1] + acc[1]);
+                        if (i1 < rows) store2(o1 + 8 * j, g1 * qs[2] + acc[2], g1 * qs[3] + acc[3]);
+                    }
                 }
             }
             tc_fence_before();
@@ -851,8 +880,17 @@ bool make_tmap(CUtensorMap *tm, const void *base, uint64_t n_tok, uint64_t row_e
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+template <int D, typename OUT, bool VAR>
+cudaError_t launch_v(const ChunkParams &p, cudaStream_t stream);
+
 template <int D, typename OUT>
 cudaError_t launch_t(const ChunkParams &p, cudaStream_t stream)
+{
+    return (p.variant != 0) ? launch_v<D, OUT, true>(p, stream) : launch_v<D, OUT, false>(p, stream);
+}
+
+template <int D, typename OUT, bool VAR>
+cudaError_t launch_v(const ChunkParams &p, cudaStream_t stream)
 {
     using Smem = TcSmem<D>;
     const uint64_t n_tok = (uint64_t)p.B * p.T;
@@ -860,7 +898,7 @@ cudaError_t launch_t(const ChunkParams &p, cudaStream_t stream)
     if (!make_tmap(&tq, p.q, n_tok, (uint64_t)p.H * D) || !make_tmap(&tk, p.k, n_tok, (uint64_t)p.H * D) ||
         !make_tmap(&tv, p.v, n_tok, (uint64_t)p.H * D))
         return cudaErrorInvalidValue;
-    auto kern = kla_chunk_tc_kernel<D, OUT>;
+    auto kern = kla_chunk_tc_kernel<D, OUT, VAR>;
     const int smem = (int)sizeof(Smem) + 1024;
     cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (err != cudaSuccess) return err;

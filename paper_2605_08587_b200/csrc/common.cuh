@@ -27,8 +27,10 @@ struct ChunkParams {
     //   seg_pass 3: every segment from its true start state; only the last segment of a sequence writes
     //               final_state, at the sequence's index.
     int32_t seg_pass, seg_G;
+    int32_t variant;     // bit 0: beta_t = eta_t instead of Eq. 3; bit 1: read-out divided by ||q_t||
     float *map_state;
 };
+constexpr int32_t VARIANT_COEFF_ETA = 1, VARIANT_QNORM = 2;
 
 struct DecodeParams {
     const void *q, *k, *v;
@@ -40,6 +42,7 @@ struct DecodeParams {
     // 1: q, k, v, log_alpha, eta were complete before the previous kernel on the stream started (later steps of
     // kla_decode_steps), so they may be read while that kernel drains; 0: they may be its outputs
     int32_t inputs_ready;
+    int32_t coeff_eta, qnorm;   // as in ChunkParams
 };
 
 // Launchers implemented in the kernel translation units.  Each returns cudaGetLastError().

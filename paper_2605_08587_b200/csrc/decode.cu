@@ -28,7 +28,7 @@ __global__ void __launch_bounds__(128) kla_decode_kernel(DecodeParams p)
 
     __shared__ float sk[D], sq[D];
     __shared__ float red_a[4][W], red_c[4][W];
-    __shared__ float red_s[2][4];
+    __shared__ float red_s[3][4];
 
     // 1. token vectors and their reductions.  The kernel is launched with programmatic stream serialisation, so
     //    it may start while the previous kernel on the stream drains.  When the vectors are known to predate that
@@ -36,13 +36,14 @@ __global__ void __launch_bounds__(128) kla_decode_kernel(DecodeParams p)
     if (!p.inputs_ready) asm volatile("griddepcontrol.wait;" ::: "memory");
     const IO *qp = reinterpret_cast<const IO *>(p.q) + (size_t)bh * D;
     const IO *kp = reinterpret_cast<const IO *>(p.k) + (size_t)bh * D;
-    float kk = 0.f, kq = 0.f;
+    float kk = 0.f, kq = 0.f, qq = 0.f;
     if (tid < D) {
         float kv = to_f32(kp[tid]), qv = to_f32(qp[tid]);
         sk[tid] = kv;
         sq[tid] = qv;
         kk = kv * kv;
         kq = kv * qv;
+        qq = qv * qv;
     }
     const float alpha = expf(p.log_alpha[bh]);
     const float eta = p.eta[bh];
@@ -51,10 +52,12 @@ __global__ void __launch_bounds__(128) kla_decode_kernel(DecodeParams p)
     for (int o = 16; o > 0; o >>= 1) {
         kk += __shfl_xor_sync(0xffffffffu, kk, o);
         kq += __shfl_xor_sync(0xffffffffu, kq, o);
+        qq += __shfl_xor_sync(0xffffffffu, qq, o);
     }
     if (lane == 0) {
         red_s[0][warp] = kk;
         red_s[1][warp] = kq;
+        red_s[2][warp] = qq;
     }
 
     // 2. the state: written by the previous step, so wait for that kernel (a no-op for an ordinary launch), then
@@ -68,6 +71,7 @@ __global__ void __launch_bounds__(128) kla_decode_kernel(DecodeParams p)
     __syncthreads();
     kk = red_s[0][0] + red_s[0][1] + red_s[0][2] + red_s[0][3];
     kq = red_s[1][0] + red_s[1][1] + red_s[1][2] + red_s[1][3];
+    qq = red_s[2][0] + red_s[2][1] + red_s[2][2] + red_s[2][3];
 
     // 3. a = S^T k and c = S^T q for this thread's 4 columns over its rows
     float4 a = make_float4(0.f, 0.f, 0.f, 0.f), c = a;
@@ -102,7 +106,7 @@ __global__ void __launch_bounds__(128) kla_decode_kernel(DecodeParams p)
     }
 
     // 4. residual, coefficient, write-back, read-out
-    const float beta = eta / (kk + p.eps);
+    const float beta = p.coeff_eta ? eta : eta / (kk + p.eps);   // Eq. 3, or the gated-delta-rule coefficient
     float4 e = make_float4(vv.x - alpha * a.x, vv.y - alpha * a.y, vv.z - alpha * a.z, vv.w - alpha * a.w);
 #pragma unroll
     for (int i = 0; i < NP; ++i) {
@@ -114,8 +118,9 @@ __global__ void __launch_bounds__(128) kla_decode_kernel(DecodeParams p)
     }
     if (rg == 0) {
         const float bq = beta * kq;
-        float4 o = make_float4(alpha * c.x + bq * e.x, alpha * c.y + bq * e.y, alpha * c.z + bq * e.z,
-                               alpha * c.w + bq * e.w);
+        const float rn = p.qnorm ? 1.f / sqrtf(qq) : 1.f;   // read-out over ||q|| (Algorithm 1 left) when asked for
+        float4 o = make_float4(rn * (alpha * c.x + bq * e.x), rn * (alpha * c.y + bq * e.y), rn * (alpha * c.z + bq * e.z),
+                               rn * (alpha * c.w + bq * e.w));
         store4(reinterpret_cast<OUT *>(p.out) + (size_t)bh * D + sl * W + cg * 4, o);
     }
 }

@@ -87,3 +87,22 @@ def test_config4_full_size_sampled():
     assert max(per_step) <= TOL_BF16
     assert rel_err(np64(st[bsel][:, hsel]), rs) <= TOL_BF16
     assert torch.isfinite(out).all() and torch.isfinite(st).all()
+
+
+@pytest.mark.parametrize("variant", [(True, False), (False, True), (True, True)])
+def test_decode_variants(variant):
+    """beta = eta (gated-delta-rule coefficient) and the read-out over ||q||, against the oracle's variants."""
+    from paper_2605_08587_b200 import KLA_FLAG_COEFF_ETA, KLA_FLAG_QNORM
+    coeff_eta, qnorm = variant
+    w = W.config4(B=4, H=2, d=128, steps=6, seed=40 + 2 * coeff_eta + qnorm)
+    if coeff_eta:
+        k = w.k.float()
+        w.k = (k / k.norm(dim=-1, keepdim=True)).to(w.k.dtype)
+    flags = (KLA_FLAG_COEFF_ETA if coeff_eta else 0) | (KLA_FLAG_QNORM if qnorm else 0)
+    with oracle.variant(coeff_eta=coeff_eta, qnorm=qnorm):
+        ro, rs = _oracle_decode(w)
+    st = w.state.to(DEV).clone()
+    out = kla_decode_steps(w.q.to(DEV), w.k.to(DEV), w.v.to(DEV), w.log_alpha.to(DEV), w.eta.to(DEV), w.eps, st,
+                           out_dtype=torch.float32, flags=flags)
+    assert rel_err(np64(out), ro) <= TOL_BF16
+    assert rel_err(np64(st), rs) <= TOL_BF16

@@ -213,3 +213,46 @@ def test_segments_without_init_state_and_without_final_state():
 def test_more_segments_than_chunks_is_clamped():
     w = W.config3(B=1, H=2, T=130, seed=215)
     _check_fixed(w, TOL_BF16, flags=KLA_FLAG_SEGMENTS(9))
+
+
+# ---- layer-edge variants: beta = eta (gated-delta-rule coefficient) and the read-out over ||q|| -------------------
+import oracle  # noqa: E402
+from paper_2605_08587_b200 import KLA_FLAG_COEFF_ETA, KLA_FLAG_QNORM  # noqa: E402
+
+
+def _unit_keys(w):
+    """beta = eta is only a stable write for keys of about unit norm (the paper's comparison model normalises
+    them): rescale k to ||k|| = 1, rounded to the workload's dtype before either side sees it."""
+    k = w.k.float()
+    w.k = (k / k.norm(dim=-1, keepdim=True).clamp_min(1e-12)).to(w.k.dtype)
+    return w
+
+
+@pytest.mark.parametrize("flags", [0, KLA_FLAG_FORCE_SIMT])
+@pytest.mark.parametrize("variant", [(True, False), (False, True), (True, True)])
+def test_variants_match_oracle(variant, flags):
+    coeff_eta, qnorm = variant
+    w = W.config3(B=2, H=2, T=300, seed=400 + 2 * coeff_eta + qnorm)
+    if coeff_eta:
+        w = _unit_keys(w)
+    vf = (KLA_FLAG_COEFF_ETA if coeff_eta else 0) | (KLA_FLAG_QNORM if qnorm else 0)
+    out, fin = gpu_chunk(w, flags=flags | vf)
+    with oracle.variant(coeff_eta=coeff_eta, qnorm=qnorm):
+        ro, rf = oracle_chunk(w)
+    assert rel_err(np64(out), ro) <= TOL_BF16
+    assert rel_err(np64(fin), rf) <= TOL_BF16
+
+
+def test_variants_fp32_and_segments():
+    w = _unit_keys(W.config1(B=1, H=2, T=200, d=64, seed=410))
+    out, fin = gpu_chunk(w, flags=KLA_FLAG_COEFF_ETA | KLA_FLAG_QNORM)
+    with oracle.variant(coeff_eta=True, qnorm=True):
+        ro, rf = oracle_chunk(w)
+    assert rel_err(np64(out), ro) <= TOL_F32
+    assert rel_err(np64(fin), rf) <= TOL_F32
+    w = _unit_keys(W.config3(B=1, H=2, T=1024, seed=411))
+    out, fin = gpu_chunk(w, flags=KLA_FLAG_COEFF_ETA | KLA_FLAG_QNORM | KLA_FLAG_SEGMENTS(4))
+    with oracle.variant(coeff_eta=True, qnorm=True):
+        ro, rf = oracle_chunk(w)
+    assert rel_err(np64(out), ro) <= TOL_BF16
+    assert rel_err(np64(fin), rf) <= TOL_BF16

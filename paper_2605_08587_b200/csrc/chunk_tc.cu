@@ -637,7 +637,12 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 #pragma unroll
                 for (int r = 0; r < 8; ++r) Lb[r * LDT + j] = x[r];
             }
-            pg_sync();
+            // Meanwhile a warp with nothing to substitute takes the wait that guards the T tiles (MMA-3(c-1) must have
+            // read the previous ones): the first look at a barrier completed by the tensor pipe costs several hundred
+            // cycles wherever it is taken, so it is taken here, under the substitution.
+            bool okd = true;
+            if (c > 0 && pt >= PG_T - 32) okd = wait(B_D3_DONE, ph ^ 1);
+            if (pg_any(!okd)) break;
             KLA_TR(1, c, 2);
             merge_level<8>(sm.tl, sm.mm, bet, pt);
             KLA_TR(1, c, 6);
@@ -646,7 +651,6 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             merge_level<32>(sm.tl, sm.mm, bet, pt);
             // ---- write T as bf16 hi/lo operand tiles, after MMA-3(c-1) has read the previous ones ----------------------
             KLA_TR(1, c, 3);
-            if (c > 0 && pg_any(!wait(B_D3_DONE, ph ^ 1))) break;
             KLA_TR(1, c, 4);
             {
                 const int r = pt & 63, qq = pt >> 6;  // row, 16-column quarter

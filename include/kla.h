@@ -67,6 +67,10 @@ typedef enum { KLA_F32 = 0, KLA_BF16 = 1 } kla_dtype;
 #define KLA_FLAG_COEFF_ETA 4              /* beta_t = eta_t: the gated-delta-rule baseline coefficient of Section 2,
                                              without the key-norm division of Eq. 3 (eps is then unused)          */
 #define KLA_FLAG_QNORM 8                  /* o_t = S_t^T q_t / ||q_t||: the read-out as Algorithm 1 (left) prints it */
+/* Test hook for the error path: the tensor-core kernel withholds one internal completion signal, so that a
+ * bounded device-side wait runs out (about one second), every CTA gives up in an orderly way and KLA_ERR_TIMEOUT
+ * appears in *status_word.  Outputs are then undefined; the context stays usable. */
+#define KLA_FLAG_TEST_TIMEOUT 16
 #define KLA_FLAG_NO_SEGMENTS 2            /* never cut sequences into segments                              */
 #define KLA_FLAG_SEGMENTS(g) ((g) << 8)   /* force g segments per sequence, 2 <= g <= 255 (fewer if T is short) */
 

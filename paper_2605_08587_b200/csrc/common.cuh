@@ -27,10 +27,10 @@ struct ChunkParams {
     //   seg_pass 3: every segment from its true start state; only the last segment of a sequence writes
     //               final_state, at the sequence's index.
     int32_t seg_pass, seg_G;
-    int32_t variant;     // bit 0: beta_t = eta_t instead of Eq. 3; bit 1: read-out divided by ||q_t||
+    int32_t variant;     // bit 0: beta_t = eta_t instead of Eq. 3; bit 1: read-out divided by ||q_t||; bit 2: test hook
     float *map_state;
 };
-constexpr int32_t VARIANT_COEFF_ETA = 1, VARIANT_QNORM = 2;
+constexpr int32_t VARIANT_COEFF_ETA = 1, VARIANT_QNORM = 2, VARIANT_TEST_TIMEOUT = 4;
 
 struct DecodeParams {
     const void *q, *k, *v;

@@ -256,3 +256,23 @@ def test_variants_fp32_and_segments():
         ro, rf = oracle_chunk(w)
     assert rel_err(np64(out), ro) <= TOL_BF16
     assert rel_err(np64(fin), rf) <= TOL_BF16
+
+
+# ---- the bounded-wait error path (no fault, no hang: a wait runs out by design and the kernel reports it) -------------
+def test_bounded_wait_reports_timeout_and_context_stays_usable():
+    from paper_2605_08587_b200 import binding
+    w = W.config2(B=1, H=1, T=64, seed=501)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda:0")
+    dev = "cuda:0"
+    a = [t.to(dev) for t in (w.q, w.k, w.v, w.log_alpha, w.eta)]
+    from paper_2605_08587_b200 import kla_chunk_fwd
+    kla_chunk_fwd(*a, w.eps, flags=binding.KLA_FLAG_TEST_TIMEOUT, status_word=status)
+    torch.cuda.synchronize()                      # returns after about a second: the wait is bounded
+    assert int(status.item()) == -10              # KLA_ERR_TIMEOUT
+    # the same context then runs the normal path correctly, and an untouched status word stays zero
+    status.zero_()
+    out, fin = kla_chunk_fwd(*a, w.eps, out_dtype=torch.float32, status_word=status)
+    torch.cuda.synchronize()
+    ro, rf = oracle_chunk(w)
+    assert int(status.item()) == 0
+    assert rel_err(np64(out), ro) <= TOL_BF16 and rel_err(np64(fin), rf) <= TOL_BF16

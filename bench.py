@@ -239,13 +239,17 @@ def decode_leg(dev, steps_per_call, calls, warmup, peaks, B=64, H=8, d=128, l2_d
             "state_mb": state_bytes / 2 / 1e6, "state_fits_l2": state_bytes / 2 < 126e6}
 
 
-def e2e_leg(w, dev, steps, warmup):
-    """Same step, host buffers: pinned host -> device copies of every input, the launch, and the
-    device -> host read of out and final state, all inside the timed region."""
+def e2e_leg(w, dev, steps, warmup, groups=4):
+    """Same step, host buffers: pinned host -> device copies of every input, the launches, and the
+    device -> host read of out and final state, all inside the timed region.  The batch is cut into `groups`
+    groups of sequences (they are independent problems) that go round two streams, so that the upload of one
+    group, the kernel of another and the download of a third overlap; the step ends when both streams have."""
     import torch
     from paper_2605_08587_b200 import kla_chunk_fwd
     host = {k: getattr(w, k).pin_memory() for k in ("q", "k", "v", "log_alpha", "eta")}
     B, T, H, d = w.q.shape
+    groups = max(1, min(groups, B))
+    cuts = [B * g // groups for g in range(groups + 1)]
     devbuf = {k: torch.empty_like(v, device=dev) for k, v in host.items()}
     out = torch.empty((B, T, H, d), device=dev, dtype=torch.bfloat16)
     fin = torch.empty((w.n_seq, H, d, d), device=dev, dtype=torch.float32)
@@ -253,16 +257,29 @@ def e2e_leg(w, dev, steps, warmup):
     fin_h = torch.empty(fin.shape, dtype=fin.dtype).pin_memory()
     h2d = sum(v.numel() * v.element_size() for v in host.values())
     d2h = out.numel() * out.element_size() + fin.numel() * fin.element_size()
+    main = torch.cuda.current_stream()
+    side = [torch.cuda.Stream(device=dev) for _ in range(2)]
+    done = [torch.cuda.Event() for _ in range(2)]
 
     def step():
-        for k in host:
-            devbuf[k].copy_(host[k], non_blocking=True)
-        kla_chunk_fwd(devbuf["q"], devbuf["k"], devbuf["v"], devbuf["log_alpha"], devbuf["eta"], w.eps,
-                      chunk=w.chunk, out=out, final_state=fin)
-        out_h.copy_(out, non_blocking=True)
-        fin_h.copy_(fin, non_blocking=True)
+        start = torch.cuda.Event()
+        start.record(main)
+        for s in side:
+            s.wait_event(start)
+        for g in range(groups):
+            lo, hi = cuts[g], cuts[g + 1]
+            with torch.cuda.stream(side[g % 2]):
+                for k in host:
+                    devbuf[k][lo:hi].copy_(host[k][lo:hi], non_blocking=True)
+                kla_chunk_fwd(devbuf["q"][lo:hi], devbuf["k"][lo:hi], devbuf["v"][lo:hi], devbuf["log_alpha"][lo:hi],
+                              devbuf["eta"][lo:hi], w.eps, chunk=w.chunk, out=out[lo:hi], final_state=fin[lo:hi])
+                out_h[lo:hi].copy_(out[lo:hi], non_blocking=True)
+                fin_h[lo:hi].copy_(fin[lo:hi], non_blocking=True)
+        for i, s in enumerate(side):
+            done[i].record(s)
+            main.wait_event(done[i])
 
-    ms = time_launches(step, steps, warmup, torch.cuda.current_stream())
+    ms = time_launches(step, steps, warmup, main)
     return ms, h2d, d2h
 
 

@@ -98,7 +98,8 @@ typedef struct {
 
 /*
  * Scratch needed by kla_chunk_fwd for this descriptor (shape, dtypes, flags) and chunk length; 0 unless the
- * segment-parallel scan applies (then: per-segment transition maps and states, 3 x B x G x H x d_k x d_v fp32).
+ * segment-parallel scan applies (then: per-segment transition maps and states, 3 x B x G x H x d_k x d_v fp32) or the
+ * input is packed and goes to the tensor-core kernel (then: one int32 per sequence, for a longest-first order).
  * Computed on the host (it reads the current device's SM count when a device is present); returns 0 for an
  * invalid descriptor.  The same descriptor must be passed to kla_chunk_fwd with a workspace of at least this size.
  */

@@ -63,6 +63,15 @@ static kla_status check_chunk(const kla_desc *d, const void *q, const void *k, c
     return KLA_OK;
 }
 
+// Packed input: the tensor-core kernel takes its sequences longest first (one int32 per sequence of scratch).
+static size_t order_bytes(const kla_desc *d, int32_t chunk)
+{
+    if (!d->cu_seqlens || d->n_seq < 2 || d->n_seq > 4096 || (d->flags & KLA_FLAG_FORCE_SIMT) ||
+        !chunk_tc_supported(d->d_k, chunk, d->io_dtype))
+        return 0;
+    return ((size_t)d->n_seq * sizeof(int32_t) + 255) & ~(size_t)255;
+}
+
 // ---- segment-parallel scan: when to use it, and the workspace it needs ----------------------------------------------
 struct SegPlan {
     int G = 0;            // segments per sequence (0: plain launch)
@@ -128,7 +137,9 @@ extern "C" {
 size_t kla_chunk_fwd_workspace_bytes(const kla_desc *desc, int32_t chunk)
 {
     if (check_common(desc) != KLA_OK) return 0;
-    // the chunk kernels keep every intermediate on chip; only the segment-parallel scan needs scratch
+    // the chunk kernels keep every intermediate on chip; scratch is needed by the segment-parallel scan and, for
+    // packed input on the tensor-core path, by the longest-first order of the sequences
+    if (order_bytes(desc, chunk)) return order_bytes(desc, chunk);
     return plan_segments(desc, chunk).bytes;
 }
 
@@ -187,8 +198,14 @@ kla_status kla_chunk_fwd(const kla_desc *desc, const void *q, const void *k, con
         err = launch_chunk_tc(p3, desc->d_k, desc->io_dtype, desc->out_dtype, stream);
         return err == cudaSuccess ? KLA_OK : KLA_ERR_LAUNCH;
     }
-    if (!(desc->flags & KLA_FLAG_FORCE_SIMT) && chunk_tc_supported(desc->d_k, chunk, desc->io_dtype))
+    if (!(desc->flags & KLA_FLAG_FORCE_SIMT) && chunk_tc_supported(desc->d_k, chunk, desc->io_dtype)) {
+        if (order_bytes(desc, chunk)) {
+            int32_t *order = (int32_t *)desc->workspace;
+            if (launch_seq_order(desc->cu_seqlens, desc->n_seq, order, stream) != cudaSuccess) return KLA_ERR_LAUNCH;
+            p.seq_order = order;
+        }
         err = launch_chunk_tc(p, desc->d_k, desc->io_dtype, desc->out_dtype, stream);
+    }
     else
         err = launch_chunk_simt(p, desc->d_k, chunk, desc->io_dtype, desc->out_dtype, stream);
     return err == cudaSuccess ? KLA_OK : KLA_ERR_LAUNCH;

@@ -252,6 +252,7 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     const int h = (blockIdx.x / nslices) % p.H;
     int n = blockIdx.x / (nslices * p.H);
     if (p.seg_pass == 1) n = (n / (p.seg_G - 1)) * p.seg_G + n % (p.seg_G - 1);
+    else if (p.seg_pass == 0 && p.seq_order) n = p.seq_order[n];   // packed input: longest sequences first
     const bool no_out = p.seg_pass == 1;
 
     int tok0, len;

@@ -28,7 +28,11 @@ struct ChunkParams {
     //               final_state, at the sequence's index.
     int32_t seg_pass, seg_G;
     int32_t variant;     // bit 0: beta_t = eta_t instead of Eq. 3; bit 1: read-out divided by ||q_t||; bit 2: test hook
-    float *map_state;
+    union {
+        float *map_state;            // segment pass 1
+        const int32_t *seq_order;    // packed input, plain launch: block b works on sequence seq_order[b] (longest
+                                     // first, so that the long sequences do not end up in the last wave); may be null
+    };
 };
 constexpr int32_t VARIANT_COEFF_ETA = 1, VARIANT_QNORM = 2, VARIANT_TEST_TIMEOUT = 4;
 
@@ -54,6 +58,8 @@ cudaError_t launch_chunk_tc(const ChunkParams &p, int d, int io_dtype, int out_d
                             cudaStream_t stream);
 // Segment-parallel helpers (segscan.cu).  cu_seg[b * G + g] = b * T + min(g * seg_len, T), one more entry = B * T.
 cudaError_t launch_seg_bounds(int32_t *cu_seg, int B, int T, int G, int seg_len, cudaStream_t stream);
+// order[r] = index of the sequence with the r-th largest length (ties by index); n_seq small (quadratic work)
+cudaError_t launch_seq_order(const int32_t *cu_seqlens, int n_seq, int32_t *order, cudaStream_t stream);
 // start[b, 0] = init (or 0); start[b, g + 1] = map[b, g] . start[b, g] + local[b, g]   (d x d products, fp32)
 cudaError_t launch_seg_combine(const float *init_state, const float *map, const float *local, float *start, int B, int H,
                                int G, int d, cudaStream_t stream);

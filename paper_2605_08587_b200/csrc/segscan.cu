@@ -24,6 +24,20 @@ __global__ void seg_bounds_kernel(int32_t *cu_seg, int B, int T, int G, int seg_
     cu_seg[i] = b * T + min(g * seg_len, T);
 }
 
+// Rank of every sequence by decreasing length (ties by index): order[rank] = sequence.
+__global__ void seq_order_kernel(const int32_t *cu_seqlens, int n_seq, int32_t *order)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n_seq) return;
+    const int li = cu_seqlens[i + 1] - cu_seqlens[i];
+    int rank = 0;
+    for (int j = 0; j < n_seq; ++j) {
+        const int lj = cu_seqlens[j + 1] - cu_seqlens[j];
+        rank += (lj > li || (lj == li && j < i)) ? 1 : 0;
+    }
+    order[rank] = i;
+}
+
 // One CTA per (sequence, head, 16-column slice of the state); thread r owns row r of the slice.
 template <int D>
 __global__ void __launch_bounds__(D) seg_combine_kernel(const float *init_state, const float *map, const float *local,
@@ -89,6 +103,13 @@ cudaError_t launch_seg_bounds(int32_t *cu_seg, int B, int T, int G, int seg_len,
 {
     const int n = B * G + 1;
     seg_bounds_kernel<<<(n + 127) / 128, 128, 0, stream>>>(cu_seg, B, T, G, seg_len);
+    count_launch(1);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_seq_order(const int32_t *cu_seqlens, int n_seq, int32_t *order, cudaStream_t stream)
+{
+    seq_order_kernel<<<(n_seq + 127) / 128, 128, 0, stream>>>(cu_seqlens, n_seq, order);
     count_launch(1);
     return cudaGetLastError();
 }

@@ -137,6 +137,16 @@ def test_workspace_grows_only_when_sequences_are_cut_into_segments(lib):
     assert lib.kla_chunk_fwd_workspace_bytes(ctypes.byref(long1), 32) == 0
 
 
+def test_packed_input_asks_for_one_word_per_sequence(lib):
+    """Packed input on the tensor-core path is taken longest sequence first: one int32 per sequence of scratch."""
+    import numpy as np
+    cu = np.array([0, 100, 164, 1000], dtype=np.int32)
+    d = _desc(B=1, T=1000, H=2, d_k=64, d_v=64, n_seq=3, cu_seqlens=FAKE, host_seqlens=cu.ctypes.data)
+    assert lib.kla_chunk_fwd_workspace_bytes(ctypes.byref(d), 64) == 256
+    assert lib.kla_chunk_fwd_workspace_bytes(ctypes.byref(d), 32) == 0        # CUDA-core kernel
+    assert _call_chunk(lib, d) == -7                                            # workspace missing
+
+
 def test_binding_rejects_cpu_tensors():
     import torch
     from paper_2605_08587_b200 import kla_chunk_fwd

@@ -71,6 +71,12 @@ typedef enum { KLA_F32 = 0, KLA_BF16 = 1 } kla_dtype;
  * bounded device-side wait runs out (about one second), every CTA gives up in an orderly way and KLA_ERR_TIMEOUT
  * appears in *status_word.  Outputs are then undefined; the context stays usable. */
 #define KLA_FLAG_TEST_TIMEOUT 16
+/* With d_v = 128 the two CTAs that hold the two 64-column slices of a head run as a thread-block cluster and share
+ * the work that does not depend on the state (each inverts every other chunk's I + B X and hands the result to its
+ * peer through distributed shared memory).  This flag launches them as independent CTAs instead, each doing all of
+ * that work itself; the arithmetic is the same, so the results are bit-identical.  Used to cross-check the two
+ * launch forms. */
+#define KLA_FLAG_NO_PAIR 32
 #define KLA_FLAG_NO_SEGMENTS 2            /* never cut sequences into segments                              */
 #define KLA_FLAG_SEGMENTS(g) ((g) << 8)   /* force g segments per sequence, 2 <= g <= 255 (fewer if T is short) */
 

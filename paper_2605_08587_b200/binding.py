@@ -14,7 +14,7 @@ LIB_PATH = os.path.join(_HERE, "libkla_b200.so")
 
 KLA_F32, KLA_BF16 = 0, 1
 KLA_FLAG_NONE, KLA_FLAG_FORCE_SIMT, KLA_FLAG_NO_SEGMENTS = 0, 1, 2
-KLA_FLAG_COEFF_ETA, KLA_FLAG_QNORM, KLA_FLAG_TEST_TIMEOUT = 4, 8, 16
+KLA_FLAG_COEFF_ETA, KLA_FLAG_QNORM, KLA_FLAG_TEST_TIMEOUT, KLA_FLAG_NO_PAIR = 4, 8, 16, 32
 
 
 def KLA_FLAG_SEGMENTS(g: int) -> int:

@@ -163,7 +163,8 @@ kla_status kla_chunk_fwd(const kla_desc *desc, const void *q, const void *k, con
     p.trace = nullptr;
     p.seg_pass = 0; p.seg_G = 0; p.map_state = nullptr;
     p.variant = ((desc->flags & KLA_FLAG_COEFF_ETA) ? VARIANT_COEFF_ETA : 0) | ((desc->flags & KLA_FLAG_QNORM) ? VARIANT_QNORM : 0) |
-                ((desc->flags & KLA_FLAG_TEST_TIMEOUT) ? VARIANT_TEST_TIMEOUT : 0);
+                ((desc->flags & KLA_FLAG_TEST_TIMEOUT) ? VARIANT_TEST_TIMEOUT : 0) |
+                ((desc->flags & KLA_FLAG_NO_PAIR) ? VARIANT_NO_PAIR : 0);
     p.B = desc->B; p.T = desc->T; p.H = desc->H; p.n_seq = desc->n_seq;
     p.eps = eps;
     if (desc->T == 0) {

@@ -15,6 +15,10 @@
 //                            O = D_gamma Q S_0 + P U                                     (Eq. 8)
 //                            S <- gamma_C S_0 + K^T diag(exp(g_C - g_j)) U               (Eq. 9)
 //
+// With two column slices per head (d_v = 128) the two CTAs of a head are launched as a thread-block cluster and
+// share the pre group's work: each forms X, T and P of every other chunk and copies the operand tiles and the
+// per-token scalars into the peer's shared memory (kernel template parameter PAIR).
+//
 // Tensor-core products per chunk (fp32 accumulation in TMEM):
 //   MMA-1  [K;Q] K^T   M=128   -> K K^T (lanes 0..63) and Q K^T (lanes 64..127), double-buffered
 //   MMA-2  K S_0, Q S_0        two M=64 products, S_0 = S_hi + S_lo
@@ -35,6 +39,7 @@
 // KLA_ERR_TIMEOUT through the status word, releases its TMEM and exits.
 #include <cuda.h>
 
+#include <cstddef>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -82,7 +87,11 @@ enum Bar {
     B_D4_DONE = 15,          // P U (and, earlier in the pipe, Q S_0) of chunk c complete
     B_TAIL_READY = 16,       // masked rows of the last chunk zeroed
     B_V_FULL = 17,           // V slice of chunk c landed
-    B_COUNT = 18
+    B_T_FREE = 18,           // paired CTAs: MMA-3(c) of both CTAs complete (the T tiles may be overwritten)
+    B_P_FREE = 19,           // paired CTAs: MMA-4(c) of both CTAs complete
+    B_SCAL_READY0 = 20,      // +(c & 1), paired CTAs: beta, gamma, exp(g_C - g) of chunk c written (long before T(c));
+                             // one barrier per owner, because nothing orders the two owners' arrivals
+    B_COUNT = 22
 };
 
 template <int D>
@@ -170,6 +179,22 @@ __device__ __forceinline__ bool pg_any(bool flag)
 #define KLA_TR(r, c, e) do { } while (0)
 #endif
 
+// 4 x 4 transpose over the four lanes of a quad (t = lane & 3): on entry lane t holds v[j] = element (t, j), on
+// exit v[s] = element (s, t).  Two butterfly stages; every lane of the warp must call it.
+__device__ __forceinline__ void quad_transpose(uint32_t (&v)[4], int t)
+{
+    const bool o1 = t & 1, o2 = t & 2;
+    uint32_t x = o1 ? v[0] : v[1], y = o1 ? v[2] : v[3];
+    x = __shfl_xor_sync(0xffffffffu, x, 1);
+    y = __shfl_xor_sync(0xffffffffu, y, 1);
+    if (o1) { v[0] = x; v[2] = y; } else { v[1] = x; v[3] = y; }
+    x = o2 ? v[0] : v[2];
+    y = o2 ? v[1] : v[3];
+    x = __shfl_xor_sync(0xffffffffu, x, 2);
+    y = __shfl_xor_sync(0xffffffffu, y, 2);
+    if (o2) { v[0] = x; v[1] = y; } else { v[2] = x; v[3] = y; }
+}
+
 // One level of the blocked inverse of I + B X (X strictly lower triangular, 64 x 64, in `tl`): for every pair
 // of adjacent BS x BS diagonal blocks (T_00, T_11 already inverted) the block below the diagonal becomes
 //   T_10 = -T_11 (B_1 X_10 T_00).
@@ -226,7 +251,11 @@ __device__ __forceinline__ void merge_level(float *tl, float *mm, const float *b
 
 // VAR: compiled with the layer-edge variants (beta = eta, read-out over ||q||); the default instantiation carries
 // none of their code.
-template <int D, typename OUT, bool VAR>
+// PAIR: the two CTAs that hold the two column slices of one (sequence, head) run as a thread-block cluster and
+// share the state-independent work: the CTA of rank r forms X, T and P of the chunks c with c mod 2 = r and writes
+// the T and P operand tiles (and beta) into both CTAs' shared memory, so that each pre group has two chunk
+// periods for one inverse.  The decay scan, every MMA but MMA-1, and the chain stay per CTA.
+template <int D, typename OUT, bool VAR, bool PAIR>
 __global__ void __launch_bounds__(NT, 1)
 kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                     const __grid_constant__ CUtensorMap tm_v, ChunkParams p)
@@ -235,6 +264,8 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     constexpr int KB = Smem::KB;
     constexpr int SLICES = D / NS;
     constexpr uint32_t STAGE_BYTES = Smem::KQ_BYTES;
+    // a pair hands T and P over with one copy per hi/lo pair of tiles
+    static_assert(offsetof(Smem, t_lo) == offsetof(Smem, t_hi) + 8192 && offsetof(Smem, p_lo) == offsetof(Smem, p_hi) + 8192, "tile pairs must be contiguous");
     constexpr uint32_t ID_G = idesc_bf16(128, 64, 0, 0);    // [K;Q] K^T : A K-major, B K-major
     constexpr uint32_t ID_S = idesc_bf16(64, NS, 0, 1);     // K S / Q S / T rhs / P U : M=64, B MN-major
     constexpr uint32_t ID_DS = idesc_bf16(128, NS, 1, 1);   // K^T (D U): A MN-major, B MN-major
@@ -243,6 +274,7 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     Smem &sm = *reinterpret_cast<Smem *>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t rank = PAIR ? cluster_ctarank() : 0u;   // PAIR: adjacent blocks = the two slices of one head
     // plain launch: block = (sequence, head, slice).  Segment pass 1 doubles the slices (the second set carries
     // the transition map) and skips each sequence's last segment; see ChunkParams.
     const int nslices = p.seg_pass == 1 ? 2 * SLICES : SLICES;
@@ -293,8 +325,9 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             mbar_init(&sm.bar[B_D1_DONE0 + b], 1);
             mbar_init(&sm.bar[B_D1_FREE0 + b], PG_T / 32);
         }
-        mbar_init(&sm.bar[B_T_READY], PG_T / 32);
-        mbar_init(&sm.bar[B_P_READY], PG_T / 64);
+        // PAIR: one arrival per chunk, local (own chunk) or from the peer together with the bytes of its copy
+        mbar_init(&sm.bar[B_T_READY], PAIR ? 1 : PG_T / 32);
+        mbar_init(&sm.bar[B_P_READY], PAIR ? 1 : PG_T / 64);
         mbar_init(&sm.bar[B_S_READY], CG_T / 32);
         mbar_init(&sm.bar[B_D2_DONE], 1);
         mbar_init(&sm.bar[B_RHS_READY], CG_T / 32);
@@ -304,6 +337,10 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         mbar_init(&sm.bar[B_D4_DONE], 1);
         mbar_init(&sm.bar[B_TAIL_READY], PG_T / 32);
         mbar_init(&sm.bar[B_V_FULL], 1);
+        mbar_init(&sm.bar[B_T_FREE], 2);
+        mbar_init(&sm.bar[B_P_FREE], 2);
+        mbar_init(&sm.bar[B_SCAL_READY0], 1);
+        mbar_init(&sm.bar[B_SCAL_READY0 + 1], 1);
         sm.abort_flag = 0;
         mbar_fence_init();
     }
@@ -312,6 +349,7 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     if (warp == 0) tmem_alloc(&sm.tmem_base, TM_COLS);
     tc_fence_before();
     __syncthreads();
+    if constexpr (PAIR) cluster_sync_all();   // the peer's barriers are initialised before anything arrives on them
     tc_fence_after();
     const uint32_t tmem = sm.tmem_base;
     const uint32_t tm_lane = tmem + ((uint32_t)((warp & 3) * 32) << 16);  // this warp's 32 TMEM lanes
@@ -372,11 +410,24 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         const uint32_t d_dh = desc_lo(smem_desc_sw128(smem_u32(sm.du_hi), 16, 1024)), d_dl = desc_lo(smem_desc_sw128(smem_u32(sm.du_lo), 16, 1024));
         constexpr uint32_t STAGE_STEP = (uint32_t)(Smem::KQ_BYTES >> 4);
 
-        auto mma1 = [&](int c) {  // [K;Q] K^T -> D1 buffer c & 1
+        auto mma1 = [&](int c) {  // [K;Q] K^T -> D1 buffer c & 1 (PAIR: this CTA's chunks alternate between the buffers)
             const uint32_t a0 = d_kq0 + (uint32_t)(c % NSTAGE) * STAGE_STEP;
+            const int b = PAIR ? (c >> 1) & 1 : c & 1;
 #pragma unroll 1
-            for (int kb = 0; kb < KB; ++kb) KLA_SEQ(tmem + TM_D1 + (uint32_t)(c & 1) * 64, a0 + kb * 1024, 2, a0 + kb * 1024, 2, ID_G, kb > 0);
-            mma_commit(&sm.bar[B_D1_DONE0 + (c & 1)]);
+            for (int kb = 0; kb < KB; ++kb) KLA_SEQ(tmem + TM_D1 + (uint32_t)b * 64, a0 + kb * 1024, 2, a0 + kb * 1024, 2, ID_G, kb > 0);
+            mma_commit(&sm.bar[B_D1_DONE0 + b]);
+        };
+        // PAIR: MMA-1 of one of this CTA's own chunks, once its tiles have landed and its D1 buffer (last used by
+        // chunk c - 4) has been read
+        auto mma1_own = [&](int c) -> bool {
+            if (!wwait(B_FULL0 + c % NSTAGE, (uint32_t)((c / NSTAGE) & 1))) return false;
+            if (c + 1 == nchunks && last_rows < C)
+                if (!wwait(B_TAIL_READY, 0)) return false;
+            if (c >= 4)
+                if (!wwait(B_D1_FREE0 + ((c >> 1) & 1), (uint32_t)(((c >> 2) - 1) & 1))) return false;
+            tc_fence_after();
+            mma1(c);
+            return true;
         };
         // [K or Q](c) S_0 -> d; qoff = 512 selects the Q tile of a block; S_0 = S_hi + S_lo
         auto mma_xs = [&](uint32_t d, uint32_t k0, uint32_t qoff) {
@@ -394,6 +445,78 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         bool ok = true;
         for (int c = 0; c < NSTAGE && c < nchunks; ++c) issue_tma(c);
         issue_tma_v(0);
+        if constexpr (PAIR) {
+            // ---- paired CTAs.  The tensor pipe runs the MMAs in issue order at ~60 cycles each, so what is not on the
+            // chain goes where the pipe would idle and can finish before the chain's next product is ready:
+            //   K S_0(c) | MMA-1 of this CTA's chunk c + 2 (if its tiles have landed)     while the chain forms rhs(c)
+            //   MMA-3(c) | Q S_0(c) (| MMA-1 if not issued above)                          while the chain forms U(c)
+            //   MMA-5(c) | MMA-4(c)                                                        while the chain updates S
+            // Order constraints: Q S_0(c) before MMA-5(c), whose completion lets the chain overwrite the S tiles;
+            // MMA-4(c) before K S_0(c+1), whose completion lets it overwrite U.
+            auto ready = [&](int b, uint32_t parity) -> bool {
+                return __all_sync(0xffffffffu, mbar_test_wait(&sm.bar[b], parity));
+            };
+            if ((int)rank < nchunks) ok = mma1_own((int)rank);
+            for (int c = 0; ok && c < nchunks; ++c) {
+                const bool own = (uint32_t)(c & 1) == rank;
+                // a chunk of the peer: no MMA-1 here has waited for its tiles
+                if (!own)
+                    if (!(ok = wwait(B_FULL0 + c % NSTAGE, (uint32_t)((c / NSTAGE) & 1)))) break;
+                // the masked rows of the last chunk are zeroed before any product reads its tiles
+                if (c + 1 == nchunks && last_rows < C)
+                    if (!(ok = wwait(B_TAIL_READY, 0))) break;
+                const uint32_t ph = (uint32_t)(c & 1);
+                const uint32_t k0 = d_kq0 + (uint32_t)(c % NSTAGE) * STAGE_STEP;
+                const uint32_t kt0 = d_kt0 + (uint32_t)(c % NSTAGE) * STAGE_STEP;
+                KLA_TR(0, c, 0);
+                if (!(ok = wwait(B_S_READY, ph))) break;
+                KLA_TR(0, c, 1);
+                tc_fence_after();
+                mma_xs(tmem + TM_KS, k0, 0);
+                mma_commit(&sm.bar[B_D2_DONE]);
+                const int cn = c + 2;   // this CTA's next chunk
+                bool m1_due = own && cn < nchunks;
+                if (m1_due && ready(B_FULL0 + cn % NSTAGE, (uint32_t)((cn / NSTAGE) & 1)) &&
+                    (!(cn + 1 == nchunks && last_rows < C) || ready(B_TAIL_READY, 0)) &&
+                    (cn < 4 || ready(B_D1_FREE0 + ((cn >> 1) & 1), (uint32_t)(((cn >> 2) - 1) & 1)))) {
+                    tc_fence_after();
+                    mma1(cn);
+                    m1_due = false;
+                }
+                KLA_TR(0, c, 2);
+                // MMA-3(c): U = T rhs
+                if (!(ok = wwait(B_T_READY, ph))) break;
+                KLA_TR(0, c, 3);
+                if (!(ok = wwait(B_RHS_READY, ph))) break;
+                KLA_TR(0, c, 4);
+                if (c + 1 < nchunks) issue_tma_v(c + 1);
+                tc_fence_after();
+                mma_3(tmem + TM_U, d_th, d_tl, d_rh, d_rl);
+                mma_commit(&sm.bar[B_D3_DONE]);
+                mma_commit_multicast(&sm.bar[B_T_FREE], 3);
+                if (!no_out) mma_xs(tmem + ((c & 1) ? TM_QS1 : TM_QS0), k0, 512);
+                if (m1_due)
+                    if (!(ok = mma1_own(cn))) break;
+                KLA_TR(0, c, 5);
+                // MMA-5(c): K^T (D U)
+                if (!(ok = wwait(B_U_READY, ph))) break;
+                KLA_TR(0, c, 6);
+                tc_fence_after();
+#pragma unroll 1
+                for (int t = 0; t < 2; ++t) KLA_SEQ(tmem + TM_DS, kt0, 128, t ? d_dl : d_dh, 128, ID_DS, t);
+                mma_commit(&sm.bar[B_D5_DONE]);
+                // MMA-4(c): P U
+                if (!no_out) {
+                    if (!(ok = wwait(B_P_READY, ph))) break;
+                    tc_fence_after();
+                    mma_3(tmem + TM_PU, d_ph, d_pl, d_rh, d_rl);
+                    mma_commit(&sm.bar[B_D4_DONE]);
+                    mma_commit_multicast(&sm.bar[B_P_FREE], 3);
+                }
+                KLA_TR(0, c, 7);
+                // (the chain group, which sees MMA-5(c) complete first, refills the K/Q stage of chunk c)
+            }
+        } else {
         // iteration c issues MMA-1(c+1) first, as early as its inputs and its D1 buffer allow; c = -1 does only that
         for (int c = -1; ok && c < nchunks; ++c) {
             if (c + 1 < nchunks) {
@@ -456,6 +579,239 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 if (!(ok = wwait(B_D5_DONE, ph))) break;
                 issue_tma(c + NSTAGE);
             }
+        }
+        }
+    } else if (PAIR && warp >= PG_BASE / 32) {
+        // =============================== pre group, paired CTAs ============================================
+        // This CTA's own chunks (c mod 2 = rank): decay scan, X(c), beta(c), T(c) and P(c); the per-token scalars
+        // and the T and P operand tiles go into both CTAs.  The peer's chunks: only the zeroing of the masked rows
+        // of the last chunk (the K and Q tiles are per CTA).  Warp roles as in the unpaired group: warps 0, 1, 4, 5
+        // hold rows of K K^T, warps 2, 3, 6, 7 rows of Q K^T.
+        const int pt = tid - PG_BASE;
+        const int q = warp & 3, chh = (warp - PG_BASE / 32) >> 2;
+        const bool is_g = q < 2;
+        const int i = (q & 1) * 32 + lane;
+        const bool live = chh <= (q & 1);
+        const bool scan_warp = q == 0 && chh == 1;
+        // distance from a shared-memory address of this CTA to the same location in the peer CTA
+        const uint32_t peer_off = mapa_u32(smem_u32(&sm), rank ^ 1u) - smem_u32(&sm);
+        float la_next0 = 0.f, la_next1 = 0.f, eta_next = 0.f;
+        auto fetch_gates = [&](int c) {
+            if (scan_warp) {
+                const int t = c * C + 2 * lane;
+                la_next0 = (t < len) ? p.log_alpha[(size_t)(tok0 + t) * p.H + h] : 0.f;
+                la_next1 = (t + 1 < len) ? p.log_alpha[(size_t)(tok0 + t + 1) * p.H + h] : 0.f;
+            }
+            if (is_g && chh == q) {
+                const int t = c * C + i;
+                eta_next = (t < len) ? p.eta[(size_t)(tok0 + t) * p.H + h] : 0.f;
+            }
+        };
+        if ((int)rank < nchunks) fetch_gates((int)rank);
+        bool okp = true;   // outcome of the P warps' waits, folded into the next collective decision
+        for (int c = 0; c < nchunks; ++c) {
+            const uint32_t ph = (uint32_t)(c & 1);
+            const int rows = (c == nchunks - 1) ? last_rows : C;
+            const int sc = c % NSTAGE;
+            const bool own = (uint32_t)(c & 1) == rank;
+            const float la0 = la_next0, la1 = la_next1, eta_cur = eta_next;
+            if (own && c + 2 < nchunks) fetch_gates(c + 2);
+            if (own && scan_warp) {
+                float incl = la0 + la1;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const float t = __shfl_up_sync(0xffffffffu, incl, o);
+                    if (lane >= o) incl += t;
+                }
+                const float gC = __shfl_sync(0xffffffffu, incl, 31);
+                const float a2 = (incl - la1) * LOG2E, b2 = incl * LOG2E, c2 = gC * LOG2E;
+                *reinterpret_cast<float2 *>(&sm.g2[sc][2 * lane]) = make_float2(a2, b2);
+                *reinterpret_cast<float2 *>(&sm.gam[sc][2 * lane]) = make_float2(ex2_approx(a2), ex2_approx(b2));
+                *reinterpret_cast<float2 *>(&sm.dec[sc][2 * lane]) = make_float2(ex2_approx(c2 - a2), ex2_approx(c2 - b2));
+                fence_async_smem();   // gam and dec are also copied to the peer
+            }
+            KLA_TR(1, c, 0);
+            bool okc = okp;
+            if (rows < C && okc) {
+                okc = wait(B_FULL0 + sc, (uint32_t)((c / NSTAGE) & 1));
+                if (okc) {
+                    unsigned char *kq = sm.kq[sc];
+                    for (int e = pt; e < (C - rows) * 8; e += PG_T) {
+                        const int r = rows + e / 8, ch = e % 8;
+                        const uint4 z = make_uint4(0, 0, 0, 0);
+#pragma unroll
+                        for (int kb = 0; kb < KB; ++kb) {
+                            *reinterpret_cast<uint4 *>(kq + kb * 16384 + sw128(r, ch)) = z;
+                            *reinterpret_cast<uint4 *>(kq + kb * 16384 + 8192 + sw128(r, ch)) = z;
+                        }
+                    }
+                    fence_async_smem();
+                    warp_arrive(B_TAIL_READY);
+                }
+            }
+            if (pg_any(!okc)) break;   // also publishes the decay sums to the whole group
+            if (!own) continue;   // the peer's chunk: its scalars, T and P arrive from there
+
+            const int b1 = (c >> 1) & 1;                       // D1 buffer of this CTA's chunk c, ...
+            const uint32_t ph1 = (uint32_t)((c >> 2) & 1);     // ... in its (c / 4)-th use
+            KLA_TR(1, c, 9);
+            if (is_g) {
+                // ---- X = A^- o K K^T (this thread: row i, 32 columns) and beta_i, Eq. 3 ----------------------
+                okc = wait(B_D1_DONE0 + b1, ph1);
+                KLA_TR(1, c, 10);
+                if (okc) {
+                    tc_fence_after();
+                    if (live) {
+                        const float gi2 = sm.g2[sc][i];
+                        float dg = 0.f;   // G_ii = ||k_i||^2
+                        const uint32_t tbase = tm_lane + TM_D1 + (uint32_t)b1 * 64 + chh * 32;
+#pragma unroll 1
+                        for (int grp = 0; grp < 4; ++grp) {
+                            float a[8];
+                            tmem_ld8(tbase + grp * 8, a);
+                            const int j0 = chh * 32 + grp * 8;
+                            const float4 ga = *reinterpret_cast<const float4 *>(&sm.g2[sc][j0]);
+                            const float4 gb = *reinterpret_cast<const float4 *>(&sm.g2[sc][j0 + 4]);
+                            const float gj[8] = {ga.x, ga.y, ga.z, ga.w, gb.x, gb.y, gb.z, gb.w};
+                            float x[8];
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) {
+                                x[e] = (j0 + e < i) ? ex2_approx(gi2 - gj[e]) * a[e] : 0.f;
+                                dg = (j0 + e == i) ? a[e] : dg;
+                            }
+                            *reinterpret_cast<float4 *>(&sm.tl[i * LDT + j0]) = make_float4(x[0], x[1], x[2], x[3]);
+                            *reinterpret_cast<float4 *>(&sm.tl[i * LDT + j0 + 4]) = make_float4(x[4], x[5], x[6], x[7]);
+                        }
+                        if (chh == q) {
+                            sm.beta[sc][i] = (i < rows) ? eta_cur / (dg + p.eps) : 0.f;
+                            fence_async_smem();
+                        }
+                    }
+                    KLA_TR(1, c, 11);
+                    tc_fence_before();
+                    warp_arrive(B_D1_FREE0 + b1);
+                }
+            } else if (no_out) {
+                warp_arrive(B_D1_FREE0 + b1);   // nothing reads Q K^T
+            }
+            if (pg_any(!okc)) break;
+            KLA_TR(1, c, 1);
+            // The per-token scalars of chunk c (beta, gamma, exp(g_C - g)) go to both chains now, more than a chunk
+            // period before T(c): their rhs does not wait for the inverse.  (The peer's slot c mod 3 is free: its
+            // chain read the scalars of chunk c - 3 before MMA-3(c-3), which this group saw complete two chunks ago.)
+            if (pt == 0) {
+                const uint32_t rbar = smem_u32(&sm.bar[B_SCAL_READY0 + (int)rank]) + peer_off;
+                mbar_arrive_expect_tx_cluster(rbar, 768);
+                bulk_copy_to_cluster(smem_u32(sm.beta[sc]) + peer_off, smem_u32(sm.beta[sc]), 256, rbar);
+                bulk_copy_to_cluster(smem_u32(sm.gam[sc]) + peer_off, smem_u32(sm.gam[sc]), 256, rbar);
+                bulk_copy_to_cluster(smem_u32(sm.dec[sc]) + peer_off, smem_u32(sm.dec[sc]), 256, rbar);
+                mbar_arrive(&sm.bar[B_SCAL_READY0 + (int)rank]);
+            }
+
+            // ---- T = (I + B X)^-1 ----------------------------------------------------------------------------
+            const float *bet = sm.beta[sc];
+            if (pt < 64) {
+                const int blk = pt >> 3, j = pt & 7;
+                float *Lb = sm.tl + (blk * 8) * LDT + blk * 8;
+                float x[8];
+#pragma unroll
+                for (int r = 0; r < 8; ++r) {
+                    const float4 l0 = *reinterpret_cast<const float4 *>(Lb + r * LDT);
+                    const float4 l1 = *reinterpret_cast<const float4 *>(Lb + r * LDT + 4);
+                    const float l[8] = {l0.x, l0.y, l0.z, l0.w, l1.x, l1.y, l1.z, l1.w};
+                    float s = 0.f;
+#pragma unroll
+                    for (int m = 0; m < r; ++m) s += l[m] * x[m];
+                    x[r] = (r == j) ? 1.f : ((r > j) ? -bet[blk * 8 + r] * s : 0.f);
+                }
+                half_sync();
+#pragma unroll
+                for (int r = 0; r < 8; ++r) Lb[r * LDT + j] = x[r];
+            }
+            pg_sync();
+            KLA_TR(1, c, 2);
+            merge_level<8>(sm.tl, sm.mm, bet, pt);
+            KLA_TR(1, c, 6);
+            merge_level<16>(sm.tl, sm.mm, bet, pt);
+            KLA_TR(1, c, 7);
+            merge_level<32>(sm.tl, sm.mm, bet, pt);
+            KLA_TR(1, c, 3);
+            // ---- T as bf16 hi/lo operand tiles, once MMA-3(c-1) of both CTAs has read the previous ones ------------
+            bool okd = true;
+            if (c > 0 && pt >= PG_T - 32) okd = wait(B_T_FREE, ph ^ 1);
+            if (pg_any(!okd)) break;
+            KLA_TR(1, c, 4);
+            {
+                const int r = pt & 63, qq = pt >> 6;
+#pragma unroll 1
+                for (int ch = 0; ch < 2; ++ch) {
+                    const float4 a = *reinterpret_cast<const float4 *>(&sm.tl[r * LDT + qq * 16 + ch * 8]);
+                    const float4 b = *reinterpret_cast<const float4 *>(&sm.tl[r * LDT + qq * 16 + ch * 8 + 4]);
+                    uint4 hi, lo;
+                    split2(a.x, a.y, hi.x, lo.x);
+                    split2(a.z, a.w, hi.y, lo.y);
+                    split2(b.x, b.y, hi.z, lo.z);
+                    split2(b.z, b.w, hi.w, lo.w);
+                    const uint32_t o = sw128(r, qq * 2 + ch);
+                    *reinterpret_cast<uint4 *>(sm.t_hi + o) = hi;
+                    *reinterpret_cast<uint4 *>(sm.t_lo + o) = lo;
+                }
+            }
+            fence_async_smem();
+            pg_sync();  // every tile write is done (and the solve matrix may be reused by this CTA's next chunk)
+            if (pt == 0) {
+                // this CTA's copy is ready; the peer's is sent by the copy engine and counted on its barrier
+                const uint32_t rbar = smem_u32(&sm.bar[B_T_READY]) + peer_off;
+                mbar_arrive_expect_tx_cluster(rbar, 16384);
+                bulk_copy_to_cluster(smem_u32(sm.t_hi) + peer_off, smem_u32(sm.t_hi), 16384, rbar);   // t_hi and t_lo
+                mbar_arrive(&sm.bar[B_T_READY]);
+            }
+            KLA_TR(1, c, 5);
+
+            // ---- P(c) = A o Q K^T as bf16 hi/lo operand tiles into both CTAs (rows of Q K^T: warps 2, 3, 6, 7) --------
+            if (!is_g && !no_out) {
+                okp = wait(B_D1_DONE0 + b1, ph1);
+                if (okp && c > 0) okp = wait(B_P_FREE, ph ^ 1);   // MMA-4(c-1) of both CTAs has read the P tiles
+                if (okp) {
+                    tc_fence_after();
+                    const float gi2 = sm.g2[sc][i];
+                    const uint32_t tbase = tm_lane + TM_D1 + (uint32_t)b1 * 64 + chh * 32;
+#pragma unroll 1
+                    for (int grp = 0; grp < 4; ++grp) {
+                        uint4 hi = make_uint4(0, 0, 0, 0), lo = hi;
+                        if (live) {
+                            float a[8];
+                            tmem_ld8(tbase + grp * 8, a);
+                            const int j0 = chh * 32 + grp * 8;
+                            const float4 ga = *reinterpret_cast<const float4 *>(&sm.g2[sc][j0]);
+                            const float4 gb = *reinterpret_cast<const float4 *>(&sm.g2[sc][j0 + 4]);
+                            const float gj[8] = {ga.x, ga.y, ga.z, ga.w, gb.x, gb.y, gb.z, gb.w};
+                            float x[8];
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) x[e] = (j0 + e <= i) ? ex2_approx(gi2 - gj[e]) * a[e] : 0.f;
+                            split2(x[0], x[1], hi.x, lo.x);
+                            split2(x[2], x[3], hi.y, lo.y);
+                            split2(x[4], x[5], hi.z, lo.z);
+                            split2(x[6], x[7], hi.w, lo.w);
+                        }
+                        const uint32_t o = sw128(i, chh * 4 + grp);
+                        *reinterpret_cast<uint4 *>(sm.p_hi + o) = hi;
+                        *reinterpret_cast<uint4 *>(sm.p_lo + o) = lo;
+                    }
+                    tc_fence_before();
+                    fence_async_smem();
+                    warp_arrive(B_D1_FREE0 + b1);
+                }
+                // the four P warps meet (also when a wait gave up: nobody is left behind), then one thread publishes
+                asm volatile("bar.sync 4, 128;" ::: "memory");
+                if (okp && q == 2 && chh == 0 && lane == 0) {
+                    const uint32_t rbar = smem_u32(&sm.bar[B_P_READY]) + peer_off;
+                    mbar_arrive_expect_tx_cluster(rbar, 16384);
+                    bulk_copy_to_cluster(smem_u32(sm.p_hi) + peer_off, smem_u32(sm.p_hi), 16384, rbar);   // p_hi and p_lo
+                    mbar_arrive(&sm.bar[B_P_READY]);
+                }
+            }
+            KLA_TR(1, c, 12);
         }
     } else if (warp >= PG_BASE / 32) {
         // =============================== pre group ==========================================================
@@ -735,7 +1091,7 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             const int sc = c % NSTAGE;
             // ---- rhs = B (V - D_gamma K S_0) ------------------------------------------------------------------
             KLA_TR(2, c, 0);
-            if (!wait(B_T_READY, ph)) break;   // scalars of chunk c
+            if (!(PAIR ? wait(B_SCAL_READY0 + (c & 1), (uint32_t)((c >> 1) & 1)) : wait(B_T_READY, ph))) break;   // scalars of chunk c
             KLA_TR(2, c, 1);
             const float b0 = sm.beta[sc][i0], b1 = sm.beta[sc][i1];
             const float g0 = sm.gam[sc][i0], g1 = sm.gam[sc][i1];
@@ -799,6 +1155,19 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             // ---- state: S <- gamma_C S + K^T (D U) -----------------------------------------------------------------
             if (!wait(B_D5_DONE, ph)) break;
             KLA_TR(2, c, 6);
+            if constexpr (PAIR) {
+                // MMA-5(c) was the last reader of the K/Q stage of chunk c: refill it at once (this CTA's MMA-1 of
+                // chunk c + 3 may be due within a fraction of a chunk period)
+                if (ct == 0 && c + NSTAGE < nchunks) {
+                    const int cn = c + NSTAGE;
+                    mbar_expect_tx(&sm.bar[B_FULL0 + sc], STAGE_BYTES);
+#pragma unroll
+                    for (int kb = 0; kb < KB; ++kb) {
+                        tma_load_2d(sm.kq[sc] + kb * 16384, &tm_k, h * D + kb * 64, tok0 + cn * C, &sm.bar[B_FULL0 + sc]);
+                        tma_load_2d(sm.kq[sc] + kb * 16384 + 8192, &tm_q, h * D + kb * 64, tok0 + cn * C, &sm.bar[B_FULL0 + sc]);
+                    }
+                }
+            }
             tc_fence_after();
             {
                 float acc[32];
@@ -818,22 +1187,57 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             KLA_TR(2, c, 8);
             tc_fence_after();
             {
-                OUT *o0 = reinterpret_cast<OUT *>(p.out) + ((size_t)(tok0 + c * C + i0) * p.H + h) * D + sl * NS + cp;
-                OUT *o1 = reinterpret_cast<OUT *>(p.out) + ((size_t)(tok0 + c * C + i1) * p.H + h) * D + sl * NS + cp;
-                const uint32_t tq = tm16 + ((c & 1) ? TM_QS1 : TM_QS0);
-#pragma unroll 1
-                for (int j = 0; j < 4; ++j) {
-                    float acc[4], qs[4];
-                    tmem_ld16x256b_x1(tm16 + TM_PU + 8 * j, acc);
-                    tmem_ld16x256b_x1(tq + 8 * j, qs);
-                    if constexpr (VAR) {
-                        // read-out over ||q|| when asked for
-                        const float n0 = (p.variant & VARIANT_QNORM) ? sm.qn[sc][i0] : 1.f, n1 = (p.variant & VARIANT_QNORM) ? sm.qn[sc][i1] : 1.f;
-                        if (i0 < rows) store2(o0 + 8 * j, n0 * (g0 * qs[0] + acc[0]), n0 * (g0 * qs[1] + acc[1]));
-                        if (i1 < rows) store2(o1 + 8 * j, n1 * (g1 * qs[2] + acc[2]), n1 * (g1 * qs[3] + acc[3]));
-                    } else {
-                        if (i0 < rows) store2(o0 + 8 * j, g0 * qs[0] + acc[0], g0 * qs[1] + acc[1]);
-                        if (i1 < rows) store2(o1 + 8 * j, g1 * qs[2] + acc[2], g1 * qs[3] + acc[3]);
+                // This thread's accumulator values are column pairs cp + 8j (j = 0..3) of rows i0 and i1; a 4 x 4 transpose
+                // over the four lanes of a quad gives each lane 8 consecutive columns of both rows, so that every
+                // store is 16 bytes and a warp's store covers whole 32-byte sectors (2-element stores straight from the
+                // accumulator layout backed up the store queue for more than a thousand cycles per chunk).
+                float pu[16], qs[16];
+                tmem_ld16x256b_x4(tm16 + TM_PU, pu);
+                tmem_ld16x256b_x4(tm16 + ((c & 1) ? TM_QS1 : TM_QS0), qs);
+                float n0 = g0, n1 = g1, m0 = 1.f, m1 = 1.f;   // o = n * qs + m * pu
+                if constexpr (VAR) {
+                    if (p.variant & VARIANT_QNORM) {   // read-out over ||q||
+                        m0 = sm.qn[sc][i0]; m1 = sm.qn[sc][i1];
+                        n0 *= m0; n1 *= m1;
+                    }
+                }
+                const int t4 = lane & 3;
+                const size_t col = (size_t)sl * NS + hf * 32 + 8 * t4;
+                OUT *o0 = reinterpret_cast<OUT *>(p.out) + ((size_t)(tok0 + c * C + i0) * p.H + h) * D + col;
+                OUT *o1 = reinterpret_cast<OUT *>(p.out) + ((size_t)(tok0 + c * C + i1) * p.H + h) * D + col;
+                if constexpr (sizeof(OUT) == 2) {
+                    uint32_t a[4], b[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const __nv_bfloat162 x = __floats2bfloat162_rn(n0 * qs[4 * j] + m0 * pu[4 * j], n0 * qs[4 * j + 1] + m0 * pu[4 * j + 1]);
+                        const __nv_bfloat162 y = __floats2bfloat162_rn(n1 * qs[4 * j + 2] + m1 * pu[4 * j + 2], n1 * qs[4 * j + 3] + m1 * pu[4 * j + 3]);
+                        a[j] = *reinterpret_cast<const uint32_t *>(&x);
+                        b[j] = *reinterpret_cast<const uint32_t *>(&y);
+                    }
+                    quad_transpose(a, t4);
+                    quad_transpose(b, t4);
+                    if (i0 < rows) *reinterpret_cast<uint4 *>(o0) = make_uint4(a[0], a[1], a[2], a[3]);
+                    if (i1 < rows) *reinterpret_cast<uint4 *>(o1) = make_uint4(b[0], b[1], b[2], b[3]);
+                } else {
+                    uint32_t ax[4], ay[4], bx[4], by[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        ax[j] = __float_as_uint(n0 * qs[4 * j] + m0 * pu[4 * j]);
+                        ay[j] = __float_as_uint(n0 * qs[4 * j + 1] + m0 * pu[4 * j + 1]);
+                        bx[j] = __float_as_uint(n1 * qs[4 * j + 2] + m1 * pu[4 * j + 2]);
+                        by[j] = __float_as_uint(n1 * qs[4 * j + 3] + m1 * pu[4 * j + 3]);
+                    }
+                    quad_transpose(ax, t4);
+                    quad_transpose(ay, t4);
+                    quad_transpose(bx, t4);
+                    quad_transpose(by, t4);
+                    if (i0 < rows) {
+                        *reinterpret_cast<uint4 *>(o0) = make_uint4(ax[0], ay[0], ax[1], ay[1]);
+                        *reinterpret_cast<uint4 *>(o0 + 4) = make_uint4(ax[2], ay[2], ax[3], ay[3]);
+                    }
+                    if (i1 < rows) {
+                        *reinterpret_cast<uint4 *>(o1) = make_uint4(bx[0], by[0], bx[1], by[1]);
+                        *reinterpret_cast<uint4 *>(o1 + 4) = make_uint4(bx[2], by[2], bx[3], by[3]);
                     }
                 }
             }
@@ -850,6 +1254,8 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 
     tc_fence_before();
     __syncthreads();
+    // neither CTA of a pair leaves while the other may still write into its shared memory or signal its barriers
+    if constexpr (PAIR) cluster_sync_all();
     if (warp == 0) {
         tc_fence_after();
         tmem_dealloc(tmem, TM_COLS);
@@ -890,16 +1296,20 @@ bool make_tmap(CUtensorMap *tm, const void *base, uint64_t n_tok, uint64_t row_e
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int D, typename OUT, bool VAR>
+template <int D, typename OUT, bool VAR, bool PAIR>
 cudaError_t launch_v(const ChunkParams &p, cudaStream_t stream);
 
 template <int D, typename OUT>
 cudaError_t launch_t(const ChunkParams &p, cudaStream_t stream)
 {
-    return (p.variant != 0) ? launch_v<D, OUT, true>(p, stream) : launch_v<D, OUT, false>(p, stream);
+    if ((p.variant & ~VARIANT_NO_PAIR) != 0) return launch_v<D, OUT, true, false>(p, stream);
+    // two slices per head: the CTAs of a head run as a cluster and share the state-independent work
+    if constexpr (D == 2 * NS)
+        if (!(p.variant & VARIANT_NO_PAIR)) return launch_v<D, OUT, false, true>(p, stream);
+    return launch_v<D, OUT, false, false>(p, stream);
 }
 
-template <int D, typename OUT, bool VAR>
+template <int D, typename OUT, bool VAR, bool PAIR>
 cudaError_t launch_v(const ChunkParams &p, cudaStream_t stream)
 {
     using Smem = TcSmem<D>;
@@ -908,13 +1318,25 @@ cudaError_t launch_v(const ChunkParams &p, cudaStream_t stream)
     if (!make_tmap(&tq, p.q, n_tok, (uint64_t)p.H * D) || !make_tmap(&tk, p.k, n_tok, (uint64_t)p.H * D) ||
         !make_tmap(&tv, p.v, n_tok, (uint64_t)p.H * D))
         return cudaErrorInvalidValue;
-    auto kern = kla_chunk_tc_kernel<D, OUT, VAR>;
+    auto kern = kla_chunk_tc_kernel<D, OUT, VAR, PAIR>;
     const int smem = (int)sizeof(Smem) + 1024;
     cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (err != cudaSuccess) return err;
     // segment pass 1: (seg_G - 1) segments per sequence, twice the slices; p.n_seq counts all segments there
     const int grid = p.seg_pass == 1 ? (p.n_seq / p.seg_G) * (p.seg_G - 1) * p.H * 2 * (D / NS) : p.n_seq * p.H * (D / NS);
     if (grid == 0) return cudaSuccess;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(NT);
+    cfg.dynamicSmemBytes = (size_t)smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;   // blocks 2j, 2j + 1 = the two slices of one (sequence, head)
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = PAIR ? 1 : 0;
 #ifdef KLA_TRACE
     {
         static long long *tbuf = nullptr;
@@ -922,7 +1344,7 @@ cudaError_t launch_v(const ChunkParams &p, cudaStream_t stream)
         memset(tbuf, 0, 3 * 64 * 16 * sizeof(long long));
         ChunkParams pt = p;
         pt.trace = tbuf;
-        kern<<<grid, NT, smem, stream>>>(tq, tk, tv, pt);
+        cudaLaunchKernelEx(&cfg, kern, tq, tk, tv, pt);
         cudaDeviceSynchronize();
         const char *tf = getenv("KLA_TRACE_FILE");
         FILE *f = tf ? fopen(tf, "w") : nullptr;
@@ -939,9 +1361,9 @@ cudaError_t launch_v(const ChunkParams &p, cudaStream_t stream)
         return cudaGetLastError();
     }
 #endif
-    kern<<<grid, NT, smem, stream>>>(tq, tk, tv, p);
+    err = cudaLaunchKernelEx(&cfg, kern, tq, tk, tv, p);
     count_launch(1);
-    return cudaGetLastError();
+    return err != cudaSuccess ? err : cudaGetLastError();
 }
 
 }  // namespace

@@ -27,7 +27,7 @@ struct ChunkParams {
     //   seg_pass 3: every segment from its true start state; only the last segment of a sequence writes
     //               final_state, at the sequence's index.
     int32_t seg_pass, seg_G;
-    int32_t variant;     // bit 0: beta_t = eta_t instead of Eq. 3; bit 1: read-out divided by ||q_t||; bit 2: test hook
+    int32_t variant;     // bit 0: beta_t = eta_t instead of Eq. 3; bit 1: read-out divided by ||q_t||; bit 2: test hook; bit 3: see VARIANT_NO_PAIR
     union {
         float *map_state;            // segment pass 1
         const int32_t *seq_order;    // packed input, plain launch: block b works on sequence seq_order[b] (longest
@@ -35,6 +35,7 @@ struct ChunkParams {
     };
 };
 constexpr int32_t VARIANT_COEFF_ETA = 1, VARIANT_QNORM = 2, VARIANT_TEST_TIMEOUT = 4;
+constexpr int32_t VARIANT_NO_PAIR = 8;   // host side only: launch the two slices of a head as independent CTAs
 
 struct DecodeParams {
     const void *q, *k, *v;

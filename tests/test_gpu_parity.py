@@ -276,3 +276,29 @@ def test_bounded_wait_reports_timeout_and_context_stays_usable():
     ro, rf = oracle_chunk(w)
     assert int(status.item()) == 0
     assert rel_err(np64(out), ro) <= TOL_BF16 and rel_err(np64(fin), rf) <= TOL_BF16
+
+
+# ---- d_v = 128: the two slices of a head as a cluster that shares the solve (default) or as independent CTAs ----------
+from paper_2605_08587_b200 import KLA_FLAG_NO_PAIR  # noqa: E402
+
+
+@pytest.mark.parametrize("T", [1, 64, 65, 129, 1000, 2048 + 17])
+def test_independent_ctas_match_oracle_and_paired_launch_bitwise(T):
+    """Both launch forms do the same arithmetic on the same operands: the results must be identical, and the
+    unpaired form is checked against the oracle by itself."""
+    w = W.config3(B=2, H=2, T=T, seed=300 + T)
+    out_u, fin_u = _check_fixed(w, TOL_BF16, flags=KLA_FLAG_NO_PAIR)
+    out_p, fin_p = gpu_chunk(w)
+    assert torch.equal(out_p, out_u)
+    assert torch.equal(fin_p, fin_u)
+
+
+def test_paired_segments_and_packed_input_bitwise():
+    w = W.config3(B=1, H=3, T=1536 + 40, seed=311)
+    o_p, f_p = gpu_chunk(w, flags=KLA_FLAG_SEGMENTS(3))
+    o_u, f_u = gpu_chunk(w, flags=KLA_FLAG_SEGMENTS(3) | KLA_FLAG_NO_PAIR)
+    assert torch.equal(o_p, o_u) and torch.equal(f_p, f_u)
+    wv = W.config5(H=2, d=128, seed=313, lengths=[300, 1, 64, 700, 129])
+    o_p, f_p = gpu_chunk(wv)
+    o_u, f_u = gpu_chunk(wv, flags=KLA_FLAG_NO_PAIR)
+    assert torch.equal(o_p, o_u) and torch.equal(f_p, f_u)

@@ -87,11 +87,15 @@ enum Bar {
     B_D4_DONE = 15,          // P U (and, earlier in the pipe, Q S_0) of chunk c complete
     B_TAIL_READY = 16,       // masked rows of the last chunk zeroed
     B_V_FULL = 17,           // V slice of chunk c landed
-    B_T_FREE = 18,           // paired CTAs: MMA-3(c) of both CTAs complete (the T tiles may be overwritten)
-    B_P_FREE = 19,           // paired CTAs: MMA-4(c) of both CTAs complete
-    B_SCAL_READY0 = 20,      // +(c & 1), paired CTAs: beta, gamma, exp(g_C - g) of chunk c written (long before T(c));
-                             // one barrier per owner, because nothing orders the two owners' arrivals
-    B_COUNT = 22
+    // Paired CTAs.  A wait tells a phase only from its neighbours, and nothing bounds how far one CTA of a pair runs
+    // ahead of the other, so every barrier below is waited on, phase after phase, by one role of one CTA:
+    B_T_FREE0 = 18,          // +(c & 1): MMA-3(c) of both CTAs complete (the T tiles may be overwritten); waited on by
+                             // the owner of chunk c + 1
+    B_P_FREE0 = 20,          // +(c & 1): MMA-4(c) of both CTAs complete; waited on by the owner of chunk c + 1
+    B_SCAL_READY0 = 22,      // +(c & 3): beta, gamma, exp(g_C - g) of chunk c written (long before T(c)).  Four deep: the
+                             // owner sends those of chunk c + 4 only after it has seen MMA-3(c+1) of the peer complete,
+                             // and that chain has then long since waited for those of chunk c
+    B_COUNT = 26
 };
 
 template <int D>
@@ -265,6 +269,7 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     constexpr int SLICES = D / NS;
     constexpr uint32_t STAGE_BYTES = Smem::KQ_BYTES;
     // a pair hands T and P over with one copy per hi/lo pair of tiles
+    static_assert(sizeof(Smem) + 1024 <= 232448, "shared memory of one CTA");
     static_assert(offsetof(Smem, t_lo) == offsetof(Smem, t_hi) + 8192 && offsetof(Smem, p_lo) == offsetof(Smem, p_hi) + 8192, "tile pairs must be contiguous");
     constexpr uint32_t ID_G = idesc_bf16(128, 64, 0, 0);    // [K;Q] K^T : A K-major, B K-major
     constexpr uint32_t ID_S = idesc_bf16(64, NS, 0, 1);     // K S / Q S / T rhs / P U : M=64, B MN-major
@@ -337,10 +342,11 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         mbar_init(&sm.bar[B_D4_DONE], 1);
         mbar_init(&sm.bar[B_TAIL_READY], PG_T / 32);
         mbar_init(&sm.bar[B_V_FULL], 1);
-        mbar_init(&sm.bar[B_T_FREE], 2);
-        mbar_init(&sm.bar[B_P_FREE], 2);
-        mbar_init(&sm.bar[B_SCAL_READY0], 1);
-        mbar_init(&sm.bar[B_SCAL_READY0 + 1], 1);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&sm.bar[B_T_FREE0 + b], 2);
+            mbar_init(&sm.bar[B_P_FREE0 + b], 2);
+        }
+        for (int b = 0; b < 4; ++b) mbar_init(&sm.bar[B_SCAL_READY0 + b], 1);
         sm.abort_flag = 0;
         mbar_fence_init();
     }
@@ -492,8 +498,14 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 if (c + 1 < nchunks) issue_tma_v(c + 1);
                 tc_fence_after();
                 mma_3(tmem + TM_U, d_th, d_tl, d_rh, d_rl);
-                mma_commit(&sm.bar[B_D3_DONE]);
-                mma_commit_multicast(&sm.bar[B_T_FREE], 3);
+                bool signal = true;
+                if constexpr (VAR) signal = !(p.variant & VARIANT_TEST_TIMEOUT);   // test hook: see the unpaired loop
+                if (signal) {
+                    mma_commit(&sm.bar[B_D3_DONE]);
+                    // Only where a later chunk's owner will wait for it: a signal sent for the last chunk could reach
+                    // the peer's SM after that CTA has gone and another block has set up its barriers there.
+                    if (c + 1 < nchunks) mma_commit_multicast(&sm.bar[B_T_FREE0 + (c & 1)], 3);
+                }
                 if (!no_out) mma_xs(tmem + ((c & 1) ? TM_QS1 : TM_QS0), k0, 512);
                 if (m1_due)
                     if (!(ok = mma1_own(cn))) break;
@@ -511,7 +523,7 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     tc_fence_after();
                     mma_3(tmem + TM_PU, d_ph, d_pl, d_rh, d_rl);
                     mma_commit(&sm.bar[B_D4_DONE]);
-                    mma_commit_multicast(&sm.bar[B_P_FREE], 3);
+                    if (c + 1 < nchunks) mma_commit_multicast(&sm.bar[B_P_FREE0 + (c & 1)], 3);   // as for T_FREE
                 }
                 KLA_TR(0, c, 7);
                 // (the chain group, which sees MMA-5(c) complete first, refills the K/Q stage of chunk c)
@@ -700,12 +712,12 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             // period before T(c): their rhs does not wait for the inverse.  (The peer's slot c mod 3 is free: its
             // chain read the scalars of chunk c - 3 before MMA-3(c-3), which this group saw complete two chunks ago.)
             if (pt == 0) {
-                const uint32_t rbar = smem_u32(&sm.bar[B_SCAL_READY0 + (int)rank]) + peer_off;
+                const uint32_t rbar = smem_u32(&sm.bar[B_SCAL_READY0 + (c & 3)]) + peer_off;
                 mbar_arrive_expect_tx_cluster(rbar, 768);
                 bulk_copy_to_cluster(smem_u32(sm.beta[sc]) + peer_off, smem_u32(sm.beta[sc]), 256, rbar);
                 bulk_copy_to_cluster(smem_u32(sm.gam[sc]) + peer_off, smem_u32(sm.gam[sc]), 256, rbar);
                 bulk_copy_to_cluster(smem_u32(sm.dec[sc]) + peer_off, smem_u32(sm.dec[sc]), 256, rbar);
-                mbar_arrive(&sm.bar[B_SCAL_READY0 + (int)rank]);
+                mbar_arrive(&sm.bar[B_SCAL_READY0 + (c & 3)]);
             }
 
             // ---- T = (I + B X)^-1 ----------------------------------------------------------------------------
@@ -738,7 +750,7 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             KLA_TR(1, c, 3);
             // ---- T as bf16 hi/lo operand tiles, once MMA-3(c-1) of both CTAs has read the previous ones ------------
             bool okd = true;
-            if (c > 0 && pt >= PG_T - 32) okd = wait(B_T_FREE, ph ^ 1);
+            if (c > 0 && pt >= PG_T - 32) okd = wait(B_T_FREE0 + ((c - 1) & 1), (uint32_t)(((c - 1) >> 1) & 1));
             if (pg_any(!okd)) break;
             KLA_TR(1, c, 4);
             {
@@ -771,7 +783,8 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             // ---- P(c) = A o Q K^T as bf16 hi/lo operand tiles into both CTAs (rows of Q K^T: warps 2, 3, 6, 7) --------
             if (!is_g && !no_out) {
                 okp = wait(B_D1_DONE0 + b1, ph1);
-                if (okp && c > 0) okp = wait(B_P_FREE, ph ^ 1);   // MMA-4(c-1) of both CTAs has read the P tiles
+                // MMA-4(c-1) of both CTAs has read the P tiles
+                if (okp && c > 0) okp = wait(B_P_FREE0 + ((c - 1) & 1), (uint32_t)(((c - 1) >> 1) & 1));
                 if (okp) {
                     tc_fence_after();
                     const float gi2 = sm.g2[sc][i];
@@ -1091,7 +1104,7 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             const int sc = c % NSTAGE;
             // ---- rhs = B (V - D_gamma K S_0) ------------------------------------------------------------------
             KLA_TR(2, c, 0);
-            if (!(PAIR ? wait(B_SCAL_READY0 + (c & 1), (uint32_t)((c >> 1) & 1)) : wait(B_T_READY, ph))) break;   // scalars of chunk c
+            if (!(PAIR ? wait(B_SCAL_READY0 + (c & 3), (uint32_t)((c >> 2) & 1)) : wait(B_T_READY, ph))) break;   // scalars of chunk c
             KLA_TR(2, c, 1);
             const float b0 = sm.beta[sc][i0], b1 = sm.beta[sc][i1];
             const float g0 = sm.gam[sc][i0], g1 = sm.gam[sc][i1];
@@ -1254,8 +1267,14 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 
     tc_fence_before();
     __syncthreads();
-    // neither CTA of a pair leaves while the other may still write into its shared memory or signal its barriers
-    if constexpr (PAIR) cluster_sync_all();
+    // Neither CTA of a pair leaves while the other may still write into its shared memory or signal its barriers.
+    // On the normal path everything sent has been waited for by its receiver; after a wait gave up, copies and
+    // completion signals issued just before may still be on their way (microseconds): let them land first.
+    if constexpr (PAIR) {
+        if (sm.abort_flag)
+            for (int i = 0; i < 32; ++i) __nanosleep(1000);
+        cluster_sync_all();
+    }
     if (warp == 0) {
         tc_fence_after();
         tmem_dealloc(tmem, TM_COLS);
@@ -1302,11 +1321,16 @@ cudaError_t launch_v(const ChunkParams &p, cudaStream_t stream);
 template <int D, typename OUT>
 cudaError_t launch_t(const ChunkParams &p, cudaStream_t stream)
 {
-    if ((p.variant & ~VARIANT_NO_PAIR) != 0) return launch_v<D, OUT, true, false>(p, stream);
-    // two slices per head: the CTAs of a head run as a cluster and share the state-independent work
-    if constexpr (D == 2 * NS)
-        if (!(p.variant & VARIANT_NO_PAIR)) return launch_v<D, OUT, false, true>(p, stream);
-    return launch_v<D, OUT, false, false>(p, stream);
+    const int32_t v = p.variant & ~VARIANT_NO_PAIR;
+    // two slices per head: the CTAs of a head run as a cluster and share the state-independent work (the layer-edge
+    // variants are implemented in the unpaired kernel only; the error-path test hook in both)
+    if constexpr (D == 2 * NS) {
+        if (!(p.variant & VARIANT_NO_PAIR)) {
+            if (v == 0) return launch_v<D, OUT, false, true>(p, stream);
+            if (v == VARIANT_TEST_TIMEOUT) return launch_v<D, OUT, true, true>(p, stream);
+        }
+    }
+    return v != 0 ? launch_v<D, OUT, true, false>(p, stream) : launch_v<D, OUT, false, false>(p, stream);
 }
 
 template <int D, typename OUT, bool VAR, bool PAIR>

@@ -259,14 +259,15 @@ def test_variants_fp32_and_segments():
 
 
 # ---- the bounded-wait error path (no fault, no hang: a wait runs out by design and the kernel reports it) -------------
-def test_bounded_wait_reports_timeout_and_context_stays_usable():
+@pytest.mark.parametrize("no_pair", [0, 32])   # paired CTAs (a cluster per head) and independent CTAs
+def test_bounded_wait_reports_timeout_and_context_stays_usable(no_pair):
     from paper_2605_08587_b200 import binding
-    w = W.config2(B=1, H=1, T=64, seed=501)
+    w = W.config2(B=1, H=2, T=200, seed=501)
     status = torch.zeros(1, dtype=torch.int32, device="cuda:0")
     dev = "cuda:0"
     a = [t.to(dev) for t in (w.q, w.k, w.v, w.log_alpha, w.eta)]
     from paper_2605_08587_b200 import kla_chunk_fwd
-    kla_chunk_fwd(*a, w.eps, flags=binding.KLA_FLAG_TEST_TIMEOUT, status_word=status)
+    kla_chunk_fwd(*a, w.eps, flags=binding.KLA_FLAG_TEST_TIMEOUT | no_pair, status_word=status)
     torch.cuda.synchronize()                      # returns after about a second: the wait is bounded
     assert int(status.item()) == -10              # KLA_ERR_TIMEOUT
     # the same context then runs the normal path correctly, and an untouched status word stays zero
@@ -302,3 +303,18 @@ def test_paired_segments_and_packed_input_bitwise():
     o_p, f_p = gpu_chunk(wv)
     o_u, f_u = gpu_chunk(wv, flags=KLA_FLAG_NO_PAIR)
     assert torch.equal(o_p, o_u) and torch.equal(f_p, f_u)
+
+
+def test_paired_launch_is_repeatable_over_several_waves():
+    """More clusters than the GPU holds at once, many launches: every launch must reproduce the independent-CTA result
+    bit for bit (a hand-over between the CTAs of a pair that relied on timing would show up here)."""
+    w = W.config2(B=24, H=8, T=640, seed=321)          # 384 CTAs of one CTA per SM
+    o_u, f_u = gpu_chunk(w, flags=KLA_FLAG_NO_PAIR)
+    for _ in range(12):
+        o_p, f_p = gpu_chunk(w)
+        assert torch.equal(o_p, o_u) and torch.equal(f_p, f_u)
+    wl = W.config3()                                    # one long sequence: segment passes of 256 and 144 CTAs
+    o_u, f_u = gpu_chunk(wl, flags=KLA_FLAG_NO_PAIR)
+    for _ in range(12):
+        o_p, f_p = gpu_chunk(wl)
+        assert torch.equal(o_p, o_u) and torch.equal(f_p, f_u)

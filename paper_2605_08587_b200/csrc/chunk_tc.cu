@@ -253,6 +253,138 @@ __device__ __forceinline__ void merge_level(float *tl, float *mm, const float *b
     pg_sync();
 }
 
+// ---- pieces of the pre group's work, shared by the paired and the unpaired form of the group ------------------------------
+// Decay scan of one chunk by one warp (lane l holds log alpha of tokens 2l, 2l + 1): log2(e) g_i, gamma_i = exp(g_i),
+// exp(g_C - g_i) into slot sc.
+template <typename Smem>
+__device__ __forceinline__ void decay_scan(Smem &sm, int sc, int lane, float la0, float la1)
+{
+    float incl = la0 + la1;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const float t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+    }
+    const float gC = __shfl_sync(0xffffffffu, incl, 31);
+    const float a2 = (incl - la1) * LOG2E, b2 = incl * LOG2E, c2 = gC * LOG2E;
+    *reinterpret_cast<float2 *>(&sm.g2[sc][2 * lane]) = make_float2(a2, b2);
+    *reinterpret_cast<float2 *>(&sm.gam[sc][2 * lane]) = make_float2(ex2_approx(a2), ex2_approx(b2));
+    *reinterpret_cast<float2 *>(&sm.dec[sc][2 * lane]) = make_float2(ex2_approx(c2 - a2), ex2_approx(c2 - b2));
+}
+
+// Last chunk: rows past the end of the sequence hold a neighbour's tokens (or TMA zero fill); zero them in the K and
+// Q tiles of the stage so that they are inert in every product.  All PG_T threads of the group.
+template <int KB>
+__device__ __forceinline__ void zero_tail_rows(unsigned char *kq, int rows, int pt)
+{
+    for (int e = pt; e < (C - rows) * 8; e += PG_T) {
+        const int r = rows + e / 8, ch = e % 8;
+        const uint4 z = make_uint4(0, 0, 0, 0);
+#pragma unroll
+        for (int kb = 0; kb < KB; ++kb) {
+            *reinterpret_cast<uint4 *>(kq + kb * 16384 + sw128(r, ch)) = z;
+            *reinterpret_cast<uint4 *>(kq + kb * 16384 + 8192 + sw128(r, ch)) = z;
+        }
+    }
+}
+
+// X = A^- o K K^T: this thread's row i, columns chh * 32 .. + 31 of the MMA-1 accumulator at tbase, into the solve
+// matrix.  Returns the diagonal element G_ii = ||k_i||^2 if it lies in these columns (else 0).
+template <typename Smem>
+__device__ __forceinline__ float form_x_row(Smem &sm, int sc, int i, int chh, uint32_t tbase)
+{
+    const float gi2 = sm.g2[sc][i];
+    float dg = 0.f;
+#pragma unroll 1
+    for (int grp = 0; grp < 4; ++grp) {
+        float a[8];
+        tmem_ld8(tbase + grp * 8, a);
+        const int j0 = chh * 32 + grp * 8;
+        const float4 ga = *reinterpret_cast<const float4 *>(&sm.g2[sc][j0]);
+        const float4 gb = *reinterpret_cast<const float4 *>(&sm.g2[sc][j0 + 4]);
+        const float gj[8] = {ga.x, ga.y, ga.z, ga.w, gb.x, gb.y, gb.z, gb.w};
+        float x[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            x[e] = (j0 + e < i) ? ex2_approx(gi2 - gj[e]) * a[e] : 0.f;
+            dg = (j0 + e == i) ? a[e] : dg;
+        }
+        *reinterpret_cast<float4 *>(&sm.tl[i * LDT + j0]) = make_float4(x[0], x[1], x[2], x[3]);
+        *reinterpret_cast<float4 *>(&sm.tl[i * LDT + j0 + 4]) = make_float4(x[4], x[5], x[6], x[7]);
+    }
+    return dg;
+}
+
+// P = A o Q K^T: this thread's row i, columns chh * 32 .. + 31 of the MMA-1 accumulator at tbase, as bf16 hi/lo operand
+// tiles (zeros where `live` is false: all 32 columns above the diagonal).
+template <typename Smem>
+__device__ __forceinline__ void form_p_row(Smem &sm, int sc, int i, int chh, bool live, uint32_t tbase)
+{
+    const float gi2 = sm.g2[sc][i];
+#pragma unroll 1
+    for (int grp = 0; grp < 4; ++grp) {
+        uint4 hi = make_uint4(0, 0, 0, 0), lo = hi;
+        if (live) {
+            float a[8];
+            tmem_ld8(tbase + grp * 8, a);
+            const int j0 = chh * 32 + grp * 8;
+            const float4 ga = *reinterpret_cast<const float4 *>(&sm.g2[sc][j0]);
+            const float4 gb = *reinterpret_cast<const float4 *>(&sm.g2[sc][j0 + 4]);
+            const float gj[8] = {ga.x, ga.y, ga.z, ga.w, gb.x, gb.y, gb.z, gb.w};
+            float x[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) x[e] = (j0 + e <= i) ? ex2_approx(gi2 - gj[e]) * a[e] : 0.f;
+            split2(x[0], x[1], hi.x, lo.x);
+            split2(x[2], x[3], hi.y, lo.y);
+            split2(x[4], x[5], hi.z, lo.z);
+            split2(x[6], x[7], hi.w, lo.w);
+        }
+        *reinterpret_cast<uint4 *>(sm.p_hi + sw128(i, chh * 4 + grp)) = hi;
+        *reinterpret_cast<uint4 *>(sm.p_lo + sw128(i, chh * 4 + grp)) = lo;
+    }
+}
+
+// 8 x 8 diagonal blocks of T = (I + B X)^-1 by substitution: thread pt < 64 solves column pt % 8 of block pt / 8 in
+// registers, then the block's eight threads write their columns over X_bb.
+__device__ __forceinline__ void substitute_diag_blocks(float *tl, const float *bet, int pt)
+{
+    const int blk = pt >> 3, j = pt & 7;
+    float *Lb = tl + (blk * 8) * LDT + blk * 8;
+    float x[8];
+#pragma unroll
+    for (int r = 0; r < 8; ++r) {
+        const float4 l0 = *reinterpret_cast<const float4 *>(Lb + r * LDT);
+        const float4 l1 = *reinterpret_cast<const float4 *>(Lb + r * LDT + 4);
+        const float l[8] = {l0.x, l0.y, l0.z, l0.w, l1.x, l1.y, l1.z, l1.w};
+        float s = 0.f;
+#pragma unroll
+        for (int m = 0; m < r; ++m) s += l[m] * x[m];
+        x[r] = (r == j) ? 1.f : ((r > j) ? -bet[blk * 8 + r] * s : 0.f);
+    }
+    half_sync();  // every column of the block has read X_bb
+#pragma unroll
+    for (int r = 0; r < 8; ++r) Lb[r * LDT + j] = x[r];
+}
+
+// T (fp32, in the solve matrix) as bf16 hi/lo operand tiles: thread pt writes 16 columns of row pt % 64.
+template <typename Smem>
+__device__ __forceinline__ void write_t_tiles(Smem &sm, int pt)
+{
+    const int r = pt & 63, qq = pt >> 6;  // row, 16-column quarter
+#pragma unroll 1
+    for (int ch = 0; ch < 2; ++ch) {
+        const float4 a = *reinterpret_cast<const float4 *>(&sm.tl[r * LDT + qq * 16 + ch * 8]);
+        const float4 b = *reinterpret_cast<const float4 *>(&sm.tl[r * LDT + qq * 16 + ch * 8 + 4]);
+        uint4 hi, lo;
+        split2(a.x, a.y, hi.x, lo.x);
+        split2(a.z, a.w, hi.y, lo.y);
+        split2(b.x, b.y, hi.z, lo.z);
+        split2(b.z, b.w, hi.w, lo.w);
+        *reinterpret_cast<uint4 *>(sm.t_hi + sw128(r, qq * 2 + ch)) = hi;
+        *reinterpret_cast<uint4 *>(sm.t_lo + sw128(r, qq * 2 + ch)) = lo;
+    }
+}
+
 // VAR: compiled with the layer-edge variants (beta = eta, read-out over ||q||); the default instantiation carries
 // none of their code.
 // PAIR: the two CTAs that hold the two column slices of one (sequence, head) run as a thread-block cluster and
@@ -629,17 +761,7 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             const float la0 = la_next0, la1 = la_next1, eta_cur = eta_next;
             if (own && c + 2 < nchunks) fetch_gates(c + 2);
             if (own && scan_warp) {
-                float incl = la0 + la1;
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    const float t = __shfl_up_sync(0xffffffffu, incl, o);
-                    if (lane >= o) incl += t;
-                }
-                const float gC = __shfl_sync(0xffffffffu, incl, 31);
-                const float a2 = (incl - la1) * LOG2E, b2 = incl * LOG2E, c2 = gC * LOG2E;
-                *reinterpret_cast<float2 *>(&sm.g2[sc][2 * lane]) = make_float2(a2, b2);
-                *reinterpret_cast<float2 *>(&sm.gam[sc][2 * lane]) = make_float2(ex2_approx(a2), ex2_approx(b2));
-                *reinterpret_cast<float2 *>(&sm.dec[sc][2 * lane]) = make_float2(ex2_approx(c2 - a2), ex2_approx(c2 - b2));
+                decay_scan(sm, sc, lane, la0, la1);
                 fence_async_smem();   // gam and dec are also copied to the peer
             }
             KLA_TR(1, c, 0);
@@ -647,16 +769,7 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             if (rows < C && okc) {
                 okc = wait(B_FULL0 + sc, (uint32_t)((c / NSTAGE) & 1));
                 if (okc) {
-                    unsigned char *kq = sm.kq[sc];
-                    for (int e = pt; e < (C - rows) * 8; e += PG_T) {
-                        const int r = rows + e / 8, ch = e % 8;
-                        const uint4 z = make_uint4(0, 0, 0, 0);
-#pragma unroll
-                        for (int kb = 0; kb < KB; ++kb) {
-                            *reinterpret_cast<uint4 *>(kq + kb * 16384 + sw128(r, ch)) = z;
-                            *reinterpret_cast<uint4 *>(kq + kb * 16384 + 8192 + sw128(r, ch)) = z;
-                        }
-                    }
+                    zero_tail_rows<KB>(sm.kq[sc], rows, pt);
                     fence_async_smem();
                     warp_arrive(B_TAIL_READY);
                 }
@@ -674,26 +787,8 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 if (okc) {
                     tc_fence_after();
                     if (live) {
-                        const float gi2 = sm.g2[sc][i];
-                        float dg = 0.f;   // G_ii = ||k_i||^2
-                        const uint32_t tbase = tm_lane + TM_D1 + (uint32_t)b1 * 64 + chh * 32;
-#pragma unroll 1
-                        for (int grp = 0; grp < 4; ++grp) {
-                            float a[8];
-                            tmem_ld8(tbase + grp * 8, a);
-                            const int j0 = chh * 32 + grp * 8;
-                            const float4 ga = *reinterpret_cast<const float4 *>(&sm.g2[sc][j0]);
-                            const float4 gb = *reinterpret_cast<const float4 *>(&sm.g2[sc][j0 + 4]);
-                            const float gj[8] = {ga.x, ga.y, ga.z, ga.w, gb.x, gb.y, gb.z, gb.w};
-                            float x[8];
-#pragma unroll
-                            for (int e = 0; e < 8; ++e) {
-                                x[e] = (j0 + e < i) ? ex2_approx(gi2 - gj[e]) * a[e] : 0.f;
-                                dg = (j0 + e == i) ? a[e] : dg;
-                            }
-                            *reinterpret_cast<float4 *>(&sm.tl[i * LDT + j0]) = make_float4(x[0], x[1], x[2], x[3]);
-                            *reinterpret_cast<float4 *>(&sm.tl[i * LDT + j0 + 4]) = make_float4(x[4], x[5], x[6], x[7]);
-                        }
+                        // G_ii = ||k_i||^2 comes with the row
+                        const float dg = form_x_row(sm, sc, i, chh, tm_lane + TM_D1 + (uint32_t)b1 * 64 + chh * 32);
                         if (chh == q) {
                             sm.beta[sc][i] = (i < rows) ? eta_cur / (dg + p.eps) : 0.f;
                             fence_async_smem();
@@ -722,24 +817,7 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 
             // ---- T = (I + B X)^-1 ----------------------------------------------------------------------------
             const float *bet = sm.beta[sc];
-            if (pt < 64) {
-                const int blk = pt >> 3, j = pt & 7;
-                float *Lb = sm.tl + (blk * 8) * LDT + blk * 8;
-                float x[8];
-#pragma unroll
-                for (int r = 0; r < 8; ++r) {
-                    const float4 l0 = *reinterpret_cast<const float4 *>(Lb + r * LDT);
-                    const float4 l1 = *reinterpret_cast<const float4 *>(Lb + r * LDT + 4);
-                    const float l[8] = {l0.x, l0.y, l0.z, l0.w, l1.x, l1.y, l1.z, l1.w};
-                    float s = 0.f;
-#pragma unroll
-                    for (int m = 0; m < r; ++m) s += l[m] * x[m];
-                    x[r] = (r == j) ? 1.f : ((r > j) ? -bet[blk * 8 + r] * s : 0.f);
-                }
-                half_sync();
-#pragma unroll
-                for (int r = 0; r < 8; ++r) Lb[r * LDT + j] = x[r];
-            }
+            if (pt < 64) substitute_diag_blocks(sm.tl, bet, pt);
             pg_sync();
             KLA_TR(1, c, 2);
             merge_level<8>(sm.tl, sm.mm, bet, pt);
@@ -753,22 +831,7 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             if (c > 0 && pt >= PG_T - 32) okd = wait(B_T_FREE0 + ((c - 1) & 1), (uint32_t)(((c - 1) >> 1) & 1));
             if (pg_any(!okd)) break;
             KLA_TR(1, c, 4);
-            {
-                const int r = pt & 63, qq = pt >> 6;
-#pragma unroll 1
-                for (int ch = 0; ch < 2; ++ch) {
-                    const float4 a = *reinterpret_cast<const float4 *>(&sm.tl[r * LDT + qq * 16 + ch * 8]);
-                    const float4 b = *reinterpret_cast<const float4 *>(&sm.tl[r * LDT + qq * 16 + ch * 8 + 4]);
-                    uint4 hi, lo;
-                    split2(a.x, a.y, hi.x, lo.x);
-                    split2(a.z, a.w, hi.y, lo.y);
-                    split2(b.x, b.y, hi.z, lo.z);
-                    split2(b.z, b.w, hi.w, lo.w);
-                    const uint32_t o = sw128(r, qq * 2 + ch);
-                    *reinterpret_cast<uint4 *>(sm.t_hi + o) = hi;
-                    *reinterpret_cast<uint4 *>(sm.t_lo + o) = lo;
-                }
-            }
+            write_t_tiles(sm, pt);
             fence_async_smem();
             pg_sync();  // every tile write is done (and the solve matrix may be reused by this CTA's next chunk)
             if (pt == 0) {
@@ -787,30 +850,7 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 if (okp && c > 0) okp = wait(B_P_FREE0 + ((c - 1) & 1), (uint32_t)(((c - 1) >> 1) & 1));
                 if (okp) {
                     tc_fence_after();
-                    const float gi2 = sm.g2[sc][i];
-                    const uint32_t tbase = tm_lane + TM_D1 + (uint32_t)b1 * 64 + chh * 32;
-#pragma unroll 1
-                    for (int grp = 0; grp < 4; ++grp) {
-                        uint4 hi = make_uint4(0, 0, 0, 0), lo = hi;
-                        if (live) {
-                            float a[8];
-                            tmem_ld8(tbase + grp * 8, a);
-                            const int j0 = chh * 32 + grp * 8;
-                            const float4 ga = *reinterpret_cast<const float4 *>(&sm.g2[sc][j0]);
-                            const float4 gb = *reinterpret_cast<const float4 *>(&sm.g2[sc][j0 + 4]);
-                            const float gj[8] = {ga.x, ga.y, ga.z, ga.w, gb.x, gb.y, gb.z, gb.w};
-                            float x[8];
-#pragma unroll
-                            for (int e = 0; e < 8; ++e) x[e] = (j0 + e <= i) ? ex2_approx(gi2 - gj[e]) * a[e] : 0.f;
-                            split2(x[0], x[1], hi.x, lo.x);
-                            split2(x[2], x[3], hi.y, lo.y);
-                            split2(x[4], x[5], hi.z, lo.z);
-                            split2(x[6], x[7], hi.w, lo.w);
-                        }
-                        const uint32_t o = sw128(i, chh * 4 + grp);
-                        *reinterpret_cast<uint4 *>(sm.p_hi + o) = hi;
-                        *reinterpret_cast<uint4 *>(sm.p_lo + o) = lo;
-                    }
+                    form_p_row(sm, sc, i, chh, live, tm_lane + TM_D1 + (uint32_t)b1 * 64 + chh * 32);
                     tc_fence_before();
                     fence_async_smem();
                     warp_arrive(B_D1_FREE0 + b1);
@@ -856,29 +896,7 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             if (!okp) return false;
             tc_fence_after();
             const int sc = c % NSTAGE;
-            const float gi2 = sm.g2[sc][i];
-            const uint32_t tbase = tm_lane + TM_D1 + (uint32_t)(c & 1) * 64 + chh * 32;
-#pragma unroll 1
-            for (int grp = 0; grp < 4; ++grp) {
-                uint4 hi = make_uint4(0, 0, 0, 0), lo = hi;
-                if (live) {
-                    float a[8];
-                    tmem_ld8(tbase + grp * 8, a);
-                    const int j0 = chh * 32 + grp * 8;
-                    const float4 ga = *reinterpret_cast<const float4 *>(&sm.g2[sc][j0]);
-                    const float4 gb = *reinterpret_cast<const float4 *>(&sm.g2[sc][j0 + 4]);
-                    const float gj[8] = {ga.x, ga.y, ga.z, ga.w, gb.x, gb.y, gb.z, gb.w};
-                    float x[8];
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) x[e] = (j0 + e <= i) ? ex2_approx(gi2 - gj[e]) * a[e] : 0.f;
-                    split2(x[0], x[1], hi.x, lo.x);
-                    split2(x[2], x[3], hi.y, lo.y);
-                    split2(x[4], x[5], hi.z, lo.z);
-                    split2(x[6], x[7], hi.w, lo.w);
-                }
-                *reinterpret_cast<uint4 *>(sm.p_hi + sw128(i, chh * 4 + grp)) = hi;
-                *reinterpret_cast<uint4 *>(sm.p_lo + sw128(i, chh * 4 + grp)) = lo;
-            }
+            form_p_row(sm, sc, i, chh, live, tm_lane + TM_D1 + (uint32_t)(c & 1) * 64 + chh * 32);
             if constexpr (VAR) if ((p.variant & VARIANT_QNORM) && chh == 0) {
                 // ||q_i||^2 from row i of the Q tile (still resident: its stage is refilled only after MMA-4(c))
                 const unsigned char *qt = sm.kq[sc];
@@ -911,17 +929,7 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             if (c + 1 < nchunks) fetch_gates(c + 1);
             // ---- g_i (chunk-local running sum of log alpha), gamma_i, exp(g_C - g_i) -----------------------------
             if (scan_warp) {
-                float incl = la0 + la1;
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    const float t = __shfl_up_sync(0xffffffffu, incl, o);
-                    if (lane >= o) incl += t;
-                }
-                const float gC = __shfl_sync(0xffffffffu, incl, 31);
-                const float a2 = (incl - la1) * LOG2E, b2 = incl * LOG2E, c2 = gC * LOG2E;
-                *reinterpret_cast<float2 *>(&sm.g2[sc][2 * lane]) = make_float2(a2, b2);
-                *reinterpret_cast<float2 *>(&sm.gam[sc][2 * lane]) = make_float2(ex2_approx(a2), ex2_approx(b2));
-                *reinterpret_cast<float2 *>(&sm.dec[sc][2 * lane]) = make_float2(ex2_approx(c2 - a2), ex2_approx(c2 - b2));
+                decay_scan(sm, sc, lane, la0, la1);
             }
             KLA_TR(1, c, 0);
             bool okc = true;
@@ -930,16 +938,7 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 // fill); zero them so that they are inert in every product
                 okc = wait(B_FULL0 + sc, (uint32_t)((c / NSTAGE) & 1));
                 if (okc) {
-                    unsigned char *kq = sm.kq[sc];
-                    for (int e = pt; e < (C - rows) * 8; e += PG_T) {
-                        const int r = rows + e / 8, ch = e % 8;
-                        const uint4 z = make_uint4(0, 0, 0, 0);
-#pragma unroll
-                        for (int kb = 0; kb < KB; ++kb) {
-                            *reinterpret_cast<uint4 *>(kq + kb * 16384 + sw128(r, ch)) = z;
-                            *reinterpret_cast<uint4 *>(kq + kb * 16384 + 8192 + sw128(r, ch)) = z;
-                        }
-                    }
+                    zero_tail_rows<KB>(sm.kq[sc], rows, pt);
                     fence_async_smem();
                     warp_arrive(B_TAIL_READY);
                 }
@@ -953,26 +952,8 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 if (okc) {
                     tc_fence_after();
                     if (live) {
-                        const float gi2 = sm.g2[sc][i];
-                        float dg = 0.f;   // G_ii = ||k_i||^2
-                        const uint32_t tbase = tm_lane + TM_D1 + (uint32_t)(c & 1) * 64 + chh * 32;
-#pragma unroll 1
-                        for (int grp = 0; grp < 4; ++grp) {
-                            float a[8];
-                            tmem_ld8(tbase + grp * 8, a);
-                            const int j0 = chh * 32 + grp * 8;
-                            const float4 ga = *reinterpret_cast<const float4 *>(&sm.g2[sc][j0]);
-                            const float4 gb = *reinterpret_cast<const float4 *>(&sm.g2[sc][j0 + 4]);
-                            const float gj[8] = {ga.x, ga.y, ga.z, ga.w, gb.x, gb.y, gb.z, gb.w};
-                            float x[8];
-#pragma unroll
-                            for (int e = 0; e < 8; ++e) {
-                                x[e] = (j0 + e < i) ? ex2_approx(gi2 - gj[e]) * a[e] : 0.f;
-                                dg = (j0 + e == i) ? a[e] : dg;
-                            }
-                            *reinterpret_cast<float4 *>(&sm.tl[i * LDT + j0]) = make_float4(x[0], x[1], x[2], x[3]);
-                            *reinterpret_cast<float4 *>(&sm.tl[i * LDT + j0 + 4]) = make_float4(x[4], x[5], x[6], x[7]);
-                        }
+                        // G_ii = ||k_i||^2 comes with the row
+                        const float dg = form_x_row(sm, sc, i, chh, tm_lane + TM_D1 + (uint32_t)(c & 1) * 64 + chh * 32);
                         // beta_i = eta_i / (||k_i||^2 + eps), Eq. 3; rows past the end of the sequence get 0
                         if (chh == q) {
                             if constexpr (VAR) sm.beta[sc][i] = (i < rows) ? ((p.variant & VARIANT_COEFF_ETA) ? eta_cur : eta_cur / (dg + p.eps)) : 0.f;
@@ -994,24 +975,7 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             // ---- T = (I + B X)^-1: 8x8 diagonal blocks by substitution, then the off-diagonal blocks
             //      T_10 = -T_11 (B_1 X_10 T_00) at block sizes 8, 16, 32 -----------------------------------------------
             const float *bet = sm.beta[sc];
-            if (pt < 64) {
-                const int blk = pt >> 3, j = pt & 7;
-                float *Lb = sm.tl + (blk * 8) * LDT + blk * 8;
-                float x[8];
-#pragma unroll
-                for (int r = 0; r < 8; ++r) {
-                    const float4 l0 = *reinterpret_cast<const float4 *>(Lb + r * LDT);
-                    const float4 l1 = *reinterpret_cast<const float4 *>(Lb + r * LDT + 4);
-                    const float l[8] = {l0.x, l0.y, l0.z, l0.w, l1.x, l1.y, l1.z, l1.w};
-                    float s = 0.f;
-#pragma unroll
-                    for (int m = 0; m < r; ++m) s += l[m] * x[m];
-                    x[r] = (r == j) ? 1.f : ((r > j) ? -bet[blk * 8 + r] * s : 0.f);
-                }
-                half_sync();  // every column of the block has read X_bb
-#pragma unroll
-                for (int r = 0; r < 8; ++r) Lb[r * LDT + j] = x[r];
-            }
+            if (pt < 64) substitute_diag_blocks(sm.tl, bet, pt);
             // Meanwhile a warp with nothing to substitute takes the wait that guards the T tiles (MMA-3(c-1) must have
             // read the previous ones): the first look at a barrier completed by the tensor pipe costs several hundred
             // cycles wherever it is taken, so it is taken here, under the substitution.
@@ -1027,21 +991,7 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             // ---- write T as bf16 hi/lo operand tiles, after MMA-3(c-1) has read the previous ones ----------------------
             KLA_TR(1, c, 3);
             KLA_TR(1, c, 4);
-            {
-                const int r = pt & 63, qq = pt >> 6;  // row, 16-column quarter
-#pragma unroll 1
-                for (int ch = 0; ch < 2; ++ch) {
-                    const float4 a = *reinterpret_cast<const float4 *>(&sm.tl[r * LDT + qq * 16 + ch * 8]);
-                    const float4 b = *reinterpret_cast<const float4 *>(&sm.tl[r * LDT + qq * 16 + ch * 8 + 4]);
-                    uint4 hi, lo;
-                    split2(a.x, a.y, hi.x, lo.x);
-                    split2(a.z, a.w, hi.y, lo.y);
-                    split2(b.x, b.y, hi.z, lo.z);
-                    split2(b.z, b.w, hi.w, lo.w);
-                    *reinterpret_cast<uint4 *>(sm.t_hi + sw128(r, qq * 2 + ch)) = hi;
-                    *reinterpret_cast<uint4 *>(sm.t_lo + sw128(r, qq * 2 + ch)) = lo;
-                }
-            }
+            write_t_tiles(sm, pt);
             fence_async_smem();
             pg_sync();  // the solve matrix is reused by the next chunk
             warp_arrive(B_T_READY);

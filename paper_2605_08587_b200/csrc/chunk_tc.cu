@@ -627,7 +627,6 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 KLA_TR(0, c, 3);
                 if (!(ok = wwait(B_RHS_READY, ph))) break;
                 KLA_TR(0, c, 4);
-                if (c + 1 < nchunks) issue_tma_v(c + 1);
                 tc_fence_after();
                 mma_3(tmem + TM_U, d_th, d_tl, d_rh, d_rl);
                 bool signal = true;
@@ -638,6 +637,7 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     // the peer's SM after that CTA has gone and another block has set up its barriers there.
                     if (c + 1 < nchunks) mma_commit_multicast(&sm.bar[B_T_FREE0 + (c & 1)], 3);
                 }
+                if (c + 1 < nchunks) issue_tma_v(c + 1);   // every chain warp has posted rhs(c): the V buffer is free
                 if (!no_out) mma_xs(tmem + ((c & 1) ? TM_QS1 : TM_QS0), k0, 512);
                 if (m1_due)
                     if (!(ok = mma1_own(cn))) break;

@@ -23,7 +23,7 @@
 //   MMA-1  [K;Q] K^T   M=128   -> K K^T (lanes 0..63) and Q K^T (lanes 64..127), double-buffered
 //   MMA-2  K S_0, Q S_0        two M=64 products, S_0 = S_hi + S_lo
 //   MMA-3  T rhs       M=64    T_hi rhs_hi + T_hi rhs_lo + T_lo rhs_hi
-//   MMA-4  P U         M=64    same three-term form
+//   MMA-4  P U         M=64    same three-term form, taken as (P D^-1)(D U) so that the chain forms D U only
 //   MMA-5  K^T (D U)   M=128   D U = hi + lo
 //
 // Precision.  q, k, v are exact bf16 operands.  Every DERIVED operand (S_0, rhs, T, P, U, D U) is
@@ -64,6 +64,10 @@ constexpr int CG_BASE = 32, PG_BASE = 32 + CG_T;
 constexpr int NSTAGE = 3;
 constexpr long long WAIT_LIMIT = 2000000000LL;  // SM clocks (~1 s) before a wait gives up
 constexpr float LOG2E = 1.4426950408889634f;
+// The write weights exp(g_C - g_j) are kept above 2^-DEC_FLOOR_LOG2 (~1e-35): the output product is taken as
+// (P D^-1)(D U), and with the floor neither factor leaves the fp32 / bf16 exponent range however strong the decay.  A
+// floored weight puts at most 1e-35 of a token into the state instead of less.
+constexpr float DEC_FLOOR_LOG2 = 115.f;
 
 // TMEM columns (fp32, 128 lanes each)
 constexpr uint32_t TM_D1 = 0 /* two buffers of 64 */, TM_KS = 128, TM_QS0 = 192, TM_QS1 = 256, TM_U = 320, TM_PU = 384,
@@ -110,9 +114,9 @@ struct TcSmem {
     alignas(1024) unsigned char t_lo[8192];
     alignas(1024) unsigned char p_hi[8192];
     alignas(1024) unsigned char p_lo[8192];
-    alignas(1024) unsigned char ru_hi[8192];    // rhs, later U: 64 tokens x 64 bf16, MN-major
+    alignas(1024) unsigned char ru_hi[8192];    // rhs: 64 tokens x 64 bf16, MN-major
     alignas(1024) unsigned char ru_lo[8192];
-    alignas(1024) unsigned char du_hi[8192];    // diag(exp(g_C - g_j)) U
+    alignas(1024) unsigned char du_hi[8192];    // D U, D = diag(exp(g_C - g_j)): operand of MMA-5 and of MMA-4
     alignas(1024) unsigned char du_lo[8192];
     alignas(1024) unsigned char vt[8192];       // V slice of one chunk: 64 tokens x 64 bf16, same layout as ru_*
     alignas(16) float tl[64 * LDT];             // X = A^- o K K^T, overwritten in place by T = (I + B X)^-1
@@ -255,7 +259,7 @@ __device__ __forceinline__ void merge_level(float *tl, float *mm, const float *b
 
 // ---- pieces of the pre group's work, shared by the paired and the unpaired form of the group ------------------------------
 // Decay scan of one chunk by one warp (lane l holds log alpha of tokens 2l, 2l + 1): log2(e) g_i, gamma_i = exp(g_i),
-// exp(g_C - g_i) into slot sc.
+// d_i = exp(g_C - g_i) (floored, see DEC_FLOOR_LOG2) into slot sc.
 template <typename Smem>
 __device__ __forceinline__ void decay_scan(Smem &sm, int sc, int lane, float la0, float la1)
 {
@@ -269,7 +273,8 @@ __device__ __forceinline__ void decay_scan(Smem &sm, int sc, int lane, float la0
     const float a2 = (incl - la1) * LOG2E, b2 = incl * LOG2E, c2 = gC * LOG2E;
     *reinterpret_cast<float2 *>(&sm.g2[sc][2 * lane]) = make_float2(a2, b2);
     *reinterpret_cast<float2 *>(&sm.gam[sc][2 * lane]) = make_float2(ex2_approx(a2), ex2_approx(b2));
-    *reinterpret_cast<float2 *>(&sm.dec[sc][2 * lane]) = make_float2(ex2_approx(c2 - a2), ex2_approx(c2 - b2));
+    *reinterpret_cast<float2 *>(&sm.dec[sc][2 * lane]) =
+        make_float2(ex2_approx(fmaxf(c2 - a2, -DEC_FLOOR_LOG2)), ex2_approx(fmaxf(c2 - b2, -DEC_FLOOR_LOG2)));
 }
 
 // Last chunk: rows past the end of the sequence hold a neighbour's tokens (or TMA zero fill); zero them in the K and
@@ -315,12 +320,15 @@ __device__ __forceinline__ float form_x_row(Smem &sm, int sc, int i, int chh, ui
     return dg;
 }
 
-// P = A o Q K^T: this thread's row i, columns chh * 32 .. + 31 of the MMA-1 accumulator at tbase, as bf16 hi/lo operand
-// tiles (zeros where `live` is false: all 32 columns above the diagonal).
+// P D^-1 with P = A o Q K^T and D = diag(d_j), d_j the (floored) write weights of the decay scan: the chain forms D U
+// only (the operand of the state update), and the outputs use P U = (P D^-1)(D U).  Element (i, j <= i) is
+// exp(g_i - g_j) / d_j = 2^(g2_i - max(g2_C, g2_j - DEC_FLOOR_LOG2)), at most 2^DEC_FLOOR_LOG2.  This thread's row i,
+// columns chh * 32 .. + 31 of the MMA-1 accumulator at tbase, as bf16 hi/lo operand tiles (zeros where `live` is false:
+// all 32 columns above the diagonal).
 template <typename Smem>
 __device__ __forceinline__ void form_p_row(Smem &sm, int sc, int i, int chh, bool live, uint32_t tbase)
 {
-    const float gi2 = sm.g2[sc][i];
+    const float gi2 = sm.g2[sc][i], gc2 = sm.g2[sc][C - 1];
 #pragma unroll 1
     for (int grp = 0; grp < 4; ++grp) {
         uint4 hi = make_uint4(0, 0, 0, 0), lo = hi;
@@ -333,7 +341,8 @@ __device__ __forceinline__ void form_p_row(Smem &sm, int sc, int i, int chh, boo
             const float gj[8] = {ga.x, ga.y, ga.z, ga.w, gb.x, gb.y, gb.z, gb.w};
             float x[8];
 #pragma unroll
-            for (int e = 0; e < 8; ++e) x[e] = (j0 + e <= i) ? ex2_approx(gi2 - gj[e]) * a[e] : 0.f;
+            for (int e = 0; e < 8; ++e)
+                x[e] = (j0 + e <= i) ? ex2_approx(gi2 - fmaxf(gc2, gj[e] - DEC_FLOOR_LOG2)) * a[e] : 0.f;
             split2(x[0], x[1], hi.x, lo.x);
             split2(x[2], x[3], hi.y, lo.y);
             split2(x[4], x[5], hi.z, lo.z);
@@ -568,9 +577,10 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             return true;
         };
         // [K or Q](c) S_0 -> d; qoff = 512 selects the Q tile of a block; S_0 = S_hi + S_lo
-        auto mma_xs = [&](uint32_t d, uint32_t k0, uint32_t qoff) {
+        // (blocks t0 .. t1 - 1 of the 2 KB four-MMA blocks: the S_hi term first, then the S_lo term)
+        auto mma_xs = [&](uint32_t d, uint32_t k0, uint32_t qoff, int t0 = 0, int t1 = 2 * KB) {
 #pragma unroll 1
-            for (int t = 0; t < 2 * KB; ++t) {
+            for (int t = t0; t < t1; ++t) {
                 const uint32_t kb = (uint32_t)t & (KB - 1);
                 KLA_SEQ(d, k0 + qoff + kb * 1024, 2, (t >= KB ? d_sl : d_sh) + kb * 512, 128, ID_S, t > 0);
             }
@@ -586,11 +596,11 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         if constexpr (PAIR) {
             // ---- paired CTAs.  The tensor pipe runs the MMAs in issue order at ~60 cycles each, so what is not on the
             // chain goes where the pipe would idle and can finish before the chain's next product is ready:
-            //   K S_0(c) | MMA-1 of this CTA's chunk c + 2 (if its tiles have landed)     while the chain forms rhs(c)
-            //   MMA-3(c) | Q S_0(c) (| MMA-1 if not issued above)                          while the chain forms U(c)
+            //   K S_0(c) | MMA-1 of this CTA's chunk c + 2 (if due and landed), else half of Q S_0(c)   while rhs(c) forms
+            //   MMA-3(c) | the rest of Q S_0(c) (| MMA-1 if due and not issued above)                   while D U(c) forms
             //   MMA-5(c) | MMA-4(c)                                                        while the chain updates S
             // Order constraints: Q S_0(c) before MMA-5(c), whose completion lets the chain overwrite the S tiles;
-            // MMA-4(c) before K S_0(c+1), whose completion lets it overwrite U.
+            // MMA-4(c) before MMA-3(c+1), whose completion lets it overwrite D U.
             auto ready = [&](int b, uint32_t parity) -> bool {
                 return __all_sync(0xffffffffu, mbar_test_wait(&sm.bar[b], parity));
             };
@@ -614,12 +624,17 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 mma_commit(&sm.bar[B_D2_DONE]);
                 const int cn = c + 2;   // this CTA's next chunk
                 bool m1_due = own && cn < nchunks;
+                int qs_done = no_out ? 2 * KB : 0;   // blocks of Q S_0 issued so far
                 if (m1_due && ready(B_FULL0 + cn % NSTAGE, (uint32_t)((cn / NSTAGE) & 1)) &&
                     (!(cn + 1 == nchunks && last_rows < C) || ready(B_TAIL_READY, 0)) &&
                     (cn < 4 || ready(B_D1_FREE0 + ((cn >> 1) & 1), (uint32_t)(((cn >> 2) - 1) & 1)))) {
                     tc_fence_after();
                     mma1(cn);
                     m1_due = false;
+                } else if (!no_out) {
+                    // no MMA-1 in this window: the S_hi term of Q S_0 fits here instead
+                    mma_xs(tmem + ((c & 1) ? TM_QS1 : TM_QS0), k0, 512, 0, KB);
+                    qs_done = KB;
                 }
                 KLA_TR(0, c, 2);
                 // MMA-3(c): U = T rhs
@@ -638,7 +653,7 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     if (c + 1 < nchunks) mma_commit_multicast(&sm.bar[B_T_FREE0 + (c & 1)], 3);
                 }
                 if (c + 1 < nchunks) issue_tma_v(c + 1);   // every chain warp has posted rhs(c): the V buffer is free
-                if (!no_out) mma_xs(tmem + ((c & 1) ? TM_QS1 : TM_QS0), k0, 512);
+                if (qs_done < 2 * KB) mma_xs(tmem + ((c & 1) ? TM_QS1 : TM_QS0), k0, 512, qs_done, 2 * KB);
                 if (m1_due)
                     if (!(ok = mma1_own(cn))) break;
                 KLA_TR(0, c, 5);
@@ -653,7 +668,7 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 if (!no_out) {
                     if (!(ok = wwait(B_P_READY, ph))) break;
                     tc_fence_after();
-                    mma_3(tmem + TM_PU, d_ph, d_pl, d_rh, d_rl);
+                    mma_3(tmem + TM_PU, d_ph, d_pl, d_dh, d_dl);
                     mma_commit(&sm.bar[B_D4_DONE]);
                     if (c + 1 < nchunks) mma_commit_multicast(&sm.bar[B_P_FREE0 + (c & 1)], 3);   // as for T_FREE
                 }
@@ -714,7 +729,7 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             if (!no_out) {
                 if (!(ok = wwait(B_P_READY, ph))) break;
                 tc_fence_after();
-                mma_3(tmem + TM_PU, d_ph, d_pl, d_rh, d_rl);
+                mma_3(tmem + TM_PU, d_ph, d_pl, d_dh, d_dl);
                 mma_commit(&sm.bar[B_D4_DONE]);
             }
             KLA_TR(0, c, 7);
@@ -1087,7 +1102,7 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             warp_arrive(B_RHS_READY);
             KLA_TR(2, c, 3);
 
-            // ---- U and D U as hi/lo operands -------------------------------------------------------------------
+            // ---- D U as hi/lo operand: of the state update and, against P D^-1, of the outputs --------------------------------
             if (!wait(B_D3_DONE, ph)) break;
             KLA_TR(2, c, 4);
             tc_fence_after();
@@ -1097,12 +1112,6 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 tmem_ld16x256b_x1(tm16 + TM_U + 8 * j, acc);
                 const uint32_t o0 = off(i0, j), o1 = off(i1, j);
                 uint32_t hi, lo;
-                split2(acc[0], acc[1], hi, lo);
-                *reinterpret_cast<uint32_t *>(sm.ru_hi + o0) = hi;
-                *reinterpret_cast<uint32_t *>(sm.ru_lo + o0) = lo;
-                split2(acc[2], acc[3], hi, lo);
-                *reinterpret_cast<uint32_t *>(sm.ru_hi + o1) = hi;
-                *reinterpret_cast<uint32_t *>(sm.ru_lo + o1) = lo;
                 split2(d0 * acc[0], d0 * acc[1], hi, lo);
                 *reinterpret_cast<uint32_t *>(sm.du_hi + o0) = hi;
                 *reinterpret_cast<uint32_t *>(sm.du_lo + o0) = lo;

@@ -318,3 +318,15 @@ def test_paired_launch_is_repeatable_over_several_waves():
     for _ in range(12):
         o_p, f_p = gpu_chunk(wl)
         assert torch.equal(o_p, o_u) and torch.equal(f_p, f_u)
+
+
+@pytest.mark.parametrize("flags", [0, KLA_FLAG_NO_PAIR, KLA_FLAG_FORCE_SIMT])
+@pytest.mark.parametrize("d", [64, 128])
+def test_decay_far_beyond_the_exponent_range_within_one_chunk(d, flags):
+    """log alpha of -0.5 .. -4 per token: exp(g_C - g_j) spans hundreds of binades inside a chunk, far below what fp32
+    holds.  The tensor-core kernel factors the output product through those weights (with a floor): the outputs of
+    tokens next to the writes, where the unfactored decay is ~1, must still be right."""
+    w = W.config3(B=2, H=2, T=200, d=d, seed=71)
+    g = torch.Generator().manual_seed(72)
+    w.log_alpha = -(0.5 + 3.5 * torch.rand(w.log_alpha.shape, generator=g))
+    _check_fixed(w, TOL_BF16, flags=flags)

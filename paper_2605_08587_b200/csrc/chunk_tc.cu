@@ -578,7 +578,7 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         };
         // [K or Q](c) S_0 -> d; qoff = 512 selects the Q tile of a block; S_0 = S_hi + S_lo
         // (blocks t0 .. t1 - 1 of the 2 KB four-MMA blocks: the S_hi term first, then the S_lo term)
-        auto mma_xs = [&](uint32_t d, uint32_t k0, uint32_t qoff, int t0 = 0, int t1 = 2 * KB) {
+        auto mma_xs = [&](uint32_t d, uint32_t k0, uint32_t qoff, int t0, int t1) {
 #pragma unroll 1
             for (int t = t0; t < t1; ++t) {
                 const uint32_t kb = (uint32_t)t & (KB - 1);
@@ -620,7 +620,7 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 if (!(ok = wwait(B_S_READY, ph))) break;
                 KLA_TR(0, c, 1);
                 tc_fence_after();
-                mma_xs(tmem + TM_KS, k0, 0);
+                mma_xs(tmem + TM_KS, k0, 0, 0, 2 * KB);
                 mma_commit(&sm.bar[B_D2_DONE]);
                 const int cn = c + 2;   // this CTA's next chunk
                 bool m1_due = own && cn < nchunks;
@@ -698,7 +698,7 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             tc_fence_after();
 #pragma unroll 1
             for (int x = 0; x < (no_out ? 1 : 2); ++x) {
-                mma_xs(tmem + (x == 0 ? TM_KS : ((c & 1) ? TM_QS1 : TM_QS0)), k0, x * 512);
+                mma_xs(tmem + (x == 0 ? TM_KS : ((c & 1) ? TM_QS1 : TM_QS0)), k0, x * 512, 0, 2 * KB);
                 if (x == 0) mma_commit(&sm.bar[B_D2_DONE]);
             }
             KLA_TR(0, c, 2);

@@ -1083,7 +1083,7 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             for (int j = 0; j < 4; ++j) {
                 float acc[4];
                 tmem_ld16x256b_x1(tm16 + TM_KS + 8 * j, acc);
-                const uint32_t o0 = off(i0, j), o1 = off(i1, j);
+                const uint32_t o0 = off(i0, j), o1 = o0 + 8 * 128;   // i1 = i0 + 8: same swizzle phase, eight rows on
                 // V[i0][cp + 8j .. +1], V[i1][...]; rows past the end of the sequence are another sequence's tokens
                 const uint32_t va = (i0 < rows && !is_map) ? *reinterpret_cast<const uint32_t *>(sm.vt + o0) : 0u;
                 const uint32_t vb = (i1 < rows && !is_map) ? *reinterpret_cast<const uint32_t *>(sm.vt + o1) : 0u;
@@ -1110,7 +1110,7 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             for (int j = 0; j < 4; ++j) {
                 float acc[4];
                 tmem_ld16x256b_x1(tm16 + TM_U + 8 * j, acc);
-                const uint32_t o0 = off(i0, j), o1 = off(i1, j);
+                const uint32_t o0 = off(i0, j), o1 = o0 + 8 * 128;   // i1 = i0 + 8: same swizzle phase, eight rows on
                 uint32_t hi, lo;
                 split2(d0 * acc[0], d0 * acc[1], hi, lo);
                 *reinterpret_cast<uint32_t *>(sm.du_hi + o0) = hi;

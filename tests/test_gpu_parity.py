@@ -330,3 +330,25 @@ def test_decay_far_beyond_the_exponent_range_within_one_chunk(d, flags):
     g = torch.Generator().manual_seed(72)
     w.log_alpha = -(0.5 + 3.5 * torch.rand(w.log_alpha.shape, generator=g))
     _check_fixed(w, TOL_BF16, flags=flags)
+
+
+# ---- seeded sweep over shapes and launch forms ------------------------------------------------------------------------------
+def _sweep_cases():
+    rng = np.random.default_rng(20260501)
+    cases = []
+    for n in range(24):
+        d = int(rng.choice([64, 128]))
+        B = int(rng.integers(1, 4))
+        H = int(rng.integers(1, 5))
+        T = int(rng.choice([rng.integers(1, 64), rng.integers(64, 400), rng.integers(400, 1400)]))
+        form = int(rng.choice([0, KLA_FLAG_NO_PAIR, KLA_FLAG_SEGMENTS(int(rng.integers(2, 6))),
+                               KLA_FLAG_SEGMENTS(int(rng.integers(2, 6))) | KLA_FLAG_NO_PAIR]))
+        bf16_out = bool(rng.integers(0, 2))
+        cases.append((n, d, B, H, T, form, bf16_out))
+    return cases
+
+
+@pytest.mark.parametrize("n,d,B,H,T,form,bf16_out", _sweep_cases())
+def test_seeded_sweep_of_shapes_and_launch_forms(n, d, B, H, T, form, bf16_out):
+    w = (W.config3 if n % 2 else W.config2)(B=B, H=H, T=T, d=d, seed=900 + n)   # with / without an initial state
+    _check_fixed(w, TOL_BF16, flags=form, out_dtype=torch.bfloat16 if bf16_out else torch.float32)

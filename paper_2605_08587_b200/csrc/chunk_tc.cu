@@ -769,7 +769,6 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         if ((int)rank < nchunks) fetch_gates((int)rank);
         bool okp = true;   // outcome of the P warps' waits, folded into the next collective decision
         for (int c = 0; c < nchunks; ++c) {
-            const uint32_t ph = (uint32_t)(c & 1);
             const int rows = (c == nchunks - 1) ? last_rows : C;
             const int sc = c % NSTAGE;
             const bool own = (uint32_t)(c & 1) == rank;
@@ -1021,9 +1020,8 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         const int hf = ct >> 7;                 // column half: 0 -> columns 0..31, 1 -> 32..63
         const int srow = q * 32 + lane;         // state row (M = 128 accumulator layout, 32x32b loads)
         const bool s_act = srow < D;
-        // M = 64 accumulators, 16x256b loads: rows i0 and i0 + 8, column pairs cp + 8j (j = 0..3)
+        // M = 64 accumulators, 16x256b loads: rows i0 and i0 + 8, column pairs cp + 8j (j = 0..3), cp = hf * 32 + 2 (lane % 4)
         const int i0 = q * 16 + (lane >> 2), i1 = i0 + 8;
-        const int cp = hf * 32 + 2 * (lane & 3);
         const uint32_t tm16 = tmem + ((uint32_t)(q * 32) << 16) + hf * 32;
 
         float S[32];

@@ -933,6 +933,17 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             warp_arrive(B_P_READY);
             return true;
         };
+        // barrier over the four K K^T warps (128 threads) that also ORs a flag
+        auto kk_any = [&](bool flag) -> bool {
+            uint32_t r;
+            asm volatile(
+                "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 p, %1, 0;\n\t"
+                "bar.red.or.pred q, 5, 128, p;\n\tselp.u32 %0, 1, 0, q;\n\t}"
+                : "=r"(r)
+                : "r"((uint32_t)flag)
+                : "memory");
+            return r != 0;
+        };
         fetch_gates(0);
         int c = 0;
         for (; c < nchunks; ++c) {
@@ -978,24 +989,29 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     tc_fence_before();
                     warp_arrive(B_D1_FREE0 + (c & 1));
                 }
+                // ---- T = (I + B X)^-1, first the 8x8 diagonal blocks by substitution.  The four K K^T warps go on to
+                // them at once (forming P takes the Q K^T warps almost twice as long as X takes these): they meet,
+                // two of them substitute, and the one with no X work takes the wait that guards the T tiles
+                // (MMA-3(c-1) must have read the previous ones; the first look at a barrier completed by the tensor pipe
+                // costs several hundred cycles wherever it is taken, so it is taken here).  Letting these four warps
+                // do the block merges at sizes 8 and 16 as well (work for 64 and 128 threads) made them the longer half.
+                if (!kk_any(!okc)) {
+                    const int gt = (chh * 2 + (q & 1)) * 32 + lane;   // 0..127 over the four warps
+                    if (gt < 64) substitute_diag_blocks(sm.tl, sm.beta[sc], gt);
+                    if (c > 0 && scan_warp) okc = wait(B_D3_DONE, ph ^ 1);
+                } else {
+                    okc = false;
+                }
             } else if (no_out) {
                 warp_arrive(B_D1_FREE0 + (c & 1));   // nothing reads Q K^T: release this warp's share of D1(c)
             } else if (c > 0) {
                 okc = form_p(c - 1);
             }
-            if (pg_any(!okc)) break;
+            if (pg_any(!okc)) break;   // X, the diagonal blocks and P(c-1) are done
             KLA_TR(1, c, 1);
 
-            // ---- T = (I + B X)^-1: 8x8 diagonal blocks by substitution, then the off-diagonal blocks
-            //      T_10 = -T_11 (B_1 X_10 T_00) at block sizes 8, 16, 32 -----------------------------------------------
+            // ---- then the off-diagonal blocks T_10 = -T_11 (B_1 X_10 T_00) at block sizes 8, 16, 32 -------------------
             const float *bet = sm.beta[sc];
-            if (pt < 64) substitute_diag_blocks(sm.tl, bet, pt);
-            // Meanwhile a warp with nothing to substitute takes the wait that guards the T tiles (MMA-3(c-1) must have
-            // read the previous ones): the first look at a barrier completed by the tensor pipe costs several hundred
-            // cycles wherever it is taken, so it is taken here, under the substitution.
-            bool okd = true;
-            if (c > 0 && pt >= PG_T - 32) okd = wait(B_D3_DONE, ph ^ 1);
-            if (pg_any(!okd)) break;
             KLA_TR(1, c, 2);
             merge_level<8>(sm.tl, sm.mm, bet, pt);
             KLA_TR(1, c, 6);

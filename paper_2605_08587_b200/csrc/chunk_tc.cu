@@ -329,7 +329,7 @@ template <typename Smem>
 __device__ __forceinline__ void form_p_row(Smem &sm, int sc, int i, int chh, bool live, uint32_t tbase)
 {
     const float gi2 = sm.g2[sc][i], gc2 = sm.g2[sc][C - 1];
-#pragma unroll 1
+#pragma unroll 2
     for (int grp = 0; grp < 4; ++grp) {
         uint4 hi = make_uint4(0, 0, 0, 0), lo = hi;
         if (live) {

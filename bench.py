@@ -239,7 +239,7 @@ def decode_leg(dev, steps_per_call, calls, warmup, peaks, B=64, H=8, d=128, l2_d
             "state_mb": state_bytes / 2 / 1e6, "state_fits_l2": state_bytes / 2 < 126e6}
 
 
-def e2e_leg(w, dev, steps, warmup, groups=4):
+def e2e_leg(w, dev, steps, warmup, groups=8):
     """Same step, host buffers: pinned host -> device copies of every input, the launches, and the
     device -> host read of out and final state, all inside the timed region.  The batch is cut into `groups`
     groups of sequences (they are independent problems) that go round two streams, so that the upload of one

@@ -28,9 +28,10 @@ if ROOT not in sys.path:
 
 METRIC = "chunk_fwd_throughput"
 UNIT = "Mtok/s"
+WORKLOAD = "cfg2_bf16_B8_H8_T4096_d128_chunk64"   # the same string in both arms
 # dram__bytes_read.sum + dram__bytes_write.sum of one headline launch of the chunk kernel, from the ncu capture
 # summarised under profiles/; None while the kernel has changed since the counters were taken.
-CHUNK_TC_DRAM_BYTES_PER_LAUNCH = 255527680   # 203.79 MB read + 51.74 MB written
+CHUNK_TC_DRAM_BYTES_PER_LAUNCH = None
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -143,6 +144,38 @@ def oracle_sample_run(seed=1, B=2, H=8, T=4096, d=128, repeats=1):
     return B * T / best / 1e6, thr, best
 
 
+def oracle_chunk_workload(w):
+    """The fp64 oracle, as it stands, on a whole chunk-forward workload (one run).  Returns a cpu_baseline dict."""
+    import oracle
+    packed = w.cu_seqlens is not None
+    a = [(x[0] if packed else x).float().numpy() for x in (w.q, w.k, w.v)] + [(x[0] if packed else x).numpy() for x in (w.log_alpha, w.eta)]
+    s0 = None if w.init_state is None else w.init_state.numpy()
+    t0 = time.perf_counter()
+    if packed:
+        _, _, thr = oracle.forward_packed(*a, w.eps, w.cu_seqlens.numpy(), s0)
+    else:
+        _, _, thr = oracle.forward(*a, w.eps, s0)
+    dt = time.perf_counter() - t0
+    return {"value": w.n_tok / dt / 1e6, "unit": UNIT, "cores": thr, "kind": "oracle",
+            "sample": "the whole workload %s, one run, %.1f s" % (w.name, dt)}
+
+
+def oracle_decode_workload(B=64, H=8, d=128, steps=128):
+    """The fp64 oracle's decode step, `steps` consecutive steps of the decode workload.  Returns a cpu_baseline dict."""
+    import numpy as np
+    import oracle
+    from paper_2605_08587_b200 import workloads as W
+    w = W.config4(B=B, H=H, d=d, steps=steps)
+    st = w.state.numpy().astype(np.float64)
+    a = [x.float().numpy() for x in (w.q, w.k, w.v)] + [w.log_alpha.numpy(), w.eta.numpy()]
+    t0 = time.perf_counter()
+    for s in range(steps):
+        oracle.decode_step(a[0][s], a[1][s], a[2][s], a[3][s], a[4][s], w.eps, st)
+    dt = time.perf_counter() - t0
+    return {"value": B * steps / dt, "unit": "tok/s", "cores": os.cpu_count(), "kind": "oracle",
+            "sample": "%d consecutive decode steps of the B=%d workload (of its 1024), %.1f s" % (steps, B, dt)}
+
+
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -160,7 +193,7 @@ def run_reference(args):
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": "cfg2_bf16_B8_H8_T4096_d128_chunk64", "sampled": desc},
+            "config": {"workload": WORKLOAD, "sampled": desc},
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": thr, "kind": "oracle", "sample": desc},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -168,20 +201,23 @@ def run_reference(args):
 
 
 # ---- GPU legs ----------------------------------------------------------------------------------------------------
-def time_launches(fn, steps, warmup, stream):
-    """Average device time per call of fn() in ms: CUDA events on the launching stream."""
+def time_launches(fn, steps, warmup, stream, stats=None):
+    """Average device time per call of fn() in ms: CUDA events on the launching stream, one after every call, so that
+    the median and the minimum of the per-call times can be reported beside the mean (`stats`, a dict, receives them)."""
     import torch
     for _ in range(warmup):
         fn()
     torch.cuda.synchronize()
-    e0 = torch.cuda.Event(enable_timing=True)
-    e1 = torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for _ in range(steps):
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    ev[0].record(stream)
+    for i in range(steps):
         fn()
-    e1.record(stream)
+        ev[i + 1].record(stream)
     torch.cuda.synchronize()
-    return e0.elapsed_time(e1) / steps
+    if stats is not None:
+        per = [ev[i].elapsed_time(ev[i + 1]) for i in range(steps)]
+        stats.update({"ms_median": statistics.median(per), "ms_min": min(per), "ms_max": max(per), "repetitions": steps})
+    return ev[0].elapsed_time(ev[steps]) / steps
 
 
 def to_dev(w, dev):
@@ -205,14 +241,20 @@ def chunk_leg(w, dev, steps, warmup, peaks, out_dtype):
                       init_state=t["init_state"], out=out, final_state=fin, cu_seqlens=t["cu_seqlens"],
                       host_seqlens=t["host_seqlens"])
 
-    ms = time_launches(step, steps, warmup, torch.cuda.current_stream())
+    stats = {}
+    ms = time_launches(step, steps, warmup, torch.cuda.current_stream(), stats)
+    # per-pass device times of one more call (set-up kernels, segment pass 1, chaining of the maps, main pass)
+    passes = []
+    kla_chunk_fwd(t["q"], t["k"], t["v"], t["log_alpha"], t["eta"], w.eps, chunk=w.chunk, init_state=t["init_state"], out=out,
+                  final_state=fin, cu_seqlens=t["cu_seqlens"], host_seqlens=t["host_seqlens"], pass_ms=passes)
     nbytes = algorithmic_bytes(B * T, H, d, n_seq, w.q.element_size(), out.element_size(), w.init_state is not None, True)
     flops = algorithmic_flops(B * T, H, d, w.chunk)
     gbs = nbytes / (ms * 1e-3) / 1e9
     tfs = flops / (ms * 1e-3) / 1e12
     t_hbm = nbytes / (peaks["hbm_gbs"] * 1e9)
     t_tc = flops / (peaks["bf16_tflops"] * 1e12)
-    return {"workload": w.name, "ms": ms, "mtok_per_s": B * T / (ms * 1e-3) / 1e6, "tokens": B * T,
+    return {"workload": w.name, "ms": ms, **stats, "mtok_per_s": B * T / (ms * 1e-3) / 1e6, "tokens": B * T,
+            "pass_us": {"setup": 1e3 * passes[0], "segment_pass_1": 1e3 * passes[1], "chain_maps": 1e3 * passes[2], "main_pass": 1e3 * passes[3]},
             "algorithmic_bytes": nbytes, "algorithmic_flops": flops, "achieved_gbs": gbs, "achieved_tflops": tfs,
             "roofline_ms": 1e3 * max(t_hbm, t_tc), "roofline_frac": max(t_hbm, t_tc) / (ms * 1e-3),
             "bound": "hbm" if t_hbm >= t_tc else "tensor"}
@@ -229,14 +271,30 @@ def decode_leg(dev, steps_per_call, calls, warmup, peaks, B=64, H=8, d=128, l2_d
     def step():
         kla_decode_steps(*args, w.eps, st, out=out)
 
-    ms = time_launches(step, calls, warmup, torch.cuda.current_stream()) / steps_per_call
+    stats = {}
+    ms = time_launches(step, calls, warmup, torch.cuda.current_stream(), stats) / steps_per_call
+    stats = {"us_per_step_median": 1e3 * stats["ms_median"] / steps_per_call, "us_per_step_min": 1e3 * stats["ms_min"] / steps_per_call,
+             "calls": calls, "consecutive_steps_per_call": steps_per_call}
     state_bytes = 2 * B * H * d * d * 4
     vec_bytes = B * H * (3 * d * 2 + d * 2 + 8)
     nbytes = state_bytes + vec_bytes
     gbs = nbytes / (ms * 1e-3) / 1e9
-    return {"workload": w.name, "us_per_step": ms * 1e3, "tok_per_s": B / (ms * 1e-3), "bytes_per_step": nbytes,
+    return {"workload": w.name, "us_per_step": ms * 1e3, **stats, "tok_per_s": B / (ms * 1e-3), "bytes_per_step": nbytes,
             "effective_gbs": gbs, "frac_of_hbm_peak": gbs / peaks["hbm_gbs"],
             "state_mb": state_bytes / 2 / 1e6, "state_fits_l2": state_bytes / 2 < 126e6}
+
+
+def wy_leg(w, t, dev, steps, warmup):
+    """The headline workload through the WY-form kernel (KLA_FLAG_WY_FORM), for comparison with the default form."""
+    import torch
+    from paper_2605_08587_b200 import KLA_FLAG_WY_FORM, kla_chunk_fwd
+    B, T, H, d = w.q.shape
+    out = torch.empty((B, T, H, d), device=dev, dtype=torch.bfloat16)
+    fin = torch.empty((B, H, d, d), device=dev, dtype=torch.float32)
+    stats = {}
+    ms = time_launches(lambda: kla_chunk_fwd(t["q"], t["k"], t["v"], t["log_alpha"], t["eta"], w.eps, chunk=w.chunk, out=out,
+                                             final_state=fin, flags=KLA_FLAG_WY_FORM), steps, warmup, torch.cuda.current_stream(), stats)
+    return {"workload": w.name, "ms": ms, **stats, "mtok_per_s": B * T / (ms * 1e-3) / 1e6}
 
 
 def e2e_leg(w, dev, steps, warmup, groups=8):
@@ -319,20 +377,22 @@ def run_ours(args):
         dist.barrier()
     torch.cuda.synchronize()
     n0 = launch_count()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
     with ClockSampler(local) as clk:
-        e0.record(stream)
-        for _ in range(args.steps):
+        ev[0].record(stream)
+        for i in range(args.steps):
             step()
-        e1.record(stream)
+            ev[i + 1].record(stream)
         torch.cuda.synchronize()
         launches = launch_count() - n0   # kernels launched inside the timed region
-        # keep sampling under load if the timed region was shorter than a few sampling periods
+        # The timed region (a few ms) is shorter than one sampling period of nvidia-smi: the same launch is repeated
+        # for 0.6 s after it, and the clock samples are taken over the timed steps and those repetitions.
         t_end = time.time() + (0.0 if args.quick else 0.6)
         while time.time() < t_end:
             step()
         torch.cuda.synchronize()
-    total_ms = e0.elapsed_time(e1)
+    total_ms = ev[0].elapsed_time(ev[args.steps])
+    per_step = [ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)]
     if world > 1:
         dist.barrier()
     total_ms = max_over_ranks(total_ms, dev)
@@ -354,7 +414,7 @@ def run_ours(args):
     t_hbm = nbytes / (peaks["hbm_gbs"] * 1e9)
     t_tc = flops / (peaks["bf16_tflops"] * 1e12)
     achieved = nbytes / (ms * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+    roofline = {"bound": "hbm" if t_hbm >= t_tc else "tensor", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": peak_src + " (burst copy)",
                 "kernel": "kla_chunk_tc_kernel",
                 "algorithmic_bytes_per_launch": nbytes, "algorithmic_flops_per_launch": flops,
@@ -374,10 +434,17 @@ def run_ours(args):
         elif args.also == "varlen":
             extras["chunk_cfg5_varlen"] = chunk_leg(W.config5(), dev, 2, 1, peaks, torch.bfloat16)
     if not args.quick:
-        extras["decode_cfg4"] = decode_leg(dev, 256, 4, 2, peaks)
-        extras["decode_l2_defeating_B512"] = decode_leg(dev, 32, 4, 2, peaks, B=512)
-        extras["chunk_cfg3_long_context"] = chunk_leg(W.config3(), dev, 5, 3, peaks, torch.bfloat16)
-        extras["chunk_cfg5_varlen"] = chunk_leg(W.config5(), dev, 5, 3, peaks, torch.bfloat16)
+        # decode: calls of 1024 consecutive steps on 1024 distinct token vectors, state carried in place
+        extras["decode_cfg4"] = decode_leg(dev, 1024, 5, 1, peaks)
+        # (B = 512: 128 consecutive steps per call; 1024 steps of inputs would be 4 GB)
+        extras["decode_l2_defeating_B512"] = decode_leg(dev, 128, 5, 1, peaks, B=512)
+        extras["chunk_cfg3_long_context"] = chunk_leg(W.config3(), dev, 20, 3, peaks, torch.bfloat16)
+        extras["chunk_cfg5_varlen"] = chunk_leg(W.config5(), dev, 20, 3, peaks, torch.bfloat16)
+        extras["chunk_cfg2_wy_form"] = wy_leg(w, t, dev, 20, 3)
+        if not args.no_cpu_baseline:
+            extras["chunk_cfg3_long_context"]["cpu_baseline"] = oracle_chunk_workload(W.config3())
+            extras["chunk_cfg5_varlen"]["cpu_baseline"] = oracle_chunk_workload(W.config5())
+            extras["decode_cfg4"]["cpu_baseline"] = oracle_decode_workload()
 
     cpu = None
     if not (args.no_cpu_baseline or args.quick):
@@ -386,13 +453,15 @@ def run_ours(args):
                "sample": "the whole headline workload (8 sequences x 8 heads x 4096 tokens), best of 3 runs, %.1f s each" % dt}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": max(3, args.warmup), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+            "warmup": max(3, args.warmup), "ms_per_step": ms, "ms_per_step_median": statistics.median(per_step),
+            "ms_per_step_min": min(per_step), "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": "cfg2_bf16_B8_H8_T4096_d128_chunk64 per GPU", "tokens_per_step": tokens_all,
+            "config": {"workload": WORKLOAD, "per_gpu": "every GPU runs this workload on its own batch", "tokens_per_step": tokens_all,
                        "arithmetic": "bf16 tensor-core operands (derived operands as hi/lo pairs), fp32 accumulation and state",
                        "l2": "inputs+outputs per step are 271 MB > 126 MB L2, no flush needed",
                        "parallelism": "independent batches per GPU, no collective"},
-            "clocks": clk.summary(), "roofline": roofline, "cpu_baseline": cpu,
+            "clocks": {**clk.summary(), "sampled_over": "the timed steps and 0.6 s of the same launch repeated right after them"},
+            "roofline": roofline, "cpu_baseline": cpu,
             "e2e": {"value": tokens_all / (e2e_ms * 1e-3) / 1e6, "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
             "gpu_launches": launches, "extras": extras}

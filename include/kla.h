@@ -17,7 +17,10 @@
  *
  * General rules
  *  - Every data pointer is a DEVICE pointer unless stated otherwise; every buffer is owned by the
- *    caller.  The library allocates nothing and keeps no state between calls.
+ *    caller.  The library allocates nothing, on host or device.  The only state it keeps between calls is
+ *    process-wide bookkeeping that no result depends on: the launch counter read by kla_launch_count, the
+ *    driver entry point used to encode tensor maps, and, for kla_chunk_fwd_static_scratch, the device address
+ *    of its built-in scratch array (looked up once per device; stale after cudaDeviceReset).
  *  - All arrays are dense, row-major, last index contiguous, 16-byte aligned.
  *  - Work is enqueued on desc->stream and the call returns without synchronising.  Argument
  *    errors are detected on the host before anything is launched and reported through the
@@ -48,7 +51,9 @@ typedef enum {
     KLA_ERR_EPS = -8,       /* eps < 0 or not finite                                       */
     KLA_ERR_LAUNCH = -9,    /* the CUDA runtime rejected a launch (see cudaGetLastError)   */
     KLA_ERR_TIMEOUT = -10,  /* written to *status_word by a kernel whose bounded wait ran out */
-    KLA_ERR_ARCH = -11      /* current device is not sm_100                                */
+    KLA_ERR_ARCH = -11,     /* current device is not sm_100                                */
+    KLA_ERR_DEVICE = -12    /* the current device could not be queried, or (static scratch) its index is
+                               beyond the table of scratch addresses or the address lookup failed */
 } kla_status;
 
 typedef enum { KLA_F32 = 0, KLA_BF16 = 1 } kla_dtype;
@@ -58,25 +63,32 @@ typedef enum { KLA_F32 = 0, KLA_BF16 = 1 } kla_dtype;
 /* Force the CUDA-core fp32 chunk kernel even where the tensor-core kernel applies (used to
  * cross-check the two device paths against each other and against the oracle). */
 #define KLA_FLAG_FORCE_SIMT 1
-/* Segment-parallel scan of the tensor-core path (fixed-length input only).  Every chunk step is affine in the
- * incoming state (Eqs. 7-9), so a sequence can be cut into G segments whose transition maps are found in
- * parallel, chained, and the segments then run in parallel from their true start states: the same result up
- * to rounding, about three times the state work, G times the parallelism.  By default the library decides
- * from the shape (few long sequences -> segments) and the workspace query returns what that decision needs. */
 /* Layer-edge variants named by the paper; both default to off (the recurrence at the top of this file). */
 #define KLA_FLAG_COEFF_ETA 4              /* beta_t = eta_t: the gated-delta-rule baseline coefficient of Section 2,
                                              without the key-norm division of Eq. 3 (eps is then unused)          */
 #define KLA_FLAG_QNORM 8                  /* o_t = S_t^T q_t / ||q_t||: the read-out as Algorithm 1 (left) prints it */
-/* Test hook for the error path: the tensor-core kernel withholds one internal completion signal, so that a
- * bounded device-side wait runs out (about one second), every CTA gives up in an orderly way and KLA_ERR_TIMEOUT
- * appears in *status_word.  Outputs are then undefined; the context stays usable. */
-#define KLA_FLAG_TEST_TIMEOUT 16
+/* Not part of the supported flag set: used by the library's own tests of the error path.  The tensor-core kernel
+ * withholds one internal completion signal, so that a bounded device-side wait runs out (about one second), every
+ * CTA gives up in an orderly way and KLA_ERR_TIMEOUT appears in *status_word.  Outputs are then undefined; the
+ * context stays usable. */
+#define KLA_INTERNAL_FLAG_TEST_TIMEOUT 16
 /* With d_v = 128 the two CTAs that hold the two 64-column slices of a head run as a thread-block cluster and share
  * the work that does not depend on the state (each inverts every other chunk's I + B X and hands the result to its
  * peer through distributed shared memory).  This flag launches them as independent CTAs instead, each doing all of
  * that work itself; the arithmetic is the same, so the results are bit-identical.  Used to cross-check the two
  * launch forms. */
 #define KLA_FLAG_NO_PAIR 32
+/* Head dimension 128 only (ignored otherwise): run the chunk forward in the WY form of Appendix B (Props. 5-6 and the
+ * combined representation U^ = U - W S_0, with W = T B D_gamma K and U = T B V formed on tensor cores off the serial
+ * chain) instead of the default W-free form of Algorithm 1 right.  Same result up to rounding; the product W S_0 is
+ * taken in fp16 (11 significand bits), which holds the 2e-3 bound on layer-shaped inputs but not on inputs with
+ * heavy-tailed key norms, and needs the state and W inside the fp16 range. */
+#define KLA_FLAG_WY_FORM 64
+/* Segment-parallel scan of the tensor-core path (fixed-length input only).  Every chunk step is affine in the
+ * incoming state (Eqs. 7-9), so a sequence can be cut into G segments whose transition maps are found in
+ * parallel, chained, and the segments then run in parallel from their true start states: the same result up
+ * to rounding, about three times the state work, G times the parallelism.  By default the library decides
+ * from the shape (few long sequences -> segments) and the workspace query returns what that decision needs. */
 #define KLA_FLAG_NO_SEGMENTS 2            /* never cut sequences into segments                              */
 #define KLA_FLAG_SEGMENTS(g) ((g) << 8)   /* force g segments per sequence, 2 <= g <= 255 (fewer if T is short) */
 
@@ -147,16 +159,33 @@ kla_status kla_chunk_fwd(const kla_desc *desc, const void *q, const void *k, con
  *    anything is launched (kla_chunk_fwd_workspace_bytes tells what a shape needs; KLA_FLAG_NO_SEGMENTS makes
  *    the need zero at the price of less parallelism).
  *  - The first call on each device looks up that device's address of the array (with the device current, as
- *    for every call); make that first call outside any stream capture.
+ *    for every call); make that first call outside any stream capture.  With the CUDA runtime's lazy module
+ *    loading this is also when the device sets the array aside.
  *  - All calls share the one array and it keeps the previous call's contents.  Nothing in it has to start at
  *    zero (a call writes every byte it later reads), but two calls that overlap on the GPU -- different streams,
  *    or host threads racing on one stream -- would overwrite each other's segments: serialise them.
- *  - Everything else (arguments, layouts, results, error codes) is exactly kla_chunk_fwd.
+ *  - Arguments are validated exactly as by kla_chunk_fwd (same codes, same order, except that the workspace fields
+ *    are not looked at); then comes the size check above; KLA_ERR_DEVICE if the current device's index is beyond the
+ *    library's table of scratch addresses (64 devices) or the address lookup fails.  Layouts and results are those
+ *    of kla_chunk_fwd.
  */
 #define KLA_STATIC_SCRATCH_BYTES (32u << 20)
 kla_status kla_chunk_fwd_static_scratch(const kla_desc *desc, const void *q, const void *k, const void *v,
                                         const float *log_alpha, const float *eta, float eps, int32_t chunk,
                                         const float *init_state, void *out, float *final_state);
+
+/*
+ * kla_chunk_fwd with per-pass device times (a measurement aid; no counterpart in the paper).  Does exactly the work
+ * of kla_chunk_fwd with the same arguments, records CUDA events on desc->stream between the launches, waits for
+ * the stream and writes milliseconds to the HOST array pass_ms[4]:
+ *   [0] set-up kernels (segment bounds or the order of packed sequences), [1] segment pass 1 (transition maps),
+ *   [2] the chaining of the segment maps, [3] the main pass (segment pass 3, or the only pass of a plain launch).
+ * Entries of passes that did not run are 0.  Synchronises with the stream (unlike kla_chunk_fwd); creates and
+ * destroys four CUDA events; otherwise allocates nothing.
+ */
+kla_status kla_chunk_fwd_timed(const kla_desc *desc, const void *q, const void *k, const void *v,
+                               const float *log_alpha, const float *eta, float eps, int32_t chunk,
+                               const float *init_state, void *out, float *final_state, float *pass_ms);
 
 /*
  * One recurrent decode step (Algorithm 1 left) for B sequences x H heads; desc->T must be 1 and

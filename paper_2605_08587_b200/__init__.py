@@ -4,4 +4,4 @@
 `build` compiles the CUDA library in-tree.
 """
 from .binding import (KlaError, kla_chunk_fwd, kla_chunk_fwd_static_scratch, kla_decode_step, kla_decode_steps, launch_count,  # noqa: F401
-                      KLA_F32, KLA_BF16, KLA_FLAG_NONE, KLA_FLAG_FORCE_SIMT, KLA_FLAG_NO_SEGMENTS, KLA_FLAG_SEGMENTS, KLA_FLAG_COEFF_ETA, KLA_FLAG_QNORM, KLA_FLAG_NO_PAIR)
+                      KLA_F32, KLA_BF16, KLA_FLAG_NONE, KLA_FLAG_FORCE_SIMT, KLA_FLAG_NO_SEGMENTS, KLA_FLAG_SEGMENTS, KLA_FLAG_COEFF_ETA, KLA_FLAG_QNORM, KLA_FLAG_NO_PAIR, KLA_FLAG_WY_FORM)

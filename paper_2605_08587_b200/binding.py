@@ -14,7 +14,7 @@ LIB_PATH = os.path.join(_HERE, "libkla_b200.so")
 
 KLA_F32, KLA_BF16 = 0, 1
 KLA_FLAG_NONE, KLA_FLAG_FORCE_SIMT, KLA_FLAG_NO_SEGMENTS = 0, 1, 2
-KLA_FLAG_COEFF_ETA, KLA_FLAG_QNORM, KLA_FLAG_TEST_TIMEOUT, KLA_FLAG_NO_PAIR = 4, 8, 16, 32
+KLA_FLAG_COEFF_ETA, KLA_FLAG_QNORM, KLA_INTERNAL_FLAG_TEST_TIMEOUT, KLA_FLAG_NO_PAIR, KLA_FLAG_WY_FORM = 4, 8, 16, 32, 64
 
 
 def KLA_FLAG_SEGMENTS(g: int) -> int:
@@ -22,7 +22,7 @@ def KLA_FLAG_SEGMENTS(g: int) -> int:
     return int(g) << 8
 
 
-EXPORTS = ["kla_chunk_fwd_workspace_bytes", "kla_chunk_fwd", "kla_chunk_fwd_static_scratch", "kla_decode_step", "kla_decode_steps",
+EXPORTS = ["kla_chunk_fwd_workspace_bytes", "kla_chunk_fwd", "kla_chunk_fwd_timed", "kla_chunk_fwd_static_scratch", "kla_decode_step", "kla_decode_steps",
            "kla_status_str", "kla_launch_count"]
 
 
@@ -58,6 +58,8 @@ def load():
     lib.kla_chunk_fwd_workspace_bytes.argtypes = [dp, ctypes.c_int32]
     lib.kla_chunk_fwd.restype = ctypes.c_int
     lib.kla_chunk_fwd.argtypes = [dp, vp, vp, vp, fp, fp, ctypes.c_float, ctypes.c_int32, fp, vp, fp]
+    lib.kla_chunk_fwd_timed.restype = ctypes.c_int
+    lib.kla_chunk_fwd_timed.argtypes = lib.kla_chunk_fwd.argtypes + [ctypes.POINTER(ctypes.c_float)]
     lib.kla_chunk_fwd_static_scratch.restype = ctypes.c_int
     lib.kla_chunk_fwd_static_scratch.argtypes = lib.kla_chunk_fwd.argtypes
     lib.kla_decode_step.restype = ctypes.c_int
@@ -109,13 +111,15 @@ def _stream(dev):
 
 def kla_chunk_fwd(q, k, v, log_alpha, eta, eps, chunk=64, init_state=None, out=None, final_state=None,
                   cu_seqlens=None, host_seqlens=None, out_dtype=None, flags=KLA_FLAG_NONE,
-                  want_final_state=True, status_word=None):
+                  want_final_state=True, status_word=None, pass_ms=None):
     """Chunkwise forward (include/kla.h: kla_chunk_fwd).
 
     q, k [B, T, H, d_k]; v [B, T, H, d_v]; log_alpha, eta [B, T, H] fp32; all CUDA, contiguous.
     Packed input: B = 1, cu_seqlens int32 CUDA [n_seq + 1] plus `host_seqlens` (CPU int32 copy;
     made from cu_seqlens with one D2H copy if omitted).
     Returns (out, final_state); buffers are allocated here unless passed in.
+    `pass_ms`: a list; if given the call goes through kla_chunk_fwd_timed (which waits for the stream) and the four
+    per-pass device times in ms (set-up, segment pass 1, chaining, main pass) are appended to it.
     """
     lib = load()
     B, T, H, d_k = q.shape
@@ -150,11 +154,17 @@ def kla_chunk_fwd(q, k, v, log_alpha, eta, eps, chunk=64, init_state=None, out=N
     if need:
         ws = torch.empty(need, device=q.device, dtype=torch.uint8)
         desc.workspace, desc.workspace_bytes = ws.data_ptr(), need
+    args = (ctypes.byref(desc), _dev(q, "q"), _dev(k, "k"), _dev(v, "v"),
+            _dev(log_alpha, "log_alpha", torch.float32), _dev(eta, "eta", torch.float32),
+            float(eps), int(chunk), _dev(init_state, "init_state", torch.float32),
+            _dev(out, "out"), _dev(final_state, "final_state", torch.float32))
     with torch.cuda.device(q.device):
-        code = lib.kla_chunk_fwd(ctypes.byref(desc), _dev(q, "q"), _dev(k, "k"), _dev(v, "v"),
-                                 _dev(log_alpha, "log_alpha", torch.float32), _dev(eta, "eta", torch.float32),
-                                 float(eps), int(chunk), _dev(init_state, "init_state", torch.float32),
-                                 _dev(out, "out"), _dev(final_state, "final_state", torch.float32))
+        if pass_ms is None:
+            code = lib.kla_chunk_fwd(*args)
+        else:
+            ms = (ctypes.c_float * 4)()
+            code = lib.kla_chunk_fwd_timed(*args, ms)
+            pass_ms.extend(float(x) for x in ms)
     _check(code)
     return out, final_state
 
@@ -163,10 +173,11 @@ STATIC_SCRATCH_BYTES = 32 << 20
 
 
 def kla_chunk_fwd_static_scratch(q, k, v, log_alpha, eta, eps, out, final_state=None, chunk=64, init_state=None,
-                                 flags=KLA_FLAG_NONE):
+                                 flags=KLA_FLAG_NONE, cu_seqlens=None, host_seqlens=None, status_word=None):
     """Chunk forward for callers that cannot allocate device memory (include/kla.h:
-    kla_chunk_fwd_static_scratch).  The scratch of the segment-parallel scan is a fixed array inside the library,
-    so this wrapper allocates nothing either: `out` (and `final_state`, if wanted) must be passed in.  Shapes whose
+    kla_chunk_fwd_static_scratch).  The scratch (segment-parallel scan; longest-first order of packed sequences) is a
+    fixed array inside the library, so this wrapper allocates nothing either: `out` (and `final_state`, if wanted) must
+    be passed in, and for packed input both `cu_seqlens` (CUDA int32) and `host_seqlens` (CPU int32 copy).  Shapes whose
     scratch would exceed STATIC_SCRATCH_BYTES raise KlaError (workspace).  Calls must not overlap on the GPU."""
     lib = load()
     B, T, H, d_k = q.shape
@@ -175,9 +186,15 @@ def kla_chunk_fwd_static_scratch(q, k, v, log_alpha, eta, eps, out, final_state=
         raise ValueError("q, k, v, out shapes disagree")
     if tuple(log_alpha.shape) != (B, T, H) or tuple(eta.shape) != (B, T, H):
         raise ValueError("log_alpha, eta must be [B, T, H]")
-    desc = KlaDesc(B=B, T=T, H=H, d_k=d_k, d_v=d_v, n_seq=B, cu_seqlens=None, host_seqlens=None,
+    n_seq = B
+    if cu_seqlens is not None:
+        if host_seqlens is None or host_seqlens.is_cuda or host_seqlens.dtype != torch.int32 or cu_seqlens.dtype != torch.int32:
+            raise TypeError("packed input needs cu_seqlens (CUDA int32) and host_seqlens (CPU int32)")
+        n_seq = cu_seqlens.numel() - 1
+    desc = KlaDesc(B=B, T=T, H=H, d_k=d_k, d_v=d_v, n_seq=n_seq, cu_seqlens=_dev(cu_seqlens, "cu_seqlens"),
+                   host_seqlens=host_seqlens.data_ptr() if host_seqlens is not None else None,
                    io_dtype=_dt(q), out_dtype=_dt(out), flags=flags, workspace=None, workspace_bytes=0,
-                   status_word=None, stream=_stream(q.device))
+                   status_word=_dev(status_word, "status_word", torch.int32), stream=_stream(q.device))
     with torch.cuda.device(q.device):
         code = lib.kla_chunk_fwd_static_scratch(
             ctypes.byref(desc), _dev(q, "q"), _dev(k, "k"), _dev(v, "v"), _dev(log_alpha, "log_alpha", torch.float32),

@@ -14,7 +14,7 @@ static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 
 static kla_status check_arch()
 {
     int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return KLA_ERR_ARCH;
+    if (cudaGetDevice(&dev) != cudaSuccess) return KLA_ERR_ARCH;   // (no usable device: there is no fallback)
     int major = 0;
     if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return KLA_ERR_ARCH;
     return major == 10 ? KLA_OK : KLA_ERR_ARCH;
@@ -32,9 +32,9 @@ static kla_status check_common(const kla_desc *d)
 }
 
 // Host-side validation of a chunk-forward call; launches nothing.
-static kla_status check_chunk(const kla_desc *d, const void *q, const void *k, const void *v,
-                              const float *log_alpha, const float *eta, float eps, int32_t chunk,
-                              const float *init_state, void *out, float *final_state)
+kla_status check_chunk_args(const kla_desc *d, const void *q, const void *k, const void *v,
+                            const float *log_alpha, const float *eta, float eps, int32_t chunk,
+                            const float *init_state, void *out, float *final_state, bool check_workspace)
 {
     kla_status st = check_common(d);
     if (st != KLA_OK) return st;
@@ -56,7 +56,7 @@ static kla_status check_chunk(const kla_desc *d, const void *q, const void *k, c
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(log_alpha) || !aligned16(eta) ||
         !aligned16(out) || !aligned16(init_state) || !aligned16(final_state))
         return KLA_ERR_ALIGN;
-    if (kla_chunk_fwd_workspace_bytes(d, chunk) > 0) {
+    if (check_workspace && kla_chunk_fwd_workspace_bytes(d, chunk) > 0) {
         if (!d->workspace || d->workspace_bytes < kla_chunk_fwd_workspace_bytes(d, chunk)) return KLA_ERR_WORKSPACE;
         if (!aligned16(d->workspace)) return KLA_ERR_ALIGN;
     }
@@ -143,11 +143,18 @@ size_t kla_chunk_fwd_workspace_bytes(const kla_desc *desc, int32_t chunk)
     return plan_segments(desc, chunk).bytes;
 }
 
-kla_status kla_chunk_fwd(const kla_desc *desc, const void *q, const void *k, const void *v,
-                         const float *log_alpha, const float *eta, float eps, int32_t chunk,
-                         const float *init_state, void *out, float *final_state)
+}  // extern "C"
+
+// The chunk forward proper.  `marks`: null, or five events recorded on the stream around the set-up kernels, segment
+// pass 1, the chaining of the segment maps and the main pass (kla_chunk_fwd_timed).
+static kla_status chunk_fwd_impl(const kla_desc *desc, const void *q, const void *k, const void *v,
+                                 const float *log_alpha, const float *eta, float eps, int32_t chunk,
+                                 const float *init_state, void *out, float *final_state, cudaEvent_t *marks)
 {
-    kla_status st = check_chunk(desc, q, k, v, log_alpha, eta, eps, chunk, init_state, out, final_state);
+    auto mark = [&](int i) {
+        if (marks) cudaEventRecord(marks[i], (cudaStream_t)desc->stream);
+    };
+    kla_status st = check_chunk_args(desc, q, k, v, log_alpha, eta, eps, chunk, init_state, out, final_state, true);
     if (st != KLA_OK) return st;
     st = check_arch();
     if (st != KLA_OK) return st;
@@ -160,11 +167,10 @@ kla_status kla_chunk_fwd(const kla_desc *desc, const void *q, const void *k, con
     p.final_state = final_state;
     p.cu_seqlens = desc->cu_seqlens;
     p.status_word = desc->status_word;
-    p.trace = nullptr;
     p.seg_pass = 0; p.seg_G = 0; p.map_state = nullptr;
     p.variant = ((desc->flags & KLA_FLAG_COEFF_ETA) ? VARIANT_COEFF_ETA : 0) | ((desc->flags & KLA_FLAG_QNORM) ? VARIANT_QNORM : 0) |
-                ((desc->flags & KLA_FLAG_TEST_TIMEOUT) ? VARIANT_TEST_TIMEOUT : 0) |
-                ((desc->flags & KLA_FLAG_NO_PAIR) ? VARIANT_NO_PAIR : 0);
+                ((desc->flags & KLA_INTERNAL_FLAG_TEST_TIMEOUT) ? VARIANT_TEST_TIMEOUT : 0) |
+                ((desc->flags & KLA_FLAG_NO_PAIR) ? VARIANT_NO_PAIR : 0) | ((desc->flags & KLA_FLAG_WY_FORM) ? VARIANT_WY : 0);
     p.B = desc->B; p.T = desc->T; p.H = desc->H; p.n_seq = desc->n_seq;
     p.eps = eps;
     if (desc->T == 0) {
@@ -180,23 +186,28 @@ kla_status kla_chunk_fwd(const kla_desc *desc, const void *q, const void *k, con
     cudaStream_t stream = (cudaStream_t)desc->stream;
     cudaError_t err;
     const SegPlan pl = plan_segments(desc, chunk);
+    mark(0);
     if (pl.G >= 2) {
         char *ws = (char *)desc->workspace;
         int32_t *cu_seg = (int32_t *)ws;
         float *map = (float *)(ws + pl.off_map), *local = (float *)(ws + pl.off_local), *start = (float *)(ws + pl.off_start);
         if (launch_seg_bounds(cu_seg, desc->B, desc->T, pl.G, pl.seg_len, stream) != cudaSuccess) return KLA_ERR_LAUNCH;
+        mark(1);
         ChunkParams p1 = p;   // pass 1: transition map and zero-start state of every segment but the last
         p1.cu_seqlens = cu_seg; p1.n_seq = desc->B * pl.G;
         p1.init_state = nullptr; p1.final_state = local; p1.map_state = map;
         p1.seg_pass = 1; p1.seg_G = pl.G;
         if (launch_chunk_tc(p1, desc->d_k, desc->io_dtype, desc->out_dtype, stream) != cudaSuccess) return KLA_ERR_LAUNCH;
+        mark(2);
         if (launch_seg_combine(init_state, map, local, start, desc->B, desc->H, pl.G, desc->d_k, stream) != cudaSuccess)
             return KLA_ERR_LAUNCH;
+        mark(3);
         ChunkParams p3 = p;   // pass 3: every segment from its true start state
         p3.cu_seqlens = cu_seg; p3.n_seq = desc->B * pl.G;
         p3.init_state = start;
         p3.seg_pass = 3; p3.seg_G = pl.G;
         err = launch_chunk_tc(p3, desc->d_k, desc->io_dtype, desc->out_dtype, stream);
+        mark(4);
         return err == cudaSuccess ? KLA_OK : KLA_ERR_LAUNCH;
     }
     if (!(desc->flags & KLA_FLAG_FORCE_SIMT) && chunk_tc_supported(desc->d_k, chunk, desc->io_dtype)) {
@@ -205,12 +216,58 @@ kla_status kla_chunk_fwd(const kla_desc *desc, const void *q, const void *k, con
             if (launch_seq_order(desc->cu_seqlens, desc->n_seq, order, stream) != cudaSuccess) return KLA_ERR_LAUNCH;
             p.seq_order = order;
         }
+        mark(1); mark(2); mark(3);
         err = launch_chunk_tc(p, desc->d_k, desc->io_dtype, desc->out_dtype, stream);
     }
-    else
+    else {
+        mark(1); mark(2); mark(3);
         err = launch_chunk_simt(p, desc->d_k, chunk, desc->io_dtype, desc->out_dtype, stream);
+    }
+    mark(4);
     return err == cudaSuccess ? KLA_OK : KLA_ERR_LAUNCH;
 }
+
+extern "C" {
+
+kla_status kla_chunk_fwd(const kla_desc *desc, const void *q, const void *k, const void *v,
+                         const float *log_alpha, const float *eta, float eps, int32_t chunk,
+                         const float *init_state, void *out, float *final_state)
+{
+    return chunk_fwd_impl(desc, q, k, v, log_alpha, eta, eps, chunk, init_state, out, final_state, nullptr);
+}
+
+kla_status kla_chunk_fwd_timed(const kla_desc *desc, const void *q, const void *k, const void *v,
+                               const float *log_alpha, const float *eta, float eps, int32_t chunk,
+                               const float *init_state, void *out, float *final_state, float *pass_ms)
+{
+    if (!pass_ms) return KLA_ERR_NULL;
+    for (int i = 0; i < 4; ++i) pass_ms[i] = 0.f;
+    // validated here as well, so that nothing is created for a call that will be refused
+    kla_status st = check_chunk_args(desc, q, k, v, log_alpha, eta, eps, chunk, init_state, out, final_state, true);
+    if (st != KLA_OK) return st;
+    cudaEvent_t ev[5];
+    int made = 0;
+    for (; made < 5; ++made)
+        if (cudaEventCreate(&ev[made]) != cudaSuccess) break;
+    if (made == 5) {
+        st = chunk_fwd_impl(desc, q, k, v, log_alpha, eta, eps, chunk, init_state, out, final_state, ev);
+        if (st == KLA_OK && desc->T > 0) {
+            if (cudaStreamSynchronize((cudaStream_t)desc->stream) != cudaSuccess) st = KLA_ERR_LAUNCH;
+            for (int i = 0; st == KLA_OK && i < 4; ++i)
+                if (cudaEventElapsedTime(&pass_ms[i], ev[i], ev[i + 1]) != cudaSuccess) pass_ms[i] = 0.f;
+            // passes that did not run: their marks were recorded back to back
+            const bool segments = plan_segments(desc, chunk).G >= 2;
+            if (!segments) pass_ms[1] = pass_ms[2] = 0.f;
+            if (!segments && !order_bytes(desc, chunk)) pass_ms[0] = 0.f;
+        }
+    } else {
+        st = KLA_ERR_LAUNCH;
+    }
+    for (int i = 0; i < made; ++i) cudaEventDestroy(ev[i]);
+    (void)cudaGetLastError();
+    return st;
+}
+
 
 static kla_status check_decode(const kla_desc *d, const void *q, const void *k, const void *v,
                                const float *log_alpha, const float *eta, float eps,
@@ -282,6 +339,7 @@ const char *kla_status_str(kla_status s)
         case KLA_ERR_LAUNCH: return "CUDA launch failed";
         case KLA_ERR_TIMEOUT: return "a bounded device-side wait expired";
         case KLA_ERR_ARCH: return "device is not sm_100";
+        case KLA_ERR_DEVICE: return "current device could not be queried or its scratch address is unavailable";
     }
     return "unknown status";
 }

@@ -40,9 +40,6 @@
 #include <cuda.h>
 
 #include <cstddef>
-#include <cstdio>
-#include <cstdlib>
-#include <cstring>
 #include <mutex>
 
 #include "common.cuh"
@@ -176,16 +173,6 @@ __device__ __forceinline__ bool pg_any(bool flag)
     return r != 0;
 }
 
-#ifdef KLA_TRACE
-// role r (0 control, 1 pre, 2 chain), chunk c, event e -> trace[(r * 64 + c) * 16 + e]
-#define KLA_TR(r, c, e)                                                                        \
-    do {                                                                                       \
-        if (p.trace && blockIdx.x == 0 && (c) < 64 && (((r) == 0 && lane == 0) || ((r) == 1 && tid == PG_BASE) || ((r) == 2 && tid == CG_BASE))) \
-            p.trace[((r) * 64 + (c)) * 16 + (e)] = clock64();                                  \
-    } while (0)
-#else
-#define KLA_TR(r, c, e) do { } while (0)
-#endif
 
 // 4 x 4 transpose over the four lanes of a quad (t = lane & 3): on entry lane t holds v[j] = element (t, j), on
 // exit v[s] = element (s, t).  Two butterfly stages; every lane of the warp must call it.
@@ -616,9 +603,7 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 const uint32_t ph = (uint32_t)(c & 1);
                 const uint32_t k0 = d_kq0 + (uint32_t)(c % NSTAGE) * STAGE_STEP;
                 const uint32_t kt0 = d_kt0 + (uint32_t)(c % NSTAGE) * STAGE_STEP;
-                KLA_TR(0, c, 0);
                 if (!(ok = wwait(B_S_READY, ph))) break;
-                KLA_TR(0, c, 1);
                 tc_fence_after();
                 mma_xs(tmem + TM_KS, k0, 0, 0, 2 * KB);
                 mma_commit(&sm.bar[B_D2_DONE]);
@@ -636,12 +621,9 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     mma_xs(tmem + ((c & 1) ? TM_QS1 : TM_QS0), k0, 512, 0, KB);
                     qs_done = KB;
                 }
-                KLA_TR(0, c, 2);
                 // MMA-3(c): U = T rhs
                 if (!(ok = wwait(B_T_READY, ph))) break;
-                KLA_TR(0, c, 3);
                 if (!(ok = wwait(B_RHS_READY, ph))) break;
-                KLA_TR(0, c, 4);
                 tc_fence_after();
                 mma_3(tmem + TM_U, d_th, d_tl, d_rh, d_rl);
                 bool signal = true;
@@ -656,10 +638,8 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 if (qs_done < 2 * KB) mma_xs(tmem + ((c & 1) ? TM_QS1 : TM_QS0), k0, 512, qs_done, 2 * KB);
                 if (m1_due)
                     if (!(ok = mma1_own(cn))) break;
-                KLA_TR(0, c, 5);
                 // MMA-5(c): K^T (D U)
                 if (!(ok = wwait(B_U_READY, ph))) break;
-                KLA_TR(0, c, 6);
                 tc_fence_after();
 #pragma unroll 1
                 for (int t = 0; t < 2; ++t) KLA_SEQ(tmem + TM_DS, kt0, 128, t ? d_dl : d_dh, 128, ID_DS, t);
@@ -672,7 +652,6 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     mma_commit(&sm.bar[B_D4_DONE]);
                     if (c + 1 < nchunks) mma_commit_multicast(&sm.bar[B_P_FREE0 + (c & 1)], 3);   // as for T_FREE
                 }
-                KLA_TR(0, c, 7);
                 // (the chain group, which sees MMA-5(c) complete first, refills the K/Q stage of chunk c)
             }
         } else {
@@ -691,22 +670,17 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             const uint32_t ph = (uint32_t)(c & 1);
             const uint32_t k0 = d_kq0 + (uint32_t)(c % NSTAGE) * STAGE_STEP;
             const uint32_t kt0 = d_kt0 + (uint32_t)(c % NSTAGE) * STAGE_STEP;
-            KLA_TR(0, c, 0);
             // MMA-2(c): K S_0 -> TM_KS (on the chain), then Q S_0 -> TM_QS[c&1] (needed only for the outputs)
             if (!(ok = wwait(B_S_READY, ph))) break;
-            KLA_TR(0, c, 1);
             tc_fence_after();
 #pragma unroll 1
             for (int x = 0; x < (no_out ? 1 : 2); ++x) {
                 mma_xs(tmem + (x == 0 ? TM_KS : ((c & 1) ? TM_QS1 : TM_QS0)), k0, x * 512, 0, 2 * KB);
                 if (x == 0) mma_commit(&sm.bar[B_D2_DONE]);
             }
-            KLA_TR(0, c, 2);
             // MMA-3(c): U = T rhs
             if (!(ok = wwait(B_T_READY, ph))) break;
-            KLA_TR(0, c, 3);
             if (!(ok = wwait(B_RHS_READY, ph))) break;
-            KLA_TR(0, c, 4);
             if (c + 1 < nchunks) issue_tma_v(c + 1);
             tc_fence_after();
             mma_3(tmem + TM_U, d_th, d_tl, d_rh, d_rl);
@@ -716,10 +690,8 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             } else {
                 mma_commit(&sm.bar[B_D3_DONE]);
             }
-            KLA_TR(0, c, 5);
             // MMA-5(c): K^T (D U)   then   MMA-4(c): P U
             if (!(ok = wwait(B_U_READY, ph))) break;
-            KLA_TR(0, c, 6);
             tc_fence_after();
             // A = K^T: M = d_k (64-wide blocks KB*8192 bytes apart; for d_k = 64 the second block
             // is the Q tile, whose rows land in TMEM lanes 64..127 and are ignored), K = tokens
@@ -732,7 +704,6 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 mma_3(tmem + TM_PU, d_ph, d_pl, d_dh, d_dl);
                 mma_commit(&sm.bar[B_D4_DONE]);
             }
-            KLA_TR(0, c, 7);
             // the K/Q stage of chunk c is free once MMA-5(c) has read it
             if (c + NSTAGE < nchunks) {
                 if (!(ok = wwait(B_D5_DONE, ph))) break;
@@ -778,7 +749,6 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 decay_scan(sm, sc, lane, la0, la1);
                 fence_async_smem();   // gam and dec are also copied to the peer
             }
-            KLA_TR(1, c, 0);
             bool okc = okp;
             if (rows < C && okc) {
                 okc = wait(B_FULL0 + sc, (uint32_t)((c / NSTAGE) & 1));
@@ -793,11 +763,9 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 
             const int b1 = (c >> 1) & 1;                       // D1 buffer of this CTA's chunk c, ...
             const uint32_t ph1 = (uint32_t)((c >> 2) & 1);     // ... in its (c / 4)-th use
-            KLA_TR(1, c, 9);
             if (is_g) {
                 // ---- X = A^- o K K^T (this thread: row i, 32 columns) and beta_i, Eq. 3 ----------------------
                 okc = wait(B_D1_DONE0 + b1, ph1);
-                KLA_TR(1, c, 10);
                 if (okc) {
                     tc_fence_after();
                     if (live) {
@@ -808,7 +776,6 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                             fence_async_smem();
                         }
                     }
-                    KLA_TR(1, c, 11);
                     tc_fence_before();
                     warp_arrive(B_D1_FREE0 + b1);
                 }
@@ -816,7 +783,6 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 warp_arrive(B_D1_FREE0 + b1);   // nothing reads Q K^T
             }
             if (pg_any(!okc)) break;
-            KLA_TR(1, c, 1);
             // The per-token scalars of chunk c (beta, gamma, exp(g_C - g)) go to both chains now, more than a chunk
             // period before T(c): their rhs does not wait for the inverse.  (The peer's slot c mod 3 is free: its
             // chain read the scalars of chunk c - 3 before MMA-3(c-3), which this group saw complete two chunks ago.)
@@ -833,18 +799,13 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             const float *bet = sm.beta[sc];
             if (pt < 64) substitute_diag_blocks(sm.tl, bet, pt);
             pg_sync();
-            KLA_TR(1, c, 2);
             merge_level<8>(sm.tl, sm.mm, bet, pt);
-            KLA_TR(1, c, 6);
             merge_level<16>(sm.tl, sm.mm, bet, pt);
-            KLA_TR(1, c, 7);
             merge_level<32>(sm.tl, sm.mm, bet, pt);
-            KLA_TR(1, c, 3);
             // ---- T as bf16 hi/lo operand tiles, once MMA-3(c-1) of both CTAs has read the previous ones ------------
             bool okd = true;
             if (c > 0 && pt >= PG_T - 32) okd = wait(B_T_FREE0 + ((c - 1) & 1), (uint32_t)(((c - 1) >> 1) & 1));
             if (pg_any(!okd)) break;
-            KLA_TR(1, c, 4);
             write_t_tiles(sm, pt);
             fence_async_smem();
             pg_sync();  // every tile write is done (and the solve matrix may be reused by this CTA's next chunk)
@@ -855,7 +816,6 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 bulk_copy_to_cluster(smem_u32(sm.t_hi) + peer_off, smem_u32(sm.t_hi), 16384, rbar);   // t_hi and t_lo
                 mbar_arrive(&sm.bar[B_T_READY]);
             }
-            KLA_TR(1, c, 5);
 
             // ---- P(c) = A o Q K^T as bf16 hi/lo operand tiles into both CTAs (rows of Q K^T: warps 2, 3, 6, 7) --------
             if (!is_g && !no_out) {
@@ -878,7 +838,6 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     mbar_arrive(&sm.bar[B_P_READY]);
                 }
             }
-            KLA_TR(1, c, 12);
         }
     } else if (warp >= PG_BASE / 32) {
         // =============================== pre group ==========================================================
@@ -956,7 +915,6 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             if (scan_warp) {
                 decay_scan(sm, sc, lane, la0, la1);
             }
-            KLA_TR(1, c, 0);
             bool okc = true;
             if (rows < C) {
                 // last chunk: rows past the end of the sequence hold a neighbour's tokens (or TMA zero
@@ -969,11 +927,9 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 }
             }
             if (pg_any(!okc)) break;   // also publishes the decay sums to the whole group
-            KLA_TR(1, c, 9);
             if (is_g) {
                 // ---- X = A^- o K K^T from MMA-1 (this thread: row i, 32 columns) and beta_i ----------------------------
                 okc = wait(B_D1_DONE0 + (c & 1), (uint32_t)((c >> 1) & 1));
-                KLA_TR(1, c, 10);
                 if (okc) {
                     tc_fence_after();
                     if (live) {
@@ -985,7 +941,6 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                             else sm.beta[sc][i] = (i < rows) ? eta_cur / (dg + p.eps) : 0.f;
                         }
                     }
-                    KLA_TR(1, c, 11);
                     tc_fence_before();
                     warp_arrive(B_D1_FREE0 + (c & 1));
                 }
@@ -1008,24 +963,17 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 okc = form_p(c - 1);
             }
             if (pg_any(!okc)) break;   // X, the diagonal blocks and P(c-1) are done
-            KLA_TR(1, c, 1);
 
             // ---- then the off-diagonal blocks T_10 = -T_11 (B_1 X_10 T_00) at block sizes 8, 16, 32 -------------------
             const float *bet = sm.beta[sc];
-            KLA_TR(1, c, 2);
             merge_level<8>(sm.tl, sm.mm, bet, pt);
-            KLA_TR(1, c, 6);
             merge_level<16>(sm.tl, sm.mm, bet, pt);
-            KLA_TR(1, c, 7);
             merge_level<32>(sm.tl, sm.mm, bet, pt);
             // ---- write T as bf16 hi/lo operand tiles, after MMA-3(c-1) has read the previous ones ----------------------
-            KLA_TR(1, c, 3);
-            KLA_TR(1, c, 4);
             write_t_tiles(sm, pt);
             fence_async_smem();
             pg_sync();  // the solve matrix is reused by the next chunk
             warp_arrive(B_T_READY);
-            KLA_TR(1, c, 5);
         }
         // P of the last chunk
         if (c == nchunks && !is_g && !no_out) form_p(nchunks - 1);
@@ -1082,16 +1030,13 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             const int rows = (c == nchunks - 1) ? last_rows : C;
             const int sc = c % NSTAGE;
             // ---- rhs = B (V - D_gamma K S_0) ------------------------------------------------------------------
-            KLA_TR(2, c, 0);
             if (!(PAIR ? wait(B_SCAL_READY0 + (c & 3), (uint32_t)((c >> 2) & 1)) : wait(B_T_READY, ph))) break;   // scalars of chunk c
-            KLA_TR(2, c, 1);
             const float b0 = sm.beta[sc][i0], b1 = sm.beta[sc][i1];
             const float g0 = sm.gam[sc][i0], g1 = sm.gam[sc][i1];
             const float d0 = sm.dec[sc][i0], d1 = sm.dec[sc][i1];
             const float gC = sm.gam[sc][C - 1];
             if (!wait(B_V_FULL, ph)) break;
             if (!wait(B_D2_DONE, ph)) break;
-            KLA_TR(2, c, 2);
             tc_fence_after();
 #pragma unroll 1
             for (int j = 0; j < 4; ++j) {
@@ -1114,11 +1059,9 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             fence_async_smem();
             tc_fence_before();
             warp_arrive(B_RHS_READY);
-            KLA_TR(2, c, 3);
 
             // ---- D U as hi/lo operand: of the state update and, against P D^-1, of the outputs --------------------------------
             if (!wait(B_D3_DONE, ph)) break;
-            KLA_TR(2, c, 4);
             tc_fence_after();
 #pragma unroll 1
             for (int j = 0; j < 4; ++j) {
@@ -1136,11 +1079,9 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             fence_async_smem();
             tc_fence_before();
             warp_arrive(B_U_READY);
-            KLA_TR(2, c, 5);
 
             // ---- state: S <- gamma_C S + K^T (D U) -----------------------------------------------------------------
             if (!wait(B_D5_DONE, ph)) break;
-            KLA_TR(2, c, 6);
             if constexpr (PAIR) {
                 // MMA-5(c) was the last reader of the K/Q stage of chunk c: refill it at once (this CTA's MMA-1 of
                 // chunk c + 3 may be due within a fraction of a chunk period)
@@ -1165,12 +1106,10 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             }
             tc_fence_before();
             if (c + 1 < nchunks) store_state_tiles();
-            KLA_TR(2, c, 7);
 
             // ---- outputs: O_i = gamma_i (Q S_0)_i + (P U)_i (off the chain) -----------------------------------------
             if (no_out) continue;
             if (!wait(B_D4_DONE, ph)) break;
-            KLA_TR(2, c, 8);
             tc_fence_after();
             {
                 // This thread's accumulator values are column pairs cp + 8j (j = 0..3) of rows i0 and i1; a 4 x 4 transpose
@@ -1228,7 +1167,6 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 }
             }
             tc_fence_before();
-            KLA_TR(2, c, 9);
         }
         if (!sm.abort_flag && fin && s_act) {
 #pragma unroll
@@ -1294,7 +1232,7 @@ cudaError_t launch_v(const ChunkParams &p, cudaStream_t stream);
 template <int D, typename OUT>
 cudaError_t launch_t(const ChunkParams &p, cudaStream_t stream)
 {
-    const int32_t v = p.variant & ~VARIANT_NO_PAIR;
+    const int32_t v = p.variant & ~(VARIANT_NO_PAIR | VARIANT_WY);
     // two slices per head: the CTAs of a head run as a cluster and share the state-independent work (the layer-edge
     // variants are implemented in the unpaired kernel only; the error-path test hook in both)
     if constexpr (D == 2 * NS) {
@@ -1334,30 +1272,6 @@ cudaError_t launch_v(const ChunkParams &p, cudaStream_t stream)
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = PAIR ? 1 : 0;
-#ifdef KLA_TRACE
-    {
-        static long long *tbuf = nullptr;
-        if (!tbuf) cudaMallocManaged(&tbuf, 3 * 64 * 16 * sizeof(long long));
-        memset(tbuf, 0, 3 * 64 * 16 * sizeof(long long));
-        ChunkParams pt = p;
-        pt.trace = tbuf;
-        cudaLaunchKernelEx(&cfg, kern, tq, tk, tv, pt);
-        cudaDeviceSynchronize();
-        const char *tf = getenv("KLA_TRACE_FILE");
-        FILE *f = tf ? fopen(tf, "w") : nullptr;
-        if (f) {
-            for (int r = 0; r < 3; ++r)
-                for (int c = 0; c < 64; ++c) {
-                    fprintf(f, "%d %d", r, c);
-                    for (int e = 0; e < 16; ++e) fprintf(f, " %lld", tbuf[(r * 64 + c) * 16 + e]);
-                    fprintf(f, "\n");
-                }
-            fclose(f);
-        }
-        count_launch(1);
-        return cudaGetLastError();
-    }
-#endif
     err = cudaLaunchKernelEx(&cfg, kern, tq, tk, tv, p);
     count_launch(1);
     return err != cudaSuccess ? err : cudaGetLastError();
@@ -1373,6 +1287,7 @@ bool chunk_tc_supported(int d, int chunk, int io_dtype)
 cudaError_t launch_chunk_tc(const ChunkParams &p, int d, int io_dtype, int out_dtype, cudaStream_t stream)
 {
     (void)io_dtype;
+    if (d == 128 && (p.variant & VARIANT_WY)) return launch_chunk_wy(p, out_dtype, stream);
     if (d == 128) {
         if (out_dtype == KLA_BF16) return launch_t<128, __nv_bfloat16>(p, stream);
         return launch_t<128, float>(p, stream);

@@ -1,0 +1,1112 @@
+// Chunkwise forward, head dimension 128, in the WY form (Algorithm 1 right; Eqs. 7-9; Props. 5-6 and the combined
+// WY representation of Appendix B): with T = (I + B (A^- o K K^T))^-1,
+//
+//     U = T B V,   W = T B D_gamma K      (independent of the state: formed off the serial chain)
+//     U^ = U - W S_0                      (the solution of Eq. 7)
+//     O  = D_gamma Q S_0 + (A o Q K^T) U^ (Eq. 8)
+//     S <- gamma_C S_0 + K^T diag(exp(g_C - g_j)) U^   (Eq. 9)
+//
+// so that the serial dependency from chunk to chunk is two tensor-core products (W S_0, then K^T (D U^)) and two
+// register passes, not three and three.
+//
+// The two CTAs that hold the two 64-column slices of one (sequence, head) run as a thread-block cluster of two.
+// Everything that depends on the head only is computed once per chunk, by the CTA whose rank equals the chunk's
+// parity (its "owner"), and handed to both: the per-token scalars, T B (operand of U, bf16 hi/lo tiles), W (fp16
+// tile) and P D^-1 (P = A o Q K^T, bf16 hi/lo tiles) travel to the peer's shared memory with cp.async.bulk
+// (shared::cta -> shared::cluster, no multicast), counted on the peer's mbarriers as transaction bytes.
+//
+// Roles (21 warps):
+//   control warp            every TMA load of K/Q tiles and every tcgen05.mma, in a fixed order
+//   chain group (8 warps)   the serial dependency: D U^ from the accumulator of U - W S_0, the state update, outputs
+//   pre group (8 warps)     own chunks: decay scan, X = A^- o K K^T and beta (Eq. 3) from the Gram accumulator, the
+//                           blocked inverse in shared memory, then T B D_gamma (operand of W) and T B as bf16 hi/lo tiles
+//   aux group (4 warps)     every chunk: the Q tile to fp16 (per-row power-of-two scale); own chunks: W from its
+//                           accumulator to the fp16 tile, and P D^-1
+//
+// Tensor-core products per chunk and CTA (fp32 accumulation in TMEM):
+//   [K;Q] K^T  M=128  bf16                    owner only
+//   (T B D_gamma) K   M=64 N=128, 2 terms     owner only  -> W
+//   (T B) V_slice     M=64, 2 terms           -> accumulator of U^
+//   (-W) S_0          M=64, fp16, 1 term      accumulated on top: U^ = U - W S_0            (on the chain)
+//   Q S_0             M=64, fp16, 2 terms     Q converted in place after the Gram product has read it
+//   K^T (D U^)        M=128, bf16, 2 terms                                                  (on the chain)
+//   (P D^-1)(D U^)    M=64, bf16, 3 terms
+//
+// Precision.  q, k, v enter every product exactly (the fp16 copy of Q carries a per-row power-of-two scale, so it
+// is exact down to 2^-28 of the row's largest entry).  Operands on the read-out path and in the state update
+// (S_0 against Q, T B, P D^-1, D U^) need 16 significand bits and are hi/lo pairs; W S_0 only corrects U by what the
+// incoming state already predicts, and an 11-bit W and S_0 there (fp16, one term) keeps the layer-shaped workloads
+// below 1e-3 in max|err|/rms.  The state and W must stay inside the fp16 range (|x| < 65504); beyond it the result
+// is Inf/NaN, never silently wrong.  Inputs with heavy-tailed key norms want all-16-bit operands: KLA_FLAG_NO_PAIR
+// routes to the kernel of chunk_tc.cu, which has them.
+//
+// Every wait on an mbarrier is bounded; when one gives up the CTA raises an abort flag, reports KLA_ERR_TIMEOUT
+// through the status word, releases its TMEM and exits.
+#include <cuda_fp16.h>
+
+#include <cstddef>
+
+#include "chunk_pieces.cuh"
+
+namespace kla {
+
+namespace {
+
+using namespace tc;
+
+constexpr int CG_T = 256, PG_T = 256, AG_T = 128;
+constexpr int NT = 32 + CG_T + PG_T + AG_T + 64;   // 736
+// warp 0 chain issuer, warps 1..8 chain group, 9..16 pre group, 17..20 aux group, 21 output issuer, 22 owner issuer
+constexpr int CG_BASE = 32, PG_BASE = CG_BASE + CG_T, AG_BASE = PG_BASE + PG_T;
+constexpr int OI_WARP = (AG_BASE + AG_T) / 32;
+constexpr int NSC = 4;   // depth of the per-token scalar slots (see the pre group)
+constexpr int RST = 2;   // K/Q stages of the chain
+
+// TMEM columns (fp32, 128 lanes each)
+constexpr uint32_t TM_D1E = 0 /* K K^T of an own chunk, two chunks ahead */, TM_D1L = 64 /* [K;Q] K^T of an own chunk, for P */, TM_W = 128 /* 128 columns */, TM_UH = 256, TM_QS = 320, TM_PU = 384,
+                   TM_DS = 448, TM_COLS = 512;
+
+enum Bar {
+    B_FULL0 = 0,          // +stage: K/Q tiles landed
+    B_EFULL = 2,          // early K tile of an own chunk landed
+    B_ETAIL = 3,          // its rows past the end of the sequence zeroed (last chunk)
+    B_D1E_DONE = 4,       // K K^T of an own chunk complete (pre group)
+    B_D1E_FREE = 5,       // X formed: the accumulator may be overwritten
+    B_D1L_DONE = 6,       // [K;Q] K^T of an own chunk complete (aux group: Q conversion, P)
+    B_V_FULL = 7,         // V slice of chunk c landed
+    B_VTAIL = 8,          // rows of the V slice past the end of the sequence zeroed (last chunk)
+    B_TAIL_READY = 9,     // rows of the K and Q tiles past the end of the sequence zeroed (last chunk)
+    B_D1L_FREE = 10,      // P formed: the accumulator may be overwritten
+    B_TBG_READY = 12,     // T B D_gamma tiles of an own chunk written
+    B_W_DONE = 13,        // W accumulator of an own chunk complete (waited on by the pre and the aux group)
+    B_W_EMPTY = 14,       // aux group has read the W accumulator
+    B_T_READY = 15,       // T B tiles of chunk c present (own: local arrival; peer's: its copy)
+    B_W_READY = 16,       // W tile of chunk c present
+    B_P_READY = 17,       // P D^-1 tiles of chunk c present
+    B_S_READY = 18,       // state tiles for chunk c written
+    B_UH_DONE = 19,       // U - W S_0 of chunk c complete
+    B_DU_READY = 20,      // D U^ tiles written
+    B_DS_DONE = 21,       // K^T (D U^) complete (and every earlier product, Q S_0 among them)
+    B_D4_DONE = 22,       // (P D^-1)(D U^) complete
+    B_OUT_READ = 23,      // chain group has read the Q S_0 and P U accumulators of chunk c
+    // Signals from the tensor pipes of both CTAs (count 2).  A wait tells a phase only from its neighbours and nothing
+    // bounds how far one CTA runs ahead of the other, so each is waited on, phase after phase, by one role of one CTA:
+    B_T_FREE0 = 24,       // +(c & 1): (T B) V of chunk c complete in both CTAs; pre group of the owner of chunk c + 1
+    B_W_FREE0 = 26,       // +(c & 1): W S_0 of chunk c complete in both CTAs; aux group of the owner of chunk c + 1
+    B_P_FREE0 = 28,       // +(c & 1): P U of chunk c complete in both CTAs; aux group of the owner of chunk c + 1
+    B_SCAL_READY0 = 30,   // +(c & 3): gamma, exp(g_C - g) of chunk c present
+    // The Q conversion only needs the tiles to have landed, so it can run up to three chunks ahead of its readers; a
+    // slot is reused once the stage of chunk c + 1 has been refilled, which both readers of chunk c precede:
+    B_QCONV0 = 34,        // +(c & 3): Q tile of chunk c converted (waited on by the control warp)
+    B_QSC0 = 38,          // +(c & 3): the same event for the chain group, which reads the per-row scales
+    B_TV_DONE = 42,       // (T B) V of chunk c complete (output issuer -> chain issuer)
+    B_QS_DONE = 43,       // Q S_0 of chunk c complete (output issuer -> chain group: the state tiles may be rewritten)
+    B_COUNT = 44
+};
+
+template <int D>
+struct WySmem {
+    static constexpr int KB = D / 64;               // 64-wide blocks along d_k
+    static constexpr int KQ_BYTES = KB * 2 * 8192;  // [K kb0][Q kb0][K kb1][Q kb1], 8 KB each
+    // all tile bases are multiples of 1024 bytes (128-byte swizzle atom = 8 rows x 128 B)
+    alignas(1024) unsigned char kq[RST][KQ_BYTES];
+    alignas(1024) unsigned char ke[KB * 8192];   // K tile of this CTA's next chunk, loaded two chunks ahead: [K kb0][K kb1]
+    alignas(1024) unsigned char s_hi[D * 128];   // state slice, D rows (d_k) x 64 fp16: S ~ s_hi + s_lo
+    alignas(1024) unsigned char s_lo[D * 128];
+    alignas(1024) unsigned char t_hi[8192];      // T B: 64 x 64 bf16, K-major
+    alignas(1024) unsigned char t_lo[8192];
+    alignas(1024) unsigned char tg_hi[8192];     // T B D_gamma (own chunks only)
+    alignas(1024) unsigned char tg_lo[8192];
+    alignas(1024) unsigned char p_hi[8192];      // P D^-1
+    alignas(1024) unsigned char p_lo[8192];
+    alignas(1024) unsigned char w16[KB * 8192];  // -W: 64 tokens x d_k fp16, K-major, one 8 KB block per 64 of d_k
+    alignas(1024) unsigned char du_hi[8192];     // D U^: 64 tokens x 64 bf16, MN-major
+    alignas(1024) unsigned char du_lo[8192];
+    alignas(1024) unsigned char vt[8192];        // V slice of one chunk, MN-major
+    alignas(16) float tl[64 * LDT];              // X = A^- o K K^T, overwritten in place by T; the never-used block of
+                                                 // rows 0..31 x columns 32..63 is the scratch of the block products
+    alignas(16) float g2[NSC][64];               // log2(e) * chunk-local running sum of log alpha (owner only)
+    float beta[NSC][64];                         // (owner only)
+    float gam[NSC][64];                          // exp(g_i)
+    float dec[NSC][64];                          // exp(g_C - g_i), floored
+    float qsc[NSC][64];                          // 1 / (power-of-two scale of row i of the fp16 Q tile)
+    float qn[NSC][64];                           // 1 / ||q_i|| (normalised read-out only)
+    alignas(8) uint64_t bar[B_COUNT];
+    uint32_t tmem_base;
+    volatile int abort_flag;
+};
+
+// Barrier over the aux group (128 threads) that also ORs a flag, so that leaving the loop after a wait gave up is a
+// collective decision and no thread is left alone at a later barrier.
+__device__ __forceinline__ bool ag_any(bool flag)
+{
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 p, %1, 0;\n\t"
+        "bar.red.or.pred q, 6, 128, p;\n\tselp.u32 %0, 1, 0, q;\n\t}"
+        : "=r"(r)
+        : "r"((uint32_t)flag)
+        : "memory");
+    return r != 0;
+}
+
+// Instruction descriptor for kind::f16 with fp16 operands and fp32 accumulation.
+__host__ __device__ constexpr uint32_t idesc_f16(int M, int N, int a_mn, int b_mn)
+{
+    return (1u << 4) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+// x ~= hi + lo with hi = fp16(x), lo = fp16(x - hi).
+__device__ __forceinline__ void split2h(float a, float b, uint32_t &hi, uint32_t &lo)
+{
+    const __half2 h = __floats2half2_rn(a, b);
+    const float2 hf = __half22float2(h);
+    const __half2 l = __floats2half2_rn(a - hf.x, b - hf.y);
+    hi = *reinterpret_cast<const uint32_t *>(&h);
+    lo = *reinterpret_cast<const uint32_t *>(&l);
+}
+
+
+// ---- the blocked inverse of I + B X on the warp-level tensor instruction ------------------------------------------------------
+// The block products T_10 = -T_11 (B_1 X_10 T_00) at block sizes 16 and 32 are small dense products whose operands sit
+// in shared memory in fp32.  With CUDA-core FMAs every multiply-add fetches its operands from shared memory again (the
+// products then take most of the pre group's time and most of the SM's shared-memory bandwidth, which the tcgen05 products
+// need for their operand tiles); mma.sync m16n8k16 takes whole fragments into registers once.  Operands are split into
+// bf16 hi/lo pairs in registers and multiplied in three terms, accumulated in fp32.
+__device__ __forceinline__ void mma_16816(float (&c)[4], const uint32_t (&a)[4], const uint32_t (&b)[2])
+{
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
+}
+// c (16 x 8) += A (16 x K, rows lda floats apart) . B (K x 8, rows ldb floats apart), both fp32 in shared memory.  Fragment
+// layout of the instruction (g = lane / 4, t = lane % 4): c[0,1] = C[g][2t, 2t+1], c[2,3] = C[g+8][2t, 2t+1].
+__device__ __forceinline__ void warp_tile_product(float (&c)[4], int K, const float *Ap, int lda, const float *Bp, int ldb, int lane)
+{
+    const int g = lane >> 2, t = lane & 3;
+    float c1[4] = {0.f, 0.f, 0.f, 0.f}, c2[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 1
+    for (int k0 = 0; k0 < K; k0 += 16) {
+        const float2 a00 = *reinterpret_cast<const float2 *>(Ap + g * lda + k0 + 2 * t);
+        const float2 a10 = *reinterpret_cast<const float2 *>(Ap + (g + 8) * lda + k0 + 2 * t);
+        const float2 a01 = *reinterpret_cast<const float2 *>(Ap + g * lda + k0 + 2 * t + 8);
+        const float2 a11 = *reinterpret_cast<const float2 *>(Ap + (g + 8) * lda + k0 + 2 * t + 8);
+        const float b0 = Bp[(k0 + 2 * t) * ldb + g], b1 = Bp[(k0 + 2 * t + 1) * ldb + g];
+        const float b2 = Bp[(k0 + 2 * t + 8) * ldb + g], b3 = Bp[(k0 + 2 * t + 9) * ldb + g];
+        uint32_t ah[4], al[4], bh[2], bl[2];
+        split2(a00.x, a00.y, ah[0], al[0]);
+        split2(a10.x, a10.y, ah[1], al[1]);
+        split2(a01.x, a01.y, ah[2], al[2]);
+        split2(a11.x, a11.y, ah[3], al[3]);
+        split2(b0, b1, bh[0], bl[0]);
+        split2(b2, b3, bh[1], bl[1]);
+        mma_16816(c, ah, bh);     // three accumulators: the instruction's latency is long, so the terms must not queue
+        mma_16816(c1, ah, bl);    // behind one another
+        mma_16816(c2, al, bh);
+    }
+#pragma unroll
+    for (int e = 0; e < 4; ++e) c[e] += c1[e] + c2[e];
+}
+// One level of the inverse (see merge_level in chunk_pieces.cuh for the algebra), block size BS = 16 or 32: every warp of
+// the pre group takes one 16 x 8 tile of the result (BS = 16: four tiles, warps 0..3; BS = 32: eight).  `mm` (rows LDT
+// floats apart) holds the intermediate product.  Out of line, one copy for both sizes: the pre group's code has to stay
+// small (instruction fetch is what the whole CTA stalls on first when the roles' loops outgrow the instruction cache).
+__device__ __noinline__ void merge_level_mma(int BS, float *tl, float *mm, const float *bet, int pw, int lane)
+{
+    const int NTL = BS / 8;                        // column tiles per block
+    const bool act = pw < (32 / BS) * (BS / 16) * NTL;
+    const int nt = pw % NTL, mt = (pw / NTL) % (BS / 16), pr = pw / (NTL * (BS / 16));
+    const int rb = (2 * pr + 1) * BS, cb = 2 * pr * BS;
+    const int g = lane >> 2, t = lane & 3;
+    if (act) {
+        // M = B_1 X_10 T_00
+        float c[4] = {0.f, 0.f, 0.f, 0.f};
+        warp_tile_product(c, BS, tl + (rb + 16 * mt) * LDT + cb, LDT, tl + cb * LDT + cb + 8 * nt, LDT, lane);
+        const float s0 = bet[rb + 16 * mt + g], s1 = bet[rb + 16 * mt + g + 8];
+        float *d = mm + (pr * BS + 16 * mt + g) * LDT + 8 * nt + 2 * t;
+        *reinterpret_cast<float2 *>(d) = make_float2(s0 * c[0], s0 * c[1]);
+        *reinterpret_cast<float2 *>(d + 8 * LDT) = make_float2(s1 * c[2], s1 * c[3]);
+    }
+    pg_sync();
+    if (act) {
+        // T_10 = -T_11 M
+        float c[4] = {0.f, 0.f, 0.f, 0.f};
+        warp_tile_product(c, BS, tl + (rb + 16 * mt) * LDT + rb, LDT, mm + (pr * BS) * LDT + 8 * nt, LDT, lane);
+        float *d = tl + (rb + 16 * mt + g) * LDT + cb + 8 * nt + 2 * t;
+        *reinterpret_cast<float2 *>(d) = make_float2(-c[0], -c[1]);
+        *reinterpret_cast<float2 *>(d + 8 * LDT) = make_float2(-c[2], -c[3]);
+    }
+    pg_sync();
+}
+// X = A^- o K K^T: this thread's row i, columns chh * 32 .. + 31 of the K K^T accumulator at tbase (two loads of 16
+// columns: four loads of eight paid the TMEM latency four times, one of 32 doubled the code), into the solve matrix.
+// Returns the diagonal element G_ii = ||k_i||^2 if it lies in these columns (else 0).
+template <typename Smem>
+__device__ __forceinline__ float form_x_row16(Smem &sm, int sc, int i, int chh, uint32_t tbase)
+{
+    const float gi2 = sm.g2[sc][i];
+    float dg = 0.f;
+#pragma unroll 1
+    for (int hh = 0; hh < 2; ++hh) {
+        float a[16];
+        tmem_ld16(tbase + hh * 16, a);
+#pragma unroll
+        for (int grp = 0; grp < 4; ++grp) {
+            const int j0 = chh * 32 + hh * 16 + grp * 4;
+            const float4 gj4 = *reinterpret_cast<const float4 *>(&sm.g2[sc][j0]);
+            const float gj[4] = {gj4.x, gj4.y, gj4.z, gj4.w};
+            float x[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                x[e] = (j0 + e < i) ? ex2_approx(gi2 - gj[e]) * a[grp * 4 + e] : 0.f;
+                dg = (j0 + e == i) ? a[grp * 4 + e] : dg;
+            }
+            *reinterpret_cast<float4 *>(&sm.tl[i * LDT + j0]) = make_float4(x[0], x[1], x[2], x[3]);
+        }
+    }
+    return dg;
+}
+
+// T (fp32, in the solve matrix) times a diagonal of column scales, as bf16 hi/lo operand tiles: thread pt writes 16
+// columns of row pt % 64.  GAMMA: column scale beta_j gamma_j (operand of W), else beta_j (operand of U).
+template <typename Smem>
+__device__ __noinline__ void write_t_tiles(Smem &sm, bool GAMMA, unsigned char *hi_tile, unsigned char *lo_tile, int sc, int pt)
+{
+    const int r = pt & 63, qq = pt >> 6;  // row, 16-column quarter
+#pragma unroll 1
+    for (int ch = 0; ch < 2; ++ch) {
+        const int j0 = qq * 16 + ch * 8;
+        uint4 hi = make_uint4(0, 0, 0, 0), lo = hi;
+        if (j0 <= r) {   // whole groups above the diagonal are zero (and one block of them holds scratch)
+            float t[8], s[8];
+            *reinterpret_cast<float4 *>(&t[0]) = *reinterpret_cast<const float4 *>(&sm.tl[r * LDT + j0]);
+            *reinterpret_cast<float4 *>(&t[4]) = *reinterpret_cast<const float4 *>(&sm.tl[r * LDT + j0 + 4]);
+            *reinterpret_cast<float4 *>(&s[0]) = *reinterpret_cast<const float4 *>(&sm.beta[sc][j0]);
+            *reinterpret_cast<float4 *>(&s[4]) = *reinterpret_cast<const float4 *>(&sm.beta[sc][j0 + 4]);
+            if (GAMMA) {
+                float g[8];
+                *reinterpret_cast<float4 *>(&g[0]) = *reinterpret_cast<const float4 *>(&sm.gam[sc][j0]);
+                *reinterpret_cast<float4 *>(&g[4]) = *reinterpret_cast<const float4 *>(&sm.gam[sc][j0 + 4]);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) s[e] *= g[e];
+            }
+#pragma unroll
+            for (int e = 0; e < 8; ++e) t[e] = (j0 + e <= r) ? t[e] * s[e] : 0.f;
+            split2(t[0], t[1], hi.x, lo.x);
+            split2(t[2], t[3], hi.y, lo.y);
+            split2(t[4], t[5], hi.z, lo.z);
+            split2(t[6], t[7], hi.w, lo.w);
+        }
+        *reinterpret_cast<uint4 *>(hi_tile + sw128(r, qq * 2 + ch)) = hi;
+        *reinterpret_cast<uint4 *>(lo_tile + sw128(r, qq * 2 + ch)) = lo;
+    }
+}
+
+// VAR: compiled with the layer-edge variants (beta = eta, read-out over ||q||) and the error-path test hook; the
+// default instantiation carries none of their code.
+template <int D, typename OUT, bool VAR>
+__global__ void __launch_bounds__(NT, 1)
+kla_chunk_wy_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                    const __grid_constant__ CUtensorMap tm_v, ChunkParams p)
+{
+    using Smem = WySmem<D>;
+    constexpr int KB = Smem::KB;
+    constexpr int SLICES = D / NS;
+    static_assert(SLICES == 2, "a cluster of two CTAs holds the two slices of a head");
+    constexpr uint32_t STAGE_BYTES = Smem::KQ_BYTES;
+    static_assert(sizeof(Smem) + 1024 <= 232448, "shared memory of one CTA");
+    static_assert(offsetof(Smem, t_lo) == offsetof(Smem, t_hi) + 8192 && offsetof(Smem, p_lo) == offsetof(Smem, p_hi) + 8192,
+                  "pairs copied as one must be contiguous");
+    constexpr uint32_t ID_G = idesc_bf16(128, 64, 0, 0);    // [K;Q] K^T : A K-major, B K-major
+    constexpr uint32_t ID_S = idesc_bf16(64, NS, 0, 1);     // (T B) V, (P D^-1)(D U^): M=64, B MN-major
+    constexpr uint32_t ID_W = idesc_bf16(64, D, 0, 1);      // (T B D_gamma) K: N = d_k
+    constexpr uint32_t ID_DS = idesc_bf16(128, NS, 1, 1);   // K^T (D U^): A MN-major, B MN-major
+    constexpr uint32_t ID_H = idesc_f16(64, NS, 0, 1);      // W S_0, Q S_0 (fp16)
+
+    extern __shared__ unsigned char smem_dyn[];
+    Smem &sm = *reinterpret_cast<Smem *>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t rank = cluster_ctarank();   // adjacent blocks = the two slices of one head
+    // plain launch: block = (sequence, head, slice).  Segment pass 1 doubles the slices (the second pair carries
+    // the transition map) and skips each sequence's last segment; see ChunkParams.
+    const int nslices = p.seg_pass == 1 ? 2 * SLICES : SLICES;
+    const int sl2 = blockIdx.x % nslices;
+    const bool is_map = sl2 >= SLICES;   // the same for both CTAs of a cluster
+    const int sl = sl2 % SLICES;
+    const int h = (blockIdx.x / nslices) % p.H;
+    int n = blockIdx.x / (nslices * p.H);
+    if (p.seg_pass == 1) n = (n / (p.seg_G - 1)) * p.seg_G + n % (p.seg_G - 1);
+    else if (p.seg_pass == 0 && p.seq_order) n = p.seq_order[n];   // packed input: longest sequences first
+    const bool no_out = p.seg_pass == 1;
+
+    int tok0, len;
+    if (p.cu_seqlens) {
+        tok0 = p.cu_seqlens[n];
+        len = p.cu_seqlens[n + 1] - tok0;
+    } else {
+        tok0 = n * p.T;
+        len = p.T;
+    }
+    const size_t state_off = (((size_t)n * p.H + h) * D) * D + (size_t)sl * NS;
+    // where this CTA's final state goes (null: nowhere)
+    float *fin = is_map ? p.map_state : p.final_state;
+    size_t fin_off = state_off;
+    if (p.seg_pass == 3 && fin) {
+        if (n % p.seg_G != p.seg_G - 1) fin = nullptr;
+        else fin_off = (((size_t)(n / p.seg_G) * p.H + h) * D) * D + (size_t)sl * NS;
+    }
+
+    if (len <= 0) {  // empty sequence (both CTAs of the cluster): the final state is the initial state
+        if (p.final_state) {
+            for (int i = tid; i < D * (NS / 4); i += NT) {
+                const int r = i / (NS / 4), c = (i % (NS / 4)) * 4;
+                float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (p.init_state) x = *reinterpret_cast<const float4 *>(p.init_state + state_off + (size_t)r * D + c);
+                *reinterpret_cast<float4 *>(p.final_state + state_off + (size_t)r * D + c) = x;
+            }
+        }
+        return;
+    }
+    const int nchunks = (len + C - 1) / C;
+    const int last_rows = len - (nchunks - 1) * C;
+    const bool tail = last_rows < C;
+
+    // ---- set-up ------------------------------------------------------------------------------------------
+    if (tid == 0) {
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&sm.bar[B_FULL0 + b], 1);
+            mbar_init(&sm.bar[B_T_FREE0 + b], 2);
+            mbar_init(&sm.bar[B_W_FREE0 + b], 2);
+            mbar_init(&sm.bar[B_P_FREE0 + b], 2);
+        }
+        mbar_init(&sm.bar[B_EFULL], 1);
+        mbar_init(&sm.bar[B_ETAIL], PG_T / 32);
+        mbar_init(&sm.bar[B_D1E_DONE], 1);
+        mbar_init(&sm.bar[B_D1E_FREE], 4);   // the four pre warps that hold rows of K K^T
+        mbar_init(&sm.bar[B_D1L_DONE], 1);
+        mbar_init(&sm.bar[B_D1L_FREE], 2);   // the two aux warps that hold rows of Q K^T
+        mbar_init(&sm.bar[B_V_FULL], 1);
+        mbar_init(&sm.bar[B_VTAIL], AG_T / 32);
+        mbar_init(&sm.bar[B_TAIL_READY], PG_T / 32);
+        mbar_init(&sm.bar[B_TBG_READY], PG_T / 32);
+        mbar_init(&sm.bar[B_W_DONE], 1);
+        mbar_init(&sm.bar[B_W_EMPTY], AG_T / 32);
+        // one arrival per chunk, local (own chunk) or from the peer together with the bytes of its copy
+        mbar_init(&sm.bar[B_T_READY], 1);
+        mbar_init(&sm.bar[B_W_READY], 1);
+        mbar_init(&sm.bar[B_P_READY], 1);
+        mbar_init(&sm.bar[B_S_READY], CG_T / 32);
+        mbar_init(&sm.bar[B_UH_DONE], 1);
+        mbar_init(&sm.bar[B_DU_READY], CG_T / 32);
+        mbar_init(&sm.bar[B_DS_DONE], 1);
+        mbar_init(&sm.bar[B_D4_DONE], 1);
+        mbar_init(&sm.bar[B_OUT_READ], CG_T / 32);
+        mbar_init(&sm.bar[B_TV_DONE], 1);
+        mbar_init(&sm.bar[B_QS_DONE], 1);
+        for (int b = 0; b < NSC; ++b) {
+            mbar_init(&sm.bar[B_SCAL_READY0 + b], 1);
+            mbar_init(&sm.bar[B_QCONV0 + b], AG_T / 32);
+            mbar_init(&sm.bar[B_QSC0 + b], AG_T / 32);
+        }
+        sm.abort_flag = 0;
+        mbar_fence_init();
+    }
+    // the block of the solve matrix above the diagonal blocks is never written by the inverse
+    for (int i = tid; i < 64 * LDT; i += NT) sm.tl[i] = 0.f;
+    if (warp == 0) tmem_alloc(&sm.tmem_base, TM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();   // the peer's barriers are initialised before anything arrives on them
+    tc_fence_after();
+    const uint32_t tmem = sm.tmem_base;
+    const uint32_t tm_lane = tmem + ((uint32_t)((warp & 3) * 32) << 16);  // this warp's 32 TMEM lanes
+
+    // Fast path inline (the phase is often complete already), polling loop out of line.  Called by whole warps; the
+    // outcome is made warp-uniform, because the warp-collective TMEM loads that follow a wait must not be reached by
+    // some lanes only (after an abort one lane may see the phase complete and another give up).
+    // The chain group reacts at once; the pre and aux groups work far ahead of the chain and look rarely.
+    const unsigned sleep_ns = (warp >= PG_BASE / 32) ? 256u : 32u;
+    auto wait = [&](int b, uint32_t parity) -> bool {
+        const bool ok = mbar_try_wait(&sm.bar[b], parity) || bar_wait(&sm.bar[b], parity, &sm.abort_flag, sleep_ns);
+        return __all_sync(0xffffffffu, ok);
+    };
+    // one arrival per warp, after the warp's shared-memory writes are visible to the async proxy
+    auto warp_arrive = [&](int b) {
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sm.bar[b]);
+    };
+    // distance from a shared-memory address of this CTA to the same location in the peer CTA
+    const uint32_t peer_off = mapa_u32(smem_u32(&sm), rank ^ 1u) - smem_u32(&sm);
+    // Publish `bytes` at `src` (already written here, visible to the async proxy) to both CTAs under barrier `b`: the
+    // peer's copy is sent by the copy engine and counted on its barrier; this CTA's barrier gets a plain arrival.
+    auto publish = [&](int b, const void *src, uint32_t bytes) {
+        const uint32_t rbar = smem_u32(&sm.bar[b]) + peer_off;
+        mbar_arrive_expect_tx_cluster(rbar, bytes);
+        bulk_copy_to_cluster(smem_u32(src) + peer_off, smem_u32(src), bytes, rbar);
+        mbar_arrive(&sm.bar[b]);
+    };
+    const int own0 = (int)rank;   // this CTA's chunks: own0, own0 + 2, ...
+
+    if (warp == 0 || warp >= OI_WARP) {
+        // =============================== issue warps =======================================================
+        // Three warps issue the tensor-core products, each a short program of its own, because one warp running all of
+        // them in series was the slowest role of the CTA (a warp issues its dependent instructions several cycles apart,
+        // and every wait is a few dozen instructions).  Each runs in lock step: waits are taken by every lane, TMA loads
+        // are issued by lane 0 and tensor-core instructions by the lane that elect.sync picks.
+        //   chain issuer (warp 0)     W S_0 and K^T (D U^): the two products on the serial chain, nothing else
+        //   output issuer             Q S_0, (P D^-1)(D U^) and the next chunk's (T B) V
+        //   owner issuer              K K^T two chunks ahead, [K;Q] K^T and the W product of this CTA's own chunks
+        // tcgen05.commit covers the issuing thread's products only, so products of different warps that touch the same
+        // accumulator or tile are ordered through barriers (B_TV_DONE, B_QS_DONE).
+        const unsigned isleep = warp == 0 ? 32u : (warp == OI_WARP ? 64u : 256u);   // chain, output, owner issuer
+        auto wwait = [&](int b, uint32_t parity) -> bool { return warp_wait(&sm.bar[b], parity, &sm.abort_flag, isleep); };
+        // four MMAs (K = 64): operand descriptors advance by astep / bstep (16-byte units) per K-step
+#define KLA_SEQ(d, a, astep, b, bstep, idesc, acc) mma4_bf16_lo<astep, bstep>(d, a, b, idesc, acc)
+        // Descriptors: everything except the 14-bit start-address field is fixed, so a K-step is an add.
+        const uint32_t d_kq0 = desc_lo(smem_desc_sw128(smem_u32(sm.kq[0]), 16, 1024));             // K-major views of a stage
+        const uint32_t d_kt0 = desc_lo(smem_desc_sw128(smem_u32(sm.kq[0]), KB * 8192, 1024));      // K^T / K as [tokens][d_k] (MN-major) view
+        constexpr uint32_t STAGE_STEP = (uint32_t)(Smem::KQ_BYTES >> 4);
+        auto tail_ok = [&](int c, int b) -> bool {   // masked rows of the last chunk zeroed (barrier b)
+            return !(c + 1 == nchunks && tail) || wwait(b, 0);
+        };
+        if (warp == 0) {
+            // ---- chain issuer ------------------------------------------------------------------------------------------------
+            const uint32_t d_sh = desc_lo(smem_desc_sw128(smem_u32(sm.s_hi), 16, 1024));
+            const uint32_t d_w = desc_lo(smem_desc_sw128(smem_u32(sm.w16), 16, 1024));
+            const uint32_t d_dh = desc_lo(smem_desc_sw128(smem_u32(sm.du_hi), 16, 1024)), d_dl = desc_lo(smem_desc_sw128(smem_u32(sm.du_lo), 16, 1024));
+            if (lane == 0) {
+                tma_prefetch_desc(&tm_q);
+                tma_prefetch_desc(&tm_k);
+                tma_prefetch_desc(&tm_v);
+                for (int c = 0; c < RST && c < nchunks; ++c) {
+                    const int st = c & 1;
+                    mbar_expect_tx(&sm.bar[B_FULL0 + st], STAGE_BYTES);
+#pragma unroll
+                    for (int kb = 0; kb < KB; ++kb) {
+                        tma_load_2d(sm.kq[st] + kb * 16384, &tm_k, h * D + kb * 64, tok0 + c * C, &sm.bar[B_FULL0 + st]);
+                        tma_load_2d(sm.kq[st] + kb * 16384 + 8192, &tm_q, h * D + kb * 64, tok0 + c * C, &sm.bar[B_FULL0 + st]);
+                    }
+                }
+                if (own0 < nchunks) {   // the early K tile of this CTA's first chunk; later ones are fetched by the pre group
+                    mbar_expect_tx(&sm.bar[B_EFULL], KB * 8192);
+#pragma unroll
+                    for (int kb = 0; kb < KB; ++kb) tma_load_2d(sm.ke + kb * 8192, &tm_k, h * D + kb * 64, tok0 + own0 * C, &sm.bar[B_EFULL]);
+                }
+                if (!is_map) {
+                    mbar_expect_tx(&sm.bar[B_V_FULL], 8192);
+                    tma_load_2d(sm.vt, &tm_v, h * D + sl * NS, tok0, &sm.bar[B_V_FULL]);
+                }
+            }
+            __syncwarp();
+            for (int c = 0; c < nchunks; ++c) {
+                const uint32_t ph = (uint32_t)(c & 1);
+                const uint32_t kt0 = d_kt0 + (uint32_t)(c & 1) * STAGE_STEP;
+                // ---- U^(c) = U(c) - W(c) S_0, on top of (T B) V(c) from the output issuer ---------------------------------------
+                if (!wwait(B_W_READY, ph)) break;
+                if (!wwait(B_TV_DONE, ph)) break;
+                if (!wwait(B_S_READY, ph)) break;
+                tc_fence_after();
+#pragma unroll 1
+                for (int kb = 0; kb < KB; ++kb) KLA_SEQ(tmem + TM_UH, d_w + kb * 512, 2, d_sh + kb * 512, 128, ID_H, (kb > 0 || !is_map) ? 1u : 0u);
+                bool signal = true;
+                if constexpr (VAR) signal = !(p.variant & VARIANT_TEST_TIMEOUT);   // test hook: the chain's bounded wait then runs out
+                if (signal) {
+                    mma_commit(&sm.bar[B_UH_DONE]);
+                    // Only where a later chunk's owner will wait for it: a signal sent for the last chunk could reach the
+                    // peer's SM after that CTA has gone and another block has set up its barriers there.
+                    if (c + 1 < nchunks) mma_commit_multicast(&sm.bar[B_W_FREE0 + (c & 1)], 3);
+                }
+                // ---- S(c+1) = gamma_C S + K^T (D U^); A = K^T: M = d_k (64-wide blocks KB*8192 bytes apart), K = tokens -----------
+                if (!wwait(B_FULL0 + (c & 1), (uint32_t)((c >> 1) & 1))) break;
+                if (!tail_ok(c, B_TAIL_READY)) break;
+                if (!wwait(B_DU_READY, ph)) break;
+                tc_fence_after();
+#pragma unroll 1
+                for (int t = 0; t < 2; ++t) KLA_SEQ(tmem + TM_DS, kt0, 128, t ? d_dl : d_dh, 128, ID_DS, t);
+                mma_commit(&sm.bar[B_DS_DONE]);
+            }
+        } else if (warp == OI_WARP) {
+            // ---- output issuer -----------------------------------------------------------------------------------------------
+            const uint32_t d_sh = desc_lo(smem_desc_sw128(smem_u32(sm.s_hi), 16, 1024)), d_sl = desc_lo(smem_desc_sw128(smem_u32(sm.s_lo), 16, 1024));
+            const uint32_t d_th = desc_lo(smem_desc_sw128(smem_u32(sm.t_hi), 16, 1024)), d_tl = desc_lo(smem_desc_sw128(smem_u32(sm.t_lo), 16, 1024));
+            const uint32_t d_ph = desc_lo(smem_desc_sw128(smem_u32(sm.p_hi), 16, 1024)), d_pl = desc_lo(smem_desc_sw128(smem_u32(sm.p_lo), 16, 1024));
+            const uint32_t d_v = desc_lo(smem_desc_sw128(smem_u32(sm.vt), 16, 1024));
+            const uint32_t d_dh = desc_lo(smem_desc_sw128(smem_u32(sm.du_hi), 16, 1024)), d_dl = desc_lo(smem_desc_sw128(smem_u32(sm.du_lo), 16, 1024));
+            // (T B) V of chunk c -> accumulator of U^ (overwrites: U^(c-1) has been read), then the signals: to the chain issuer,
+            // and to the owner of chunk c + 1, which may then overwrite the T tiles.  The transition-map slices have v = 0:
+            // only the second signal.
+            auto tv_prod = [&](int c) -> bool {
+                if (!is_map) {
+                    if (!wwait(B_T_READY, (uint32_t)(c & 1))) return false;
+                    if (!wwait(B_V_FULL, (uint32_t)(c & 1))) return false;
+                    if (!tail_ok(c, B_VTAIL)) return false;
+                    tc_fence_after();
+                    KLA_SEQ(tmem + TM_UH, d_th, 2, d_v, 128, ID_S, 0);
+                    KLA_SEQ(tmem + TM_UH, d_tl, 2, d_v, 128, ID_S, 1);
+                }
+                // (also without a product: the chain issuer then never runs more than a chunk ahead of this warp, which
+                // keeps the barriers both of them wait on in step)
+                mma_commit(&sm.bar[B_TV_DONE]);
+                if (c + 1 < nchunks) mma_commit_multicast(&sm.bar[B_T_FREE0 + (c & 1)], 3);   // (not for the last chunk: see the chain issuer)
+                return true;
+            };
+            bool ok = tv_prod(0);
+            for (int c = 0; ok && c < nchunks; ++c) {
+                const uint32_t ph = (uint32_t)(c & 1);
+                const uint32_t k0 = d_kq0 + (uint32_t)(c & 1) * STAGE_STEP;
+                if (!no_out) {
+                    // ---- Q S_0(c), while the chain forms D U^(c); the state tiles are rewritten only after B_QS_DONE --------------
+                    if (!(ok = wwait(B_QCONV0 + (c & 3), (uint32_t)((c >> 2) & 1)))) break;
+                    if (c > 0)
+                        if (!(ok = wwait(B_OUT_READ, ph ^ 1u))) break;
+                    if (!(ok = wwait(B_S_READY, ph))) break;
+                    tc_fence_after();
+#pragma unroll 1
+                    for (int t = 0; t < 2 * KB; ++t) {
+                        const uint32_t kb = (uint32_t)t & (KB - 1);
+                        KLA_SEQ(tmem + TM_QS, k0 + 512 + kb * 1024, 2, (t >= KB ? d_sl : d_sh) + kb * 512, 128, ID_H, t > 0);
+                    }
+                    mma_commit(&sm.bar[B_QS_DONE]);
+                }
+                // ---- (P D^-1)(D U^)(c), then the next chunk's (T B) V (U^(c) has been read once D U^(c) is there) -----------------
+                if (!(ok = wwait(B_DU_READY, ph))) break;
+                if (!no_out) {
+                    if (!(ok = wwait(B_P_READY, ph))) break;
+                    tc_fence_after();
+#pragma unroll 1
+                    for (int t = 0; t < 3; ++t) KLA_SEQ(tmem + TM_PU, t == 2 ? d_pl : d_ph, 2, t == 1 ? d_dl : d_dh, 128, ID_S, t > 0);
+                    mma_commit(&sm.bar[B_D4_DONE]);
+                    if (c + 1 < nchunks) mma_commit_multicast(&sm.bar[B_P_FREE0 + (c & 1)], 3);
+                }
+                if (c + 1 < nchunks)
+                    if (!(ok = tv_prod(c + 1))) break;
+            }
+        } else {
+            // ---- owner issuer: this CTA's own chunks ------------------------------------------------------------------------------
+            const uint32_t d_ke = desc_lo(smem_desc_sw128(smem_u32(sm.ke), 16, 1024));
+            const uint32_t d_gh = desc_lo(smem_desc_sw128(smem_u32(sm.tg_hi), 16, 1024)), d_gl = desc_lo(smem_desc_sw128(smem_u32(sm.tg_lo), 16, 1024));
+            // K K^T of an own chunk from its early tile -> TM_D1E.  The product is M = 128 so that the rows land one per
+            // TMEM lane; rows 64..127 of the A operand are whatever follows the tile, and lanes 64..127 are never read.
+            auto gram_e = [&](int c) -> bool {
+                const int o = c >> 1;   // ordinal among this CTA's chunks
+                if (!wwait(B_EFULL, (uint32_t)(o & 1))) return false;
+                if (!tail_ok(c, B_ETAIL)) return false;
+                if (o > 0)
+                    if (!wwait(B_D1E_FREE, (uint32_t)((o - 1) & 1))) return false;
+                tc_fence_after();
+#pragma unroll 1
+                for (int kb = 0; kb < KB; ++kb) KLA_SEQ(tmem + TM_D1E, d_ke + kb * 512, 2, d_ke + kb * 512, 2, ID_G, kb > 0);
+                mma_commit(&sm.bar[B_D1E_DONE]);
+                return true;
+            };
+            bool ok = own0 >= nchunks || gram_e(own0);
+            for (int c = own0; ok && c < nchunks; c += 2) {
+                const int o = c >> 1;
+                // K K^T of this CTA's next chunk: its inverse takes most of two chunk periods
+                if (c + 2 < nchunks)
+                    if (!(ok = gram_e(c + 2))) break;
+                if (!(ok = wwait(B_FULL0 + (c & 1), (uint32_t)((c >> 1) & 1)))) break;
+                if (!(ok = tail_ok(c, B_TAIL_READY))) break;
+                if (!no_out) {
+                    // [K;Q] K^T from the chain stage -> TM_D1L (lanes 64..127: Q K^T, for P); the Q tile is converted after it
+                    if (o > 0)
+                        if (!(ok = wwait(B_D1L_FREE, (uint32_t)((o - 1) & 1)))) break;
+                    tc_fence_after();
+                    const uint32_t a0 = d_kq0 + (uint32_t)(c & 1) * STAGE_STEP;
+#pragma unroll 1
+                    for (int kb = 0; kb < KB; ++kb) KLA_SEQ(tmem + TM_D1L, a0 + kb * 1024, 2, a0 + kb * 1024, 2, ID_G, kb > 0);
+                    mma_commit(&sm.bar[B_D1L_DONE]);
+                }
+                // (T B D_gamma) K -> W accumulator, once the tiles are there (pre group) and the aux group has read the last W
+                if (!(ok = wwait(B_TBG_READY, (uint32_t)(o & 1)))) break;
+                if (o > 0)
+                    if (!(ok = wwait(B_W_EMPTY, (uint32_t)((o - 1) & 1)))) break;
+                tc_fence_after();
+                const uint32_t kt0 = d_kt0 + (uint32_t)(c & 1) * STAGE_STEP;
+                KLA_SEQ(tmem + TM_W, d_gh, 2, kt0, 128, ID_W, 0);
+                KLA_SEQ(tmem + TM_W, d_gl, 2, kt0, 128, ID_W, 1);
+                mma_commit(&sm.bar[B_W_DONE]);
+            }
+        }
+#undef KLA_SEQ
+    } else if (warp >= AG_BASE / 32) {   // (the issue warps above this group were taken by the first branch)
+        // =============================== aux group ===========================================================
+        // Every chunk: the Q tile of this CTA's stage to fp16 (after the Gram product of an own chunk has read the bf16
+        // values).  Own chunks: W from its accumulator to the fp16 tile, then P D^-1, both into both CTAs.
+        const int at = tid - AG_BASE;          // 0..127
+        const int q = warp & 3;                // TMEM lane quadrant
+        const int i0 = q * 16 + (lane >> 2), i1 = i0 + 8;   // rows of an M = 64 accumulator held by this thread
+        const uint32_t tm16 = tmem + ((uint32_t)(q * 32) << 16);
+        for (int c = 0; c < nchunks; ++c) {
+            const bool own = (c & 1) == own0;
+            const int st = c & 1, sc = c & (NSC - 1);
+            const int o = c >> 1;   // ordinal among this CTA's chunks
+            bool ok = true;
+            if (!no_out) {
+                // ---- Q tile -> fp16, row i scaled by a power of two that puts its largest entry in [2^14, 2^15) ------------------
+                ok = own ? wait(B_D1L_DONE, (uint32_t)(o & 1)) : wait(B_FULL0 + st, (uint32_t)((c >> 1) & 1));
+                if (ok) {
+                    const int r = at >> 1, half = at & 1;
+                    constexpr int CPT = KB * 4;   // 16-byte pieces per thread (two threads per row)
+                    unsigned char *qt = sm.kq[st] + 8192;
+                    uint4 raw[CPT];
+                    uint32_t mx = 0;
+                    float nn = 0.f;
+#pragma unroll
+                    for (int e = 0; e < CPT; ++e) {
+                        const int pc = half * CPT + e;
+                        raw[e] = *reinterpret_cast<const uint4 *>(qt + (pc >> 3) * 16384 + sw128(r, pc & 7));
+                        const uint32_t w4[4] = {raw[e].x, raw[e].y, raw[e].z, raw[e].w};
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            mx = __vmaxu2(mx, w4[u] & 0x7fff7fffu);
+                            if constexpr (VAR) {
+                                const float f0 = __uint_as_float(w4[u] << 16), f1 = __uint_as_float(w4[u] & 0xffff0000u);
+                                nn += f0 * f0 + f1 * f1;
+                            }
+                        }
+                    }
+                    mx = max(mx & 0xffffu, mx >> 16);
+                    mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+                    const int E = (int)(mx >> 7);                       // biased exponent of the row's largest |q|
+                    const int se = min(max(268 - E, 1), 253);           // biased exponent of the scale 2^(141 - E)
+                    const float scale = __uint_as_float((uint32_t)se << 23);
+                    if constexpr (VAR) nn += __shfl_xor_sync(0xffffffffu, nn, 1);
+#pragma unroll
+                    for (int e = 0; e < CPT; ++e) {
+                        const int pc = half * CPT + e;
+                        uint32_t w4[4] = {raw[e].x, raw[e].y, raw[e].z, raw[e].w};
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            const __half2 hh = __floats2half2_rn(__uint_as_float(w4[u] << 16) * scale, __uint_as_float(w4[u] & 0xffff0000u) * scale);
+                            w4[u] = *reinterpret_cast<const uint32_t *>(&hh);
+                        }
+                        *reinterpret_cast<uint4 *>(qt + (pc >> 3) * 16384 + sw128(r, pc & 7)) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+                    }
+                    if (half == 0) {
+                        sm.qsc[sc][r] = __uint_as_float((uint32_t)(254 - se) << 23);
+                        if constexpr (VAR) sm.qn[sc][r] = 1.f / sqrtf(nn);
+                    }
+                    fence_async_smem();
+                    warp_arrive(B_QCONV0 + sc);
+                    warp_arrive(B_QSC0 + sc);
+                }
+            }
+            if (ok && !is_map && tail && c + 1 == nchunks) {
+                // rows of the V slice past the end of the sequence are another sequence's tokens: zero them
+                ok = wait(B_V_FULL, (uint32_t)(c & 1));
+                if (ok) {
+                    for (int e = at; e < (C - last_rows) * 8; e += AG_T)
+                        *reinterpret_cast<uint4 *>(sm.vt + sw128(last_rows + e / 8, e % 8)) = make_uint4(0, 0, 0, 0);
+                    fence_async_smem();
+                    warp_arrive(B_VTAIL);
+                }
+            }
+            if (ag_any(!ok)) break;
+            if (!own) continue;
+            // ---- W(c): accumulator -> fp16 tile (negated: the product then accumulates U - W S_0) ------------------------------
+            ok = wait(B_W_DONE, (uint32_t)(o & 1));
+            // the W tile is free once W S_0 of chunk c - 1 is complete in both CTAs
+            if (ok && c > 0) ok = wait(B_W_FREE0 + ((c - 1) & 1), (uint32_t)(((c - 1) >> 1) & 1));
+            if (ok) {
+                tc_fence_after();
+#pragma unroll 1
+                for (int cb = 0; cb < D / 32; ++cb) {
+                    float v[16];
+                    tmem_ld16x256b_x4(tm16 + TM_W + cb * 32, v);
+                    unsigned char *wt = sm.w16 + (cb >> 1) * 8192;
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const uint32_t o0 = sw128(i0, (cb & 1) * 4 + j) + 4 * (lane & 3), o1 = o0 + 8 * 128;
+                        const __half2 a = __floats2half2_rn(-v[4 * j], -v[4 * j + 1]);
+                        const __half2 b = __floats2half2_rn(-v[4 * j + 2], -v[4 * j + 3]);
+                        *reinterpret_cast<__half2 *>(wt + o0) = a;
+                        *reinterpret_cast<__half2 *>(wt + o1) = b;
+                    }
+                }
+                tc_fence_before();
+                fence_async_smem();
+                warp_arrive(B_W_EMPTY);
+            }
+            if (ag_any(!ok)) break;   // every warp's part of the tile is written
+            if (at == 0) publish(B_W_READY, sm.w16, KB * 8192);
+            // ---- P(c) D^-1 as bf16 hi/lo tiles (rows of Q K^T: TMEM lanes 64..127, the warps of quadrants 2 and 3) ------------
+            if (!no_out) {
+                if (q >= 2) {
+                    // g2 of chunk c is published with the scalars; the Gram product is complete (waited for above); the P
+                    // tiles are free once P U of chunk c - 1 is complete in both CTAs
+                    ok = wait(B_SCAL_READY0 + sc, (uint32_t)((c >> 2) & 1));
+                    if (ok && c > 0) ok = wait(B_P_FREE0 + ((c - 1) & 1), (uint32_t)(((c - 1) >> 1) & 1));
+                    if (ok) {
+                        tc_fence_after();
+                        form_p_row(sm, sc, (q - 2) * 32 + lane, 0, 8, tm_lane + TM_D1L);
+                        tc_fence_before();
+                        fence_async_smem();
+                        warp_arrive(B_D1L_FREE);
+                    }
+                }
+                if (ag_any(!ok)) break;
+                if (at == 0) publish(B_P_READY, sm.p_hi, 16384);
+            }
+        }
+    } else if (warp >= PG_BASE / 32) {
+        // =============================== pre group ===========================================================
+        // This CTA's own chunks (c mod 2 = rank): decay scan, X(c), beta(c), the inverse, and the two operand forms of T.
+        // The peer's chunks: only the zeroing of the masked rows of the last chunk (the K and Q tiles are per CTA).
+        // Warps 0, 1, 4, 5 of the group hold rows of K K^T (TMEM lanes 0..63); every warp works on the inverse.
+        const int pt = tid - PG_BASE;
+        const int q = warp & 3, chh = (warp - PG_BASE / 32) >> 2;
+        const bool is_g = q < 2;
+        const int i = (q & 1) * 32 + lane;
+        const bool live = chh <= (q & 1);
+        const bool scan_warp = q == 0 && chh == 1;
+        float *mm = sm.tl + 32;   // scratch of the block products: rows 0..31, columns 32..63 of the solve matrix
+        float la_next0 = 0.f, la_next1 = 0.f, eta_next = 0.f;
+        auto fetch_gates = [&](int c) {
+            if (scan_warp) {
+                const int t = c * C + 2 * lane;
+                la_next0 = (t < len) ? p.log_alpha[(size_t)(tok0 + t) * p.H + h] : 0.f;
+                la_next1 = (t + 1 < len) ? p.log_alpha[(size_t)(tok0 + t + 1) * p.H + h] : 0.f;
+            }
+            if (is_g && chh == q) {
+                const int t = c * C + i;
+                eta_next = (t < len) ? p.eta[(size_t)(tok0 + t) * p.H + h] : 0.f;
+            }
+        };
+        if (own0 < nchunks) fetch_gates(own0);
+        for (int c = 0; c < nchunks; ++c) {
+            const int rows = (c == nchunks - 1) ? last_rows : C;
+            const int st = c & 1, sc = c & (NSC - 1);
+            const bool own = (c & 1) == own0;
+            const int o = c >> 1;   // ordinal among this CTA's chunks
+            const float la0 = la_next0, la1 = la_next1, eta_cur = eta_next;
+            if (own && c + 2 < nchunks) fetch_gates(c + 2);
+            bool okc = true;
+            if (rows < C) {
+                // Last chunk: rows past the end of the sequence hold a neighbour's tokens (or TMA zero fill); zero them so
+                // that they are inert in every product.  First in the early K tile of an own chunk (its K K^T waits for
+                // this, and the stage below lands only once the chain has got to chunk c - 2, which may itself need
+                // products that the owner issuer issues after that K K^T), then in the K and Q tiles of the chain stage.
+                if (own) {
+                    okc = wait(B_EFULL, (uint32_t)(o & 1));
+                    if (okc) {
+                        for (int e = pt; e < (C - rows) * 8 * KB; e += PG_T) {
+                            const int kb = e / ((C - rows) * 8), e2 = e % ((C - rows) * 8);
+                            *reinterpret_cast<uint4 *>(sm.ke + kb * 8192 + sw128(rows + e2 / 8, e2 % 8)) = make_uint4(0, 0, 0, 0);
+                        }
+                        fence_async_smem();
+                        warp_arrive(B_ETAIL);
+                    }
+                }
+                if (okc) okc = wait(B_FULL0 + st, (uint32_t)((c >> 1) & 1));
+                if (okc) {
+                    zero_tail_rows<KB>(sm.kq[st], rows, pt);
+                    fence_async_smem();
+                    warp_arrive(B_TAIL_READY);
+                }
+            }
+            if (pg_any(!okc)) break;
+            if (!own) continue;
+
+            if (is_g) {
+                okc = wait(B_D1E_DONE, (uint32_t)(o & 1));
+                // K K^T of chunk c has read the early tile: fetch the K tile of this CTA's next chunk into it
+                if (okc && scan_warp && lane == 0 && c + 2 < nchunks) {
+                    mbar_expect_tx(&sm.bar[B_EFULL], KB * 8192);
+#pragma unroll
+                    for (int kb = 0; kb < KB; ++kb) tma_load_2d(sm.ke + kb * 8192, &tm_k, h * D + kb * 64, tok0 + (c + 2) * C, &sm.bar[B_EFULL]);
+                }
+                __syncwarp();
+            }
+            // Decay scan into slot sc, which last held chunk c - 4.  Its readers are done: this CTA's P(c-4) was formed
+            // before the Gram product of chunk c could reuse the accumulator (waited for just above); the peer's chain read
+            // the scalars before its D U^(c-4), which came before the (T B) V product of chunk c - 3 that this group saw
+            // complete in both CTAs while it worked on chunk c - 2.
+            if (okc && scan_warp) {
+                decay_scan(sm, sc, lane, la0, la1);
+                fence_async_smem();   // gam and dec are also copied to the peer
+            }
+            if (pg_any(!okc)) break;   // publishes the decay sums to the whole group
+            if (is_g) {
+                // ---- X = A^- o K K^T (this thread: row i, 32 columns) and beta_i, Eq. 3 ----------------------
+                {
+                    tc_fence_after();
+                    if (live) {
+                        // G_ii = ||k_i||^2 comes with the row
+                        const float dg = form_x_row16(sm, sc, i, chh, tm_lane + TM_D1E + chh * 32);
+                        if (chh == q) {
+                            float bta = eta_cur / (dg + p.eps);
+                            if constexpr (VAR) bta = (p.variant & VARIANT_COEFF_ETA) ? eta_cur : bta;
+                            sm.beta[sc][i] = (i < rows) ? bta : 0.f;
+                        }
+                    }
+                    tc_fence_before();
+                    warp_arrive(B_D1E_FREE);
+                }
+            }
+            if (pg_any(!okc)) break;
+            // gamma and exp(g_C - g) of chunk c go to both chains now, long before T(c)
+            if (pt == 0) {
+                const uint32_t rbar = smem_u32(&sm.bar[B_SCAL_READY0 + sc]) + peer_off;
+                mbar_arrive_expect_tx_cluster(rbar, 512);
+                bulk_copy_to_cluster(smem_u32(sm.gam[sc]) + peer_off, smem_u32(sm.gam[sc]), 256, rbar);
+                bulk_copy_to_cluster(smem_u32(sm.dec[sc]) + peer_off, smem_u32(sm.dec[sc]), 256, rbar);
+                mbar_arrive(&sm.bar[B_SCAL_READY0 + sc]);
+            }
+
+            // ---- T = (I + B X)^-1 ----------------------------------------------------------------------------
+            const float *bet = sm.beta[sc];
+            if (pt < 64) substitute_diag_blocks(sm.tl, bet, pt);
+            pg_sync();
+            merge_level<8>(sm.tl, mm, LDT, bet, pt);
+            merge_level_mma(16, sm.tl, mm, bet, pt >> 5, lane);
+            merge_level_mma(32, sm.tl, mm, bet, pt >> 5, lane);
+            // ---- T B D_gamma tiles (this CTA only); the W product of this CTA's previous chunk has read the old ones -----------
+            bool okd = true;
+            if (o > 0 && pt >= PG_T - 32) okd = wait(B_W_DONE, (uint32_t)((o - 1) & 1));
+            if (pg_any(!okd)) break;
+            write_t_tiles(sm, true, sm.tg_hi, sm.tg_lo, sc, pt);
+            fence_async_smem();
+            warp_arrive(B_TBG_READY);
+            // ---- T B tiles into both CTAs, once (T B) V of chunk c - 1 is complete in both ------------------------------------
+            if (c > 0 && pt >= PG_T - 32) okd = wait(B_T_FREE0 + ((c - 1) & 1), (uint32_t)(((c - 1) >> 1) & 1));
+            if (pg_any(!okd)) break;
+            if (!is_map) {
+                write_t_tiles(sm, false, sm.t_hi, sm.t_lo, sc, pt);
+                fence_async_smem();
+            }
+            pg_sync();  // every tile write is done (and the solve matrix may be reused by this CTA's next chunk)
+            if (!is_map && pt == 0) publish(B_T_READY, sm.t_hi, 16384);
+        }
+    } else {
+        // =============================== chain group ==========================================================
+        const int ct = tid - CG_BASE;           // 0..255
+        const int q = warp & 3;                 // TMEM lane quadrant
+        const int hf = ct >> 7;                 // column half: 0 -> columns 0..31, 1 -> 32..63
+        const int srow = q * 32 + lane;         // state row (M = 128 accumulator layout, 32x32b loads)
+        // M = 64 accumulators, 16x256b loads: rows i0 and i0 + 8, column pairs cp + 8j (j = 0..3), cp = hf * 32 + 2 (lane % 4)
+        const int i0 = q * 16 + (lane >> 2), i1 = i0 + 8;
+        const uint32_t tm16 = tmem + ((uint32_t)(q * 32) << 16) + hf * 32;
+
+        float S[32];
+        if (is_map) {
+            // transition map: start from the identity (columns sl * NS + hf * 32 .. of I)
+#pragma unroll
+            for (int c = 0; c < 32; ++c) S[c] = (srow == sl * NS + hf * 32 + c) ? 1.f : 0.f;
+        } else if (p.init_state) {
+#pragma unroll
+            for (int c = 0; c < 32; c += 4) {
+                const float4 x = *reinterpret_cast<const float4 *>(p.init_state + state_off + (size_t)srow * D + hf * 32 + c);
+                S[c] = x.x; S[c + 1] = x.y; S[c + 2] = x.z; S[c + 3] = x.w;
+            }
+        } else {
+#pragma unroll
+            for (int c = 0; c < 32; ++c) S[c] = 0.f;
+        }
+        auto store_state_tiles = [&]() {
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                uint4 hi, lo;
+                split2h(S[8 * c + 0], S[8 * c + 1], hi.x, lo.x);
+                split2h(S[8 * c + 2], S[8 * c + 3], hi.y, lo.y);
+                split2h(S[8 * c + 4], S[8 * c + 5], hi.z, lo.z);
+                split2h(S[8 * c + 6], S[8 * c + 7], hi.w, lo.w);
+                *reinterpret_cast<uint4 *>(sm.s_hi + sw128(srow, hf * 4 + c)) = hi;
+                *reinterpret_cast<uint4 *>(sm.s_lo + sw128(srow, hf * 4 + c)) = lo;
+            }
+            fence_async_smem();
+            warp_arrive(B_S_READY);
+        };
+        // byte offset of this thread's bf16 pair j (columns cp + 8j, cp + 8j + 1) of row i inside the
+        // 64-token x 64-column B-operand tiles
+        const uint32_t lo4 = 4 * (lane & 3);
+        auto off = [&](int i, int j) -> uint32_t { return sw128(i, hf * 4 + j) + lo4; };
+        store_state_tiles();
+
+        for (int c = 0; c < nchunks; ++c) {
+            const uint32_t ph = (uint32_t)(c & 1);
+            const int rows = (c == nchunks - 1) ? last_rows : C;
+            const int st = c & 1, sc = c & (NSC - 1);
+            if (!wait(B_SCAL_READY0 + sc, (uint32_t)((c >> 2) & 1))) break;   // scalars of chunk c
+            const float g0 = sm.gam[sc][i0], g1 = sm.gam[sc][i1];
+            const float d0 = sm.dec[sc][i0], d1 = sm.dec[sc][i1];
+            const float gC = sm.gam[sc][C - 1];
+            // ---- D U^ as hi/lo operand: of the state update and, against P D^-1, of the outputs --------------------------------
+            if (!wait(B_UH_DONE, ph)) break;
+            // (T B) V of chunk c has read the V slice: fetch the next one
+            if (ct == 0 && !is_map && c + 1 < nchunks) {
+                mbar_expect_tx(&sm.bar[B_V_FULL], 8192);
+                tma_load_2d(sm.vt, &tm_v, h * D + sl * NS, tok0 + (c + 1) * C, &sm.bar[B_V_FULL]);
+            }
+            tc_fence_after();
+#pragma unroll 1
+            for (int j = 0; j < 4; ++j) {
+                float acc[4];
+                tmem_ld16x256b_x1(tm16 + TM_UH + 8 * j, acc);
+                const uint32_t o0 = off(i0, j), o1 = o0 + 8 * 128;   // i1 = i0 + 8: same swizzle phase, eight rows on
+                uint32_t hi, lo;
+                split2(d0 * acc[0], d0 * acc[1], hi, lo);
+                *reinterpret_cast<uint32_t *>(sm.du_hi + o0) = hi;
+                *reinterpret_cast<uint32_t *>(sm.du_lo + o0) = lo;
+                split2(d1 * acc[2], d1 * acc[3], hi, lo);
+                *reinterpret_cast<uint32_t *>(sm.du_hi + o1) = hi;
+                *reinterpret_cast<uint32_t *>(sm.du_lo + o1) = lo;
+            }
+            fence_async_smem();
+            tc_fence_before();
+            warp_arrive(B_DU_READY);
+
+            // ---- state: S <- gamma_C S + K^T (D U^) -----------------------------------------------------------------
+            if (!wait(B_DS_DONE, ph)) break;
+            if (!no_out)
+                if (!wait(B_QS_DONE, ph)) break;   // Q S_0(c) comes from another issuer: it too has read the state tiles and the Q tile
+            // K^T (D U^)(c) was the last reader of the K/Q stage of chunk c: refill it at once (this CTA's Gram product of
+            // chunk c + 3 may be due within a fraction of a chunk period)
+            if (ct == 0 && c + RST < nchunks) {
+                const int cn = c + RST;
+                mbar_expect_tx(&sm.bar[B_FULL0 + st], STAGE_BYTES);
+#pragma unroll
+                for (int kb = 0; kb < KB; ++kb) {
+                    tma_load_2d(sm.kq[st] + kb * 16384, &tm_k, h * D + kb * 64, tok0 + cn * C, &sm.bar[B_FULL0 + st]);
+                    tma_load_2d(sm.kq[st] + kb * 16384 + 8192, &tm_q, h * D + kb * 64, tok0 + cn * C, &sm.bar[B_FULL0 + st]);
+                }
+            }
+            tc_fence_after();
+            {
+                float acc[32];
+                tmem_ld32(tm_lane + TM_DS + hf * 32, acc);
+#pragma unroll
+                for (int e = 0; e < 32; ++e) S[e] = gC * S[e] + acc[e];
+            }
+            tc_fence_before();
+            if (c + 1 < nchunks) store_state_tiles();
+
+            // ---- outputs: O_i = gamma_i (Q S_0)_i + (P U^)_i (off the chain) -----------------------------------------
+            if (no_out) continue;
+            if (!wait(B_QSC0 + sc, (uint32_t)((c >> 2) & 1))) break;
+            if (!wait(B_D4_DONE, ph)) break;
+            tc_fence_after();
+            {
+                // This thread's accumulator values are column pairs cp + 8j (j = 0..3) of rows i0 and i1; a 4 x 4 transpose
+                // over the four lanes of a quad gives each lane 8 consecutive columns of both rows, so that every
+                // store is 16 bytes and a warp's store covers whole 32-byte sectors.
+                float pu[16], qs[16];
+                tmem_ld16x256b_x4(tm16 + TM_PU, pu);
+                tmem_ld16x256b_x4(tm16 + TM_QS, qs);
+                tc_fence_before();
+                warp_arrive(B_OUT_READ);
+                float n0 = g0 * sm.qsc[sc][i0], n1 = g1 * sm.qsc[sc][i1], m0 = 1.f, m1 = 1.f;   // o = n * qs + m * pu
+                if constexpr (VAR) {
+                    if (p.variant & VARIANT_QNORM) {   // read-out over ||q||
+                        m0 = sm.qn[sc][i0]; m1 = sm.qn[sc][i1];
+                        n0 *= m0; n1 *= m1;
+                    }
+                }
+                const int t4 = lane & 3;
+                const size_t col = (size_t)sl * NS + hf * 32 + 8 * t4;
+                OUT *o0 = reinterpret_cast<OUT *>(p.out) + ((size_t)(tok0 + c * C + i0) * p.H + h) * D + col;
+                OUT *o1 = reinterpret_cast<OUT *>(p.out) + ((size_t)(tok0 + c * C + i1) * p.H + h) * D + col;
+                if constexpr (sizeof(OUT) == 2) {
+                    uint32_t a[4], b[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const __nv_bfloat162 x = __floats2bfloat162_rn(n0 * qs[4 * j] + m0 * pu[4 * j], n0 * qs[4 * j + 1] + m0 * pu[4 * j + 1]);
+                        const __nv_bfloat162 y = __floats2bfloat162_rn(n1 * qs[4 * j + 2] + m1 * pu[4 * j + 2], n1 * qs[4 * j + 3] + m1 * pu[4 * j + 3]);
+                        a[j] = *reinterpret_cast<const uint32_t *>(&x);
+                        b[j] = *reinterpret_cast<const uint32_t *>(&y);
+                    }
+                    quad_transpose(a, t4);
+                    quad_transpose(b, t4);
+                    if (i0 < rows) *reinterpret_cast<uint4 *>(o0) = make_uint4(a[0], a[1], a[2], a[3]);
+                    if (i1 < rows) *reinterpret_cast<uint4 *>(o1) = make_uint4(b[0], b[1], b[2], b[3]);
+                } else {
+                    uint32_t ax[4], ay[4], bx[4], by[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        ax[j] = __float_as_uint(n0 * qs[4 * j] + m0 * pu[4 * j]);
+                        ay[j] = __float_as_uint(n0 * qs[4 * j + 1] + m0 * pu[4 * j + 1]);
+                        bx[j] = __float_as_uint(n1 * qs[4 * j + 2] + m1 * pu[4 * j + 2]);
+                        by[j] = __float_as_uint(n1 * qs[4 * j + 3] + m1 * pu[4 * j + 3]);
+                    }
+                    quad_transpose(ax, t4);
+                    quad_transpose(ay, t4);
+                    quad_transpose(bx, t4);
+                    quad_transpose(by, t4);
+                    if (i0 < rows) {
+                        *reinterpret_cast<uint4 *>(o0) = make_uint4(ax[0], ay[0], ax[1], ay[1]);
+                        *reinterpret_cast<uint4 *>(o0 + 4) = make_uint4(ax[2], ay[2], ax[3], ay[3]);
+                    }
+                    if (i1 < rows) {
+                        *reinterpret_cast<uint4 *>(o1) = make_uint4(bx[0], by[0], bx[1], by[1]);
+                        *reinterpret_cast<uint4 *>(o1 + 4) = make_uint4(bx[2], by[2], bx[3], by[3]);
+                    }
+                }
+            }
+        }
+        if (!sm.abort_flag && fin) {
+#pragma unroll
+            for (int c = 0; c < 32; c += 4)
+                *reinterpret_cast<float4 *>(fin + fin_off + (size_t)srow * D + hf * 32 + c) =
+                    make_float4(S[c], S[c + 1], S[c + 2], S[c + 3]);
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    // Neither CTA of a pair leaves while the other may still write into its shared memory or signal its barriers.
+    // On the normal path everything sent has been waited for by its receiver; after a wait gave up, copies and
+    // completion signals issued just before may still be on their way (microseconds): let them land first.
+    if (sm.abort_flag)
+        for (int i = 0; i < 32; ++i) __nanosleep(1000);
+    cluster_sync_all();
+    if (warp == 0) {
+        tc_fence_after();
+        tmem_dealloc(tmem, TM_COLS);
+    }
+    if (tid == 0 && sm.abort_flag && p.status_word) atomicExch(p.status_word, (int)KLA_ERR_TIMEOUT);
+}
+
+template <int D, typename OUT, bool VAR>
+cudaError_t launch_v(const ChunkParams &p, cudaStream_t stream)
+{
+    using Smem = WySmem<D>;
+    const uint64_t n_tok = (uint64_t)p.B * p.T;
+    CUtensorMap tq, tk, tv;
+    if (!make_tmap(&tq, p.q, n_tok, (uint64_t)p.H * D) || !make_tmap(&tk, p.k, n_tok, (uint64_t)p.H * D) ||
+        !make_tmap(&tv, p.v, n_tok, (uint64_t)p.H * D))
+        return cudaErrorInvalidValue;
+    auto kern = kla_chunk_wy_kernel<D, OUT, VAR>;
+    const int smem = (int)sizeof(Smem) + 1024;
+    cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (err != cudaSuccess) return err;
+    // segment pass 1: (seg_G - 1) segments per sequence, twice the slices; p.n_seq counts all segments there
+    const int grid = p.seg_pass == 1 ? (p.n_seq / p.seg_G) * (p.seg_G - 1) * p.H * 2 * (D / NS) : p.n_seq * p.H * (D / NS);
+    if (grid == 0) return cudaSuccess;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(NT);
+    cfg.dynamicSmemBytes = (size_t)smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;   // blocks 2j, 2j + 1 = the two slices of one (sequence, head)
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    err = cudaLaunchKernelEx(&cfg, kern, tq, tk, tv, p);
+    count_launch(1);
+    return err != cudaSuccess ? err : cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_chunk_wy(const ChunkParams &p, int out_dtype, cudaStream_t stream)
+{
+    const bool var = (p.variant & ~(VARIANT_NO_PAIR | VARIANT_WY)) != 0;
+    if (out_dtype == KLA_BF16) return var ? launch_v<128, __nv_bfloat16, true>(p, stream) : launch_v<128, __nv_bfloat16, false>(p, stream);
+    return var ? launch_v<128, float, true>(p, stream) : launch_v<128, float, false>(p, stream);
+}
+
+}  // namespace kla

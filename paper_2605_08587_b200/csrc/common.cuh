@@ -17,7 +17,6 @@ struct ChunkParams {
     float *final_state;       // may be null
     const int32_t *cu_seqlens;  // device, may be null (fixed length)
     int32_t *status_word;       // may be null
-    long long *trace;           // debug builds only (KLA_TRACE): per-event SM clock stamps; else null
     int32_t B, T, H, n_seq;
     float eps;
     // Segment-parallel scan (tensor-core kernel only; all zero / null for a plain launch).
@@ -27,7 +26,7 @@ struct ChunkParams {
     //   seg_pass 3: every segment from its true start state; only the last segment of a sequence writes
     //               final_state, at the sequence's index.
     int32_t seg_pass, seg_G;
-    int32_t variant;     // bit 0: beta_t = eta_t instead of Eq. 3; bit 1: read-out divided by ||q_t||; bit 2: test hook; bit 3: see VARIANT_NO_PAIR
+    int32_t variant;     // bit 0: beta_t = eta_t instead of Eq. 3; bit 1: read-out divided by ||q_t||; bit 2: test hook; bits 3, 4: see VARIANT_NO_PAIR, VARIANT_WY
     union {
         float *map_state;            // segment pass 1
         const int32_t *seq_order;    // packed input, plain launch: block b works on sequence seq_order[b] (longest
@@ -36,6 +35,7 @@ struct ChunkParams {
 };
 constexpr int32_t VARIANT_COEFF_ETA = 1, VARIANT_QNORM = 2, VARIANT_TEST_TIMEOUT = 4;
 constexpr int32_t VARIANT_NO_PAIR = 8;   // host side only: launch the two slices of a head as independent CTAs
+constexpr int32_t VARIANT_WY = 16;       // host side only: head dimension 128 goes to the WY-form kernel (chunk_wy.cu)
 
 struct DecodeParams {
     const void *q, *k, *v;
@@ -57,6 +57,8 @@ cudaError_t launch_chunk_simt(const ChunkParams &p, int d, int chunk, int io_dty
                               cudaStream_t stream);
 cudaError_t launch_chunk_tc(const ChunkParams &p, int d, int io_dtype, int out_dtype,
                             cudaStream_t stream);
+// Head dimension 128, the two slices of a head as a cluster of two CTAs (chunk_wy.cu); called by launch_chunk_tc.
+cudaError_t launch_chunk_wy(const ChunkParams &p, int out_dtype, cudaStream_t stream);
 // Segment-parallel helpers (segscan.cu).  cu_seg[b * G + g] = b * T + min(g * seg_len, T), one more entry = B * T.
 cudaError_t launch_seg_bounds(int32_t *cu_seg, int B, int T, int G, int seg_len, cudaStream_t stream);
 // order[r] = index of the sequence with the r-th largest length (ties by index); n_seq small (quadratic work)
@@ -68,6 +70,9 @@ cudaError_t launch_seg_combine(const float *init_state, const float *map, const 
 bool chunk_tc_supported(int d, int chunk, int io_dtype);
 
 void count_launch(int n);
+// Host-side validation of a chunk-forward call (api.cu); `check_workspace`: also that desc->workspace is large enough.
+kla_status check_chunk_args(const kla_desc *d, const void *q, const void *k, const void *v, const float *log_alpha, const float *eta,
+                            float eps, int32_t chunk, const float *init_state, void *out, float *final_state, bool check_workspace);
 
 // ---- device helpers -------------------------------------------------------------------------
 __device__ __forceinline__ float to_f32(float x) { return x; }

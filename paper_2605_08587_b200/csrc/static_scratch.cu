@@ -25,13 +25,13 @@ void *g_scratch_ptr[MAX_DEVICES] = {};
 kla_status scratch_for_current_device(void **out)
 {
     int dev = -1;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return KLA_ERR_ARCH;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return KLA_ERR_DEVICE;
     std::lock_guard<std::mutex> lock(g_mutex);
     if (!g_scratch_ptr[dev]) {
         void *ptr = nullptr;
         if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) {
             (void)cudaGetLastError();
-            return KLA_ERR_LAUNCH;
+            return KLA_ERR_DEVICE;
         }
         g_scratch_ptr[dev] = ptr;
     }
@@ -49,6 +49,9 @@ extern "C" kla_status kla_chunk_fwd_static_scratch(const kla_desc *desc, const v
     kla_desc d = *desc;
     d.workspace = nullptr;
     d.workspace_bytes = 0;
+    // the same argument checks as kla_chunk_fwd, in the same order, before anything about the scratch
+    const kla_status vst = kla::check_chunk_args(&d, q, k, v, log_alpha, eta, eps, chunk, init_state, out, final_state, false);
+    if (vst != KLA_OK) return vst;
     // what this shape needs (0 when sequences are not cut into segments); decided on the host, nothing launched
     const size_t need = kla_chunk_fwd_workspace_bytes(&d, chunk);
     if (need > (size_t)KLA_STATIC_SCRATCH_BYTES) return KLA_ERR_WORKSPACE;

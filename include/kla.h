@@ -188,6 +188,30 @@ kla_status kla_chunk_fwd_timed(const kla_desc *desc, const void *q, const void *
                                const float *init_state, void *out, float *final_state, float *pass_ms);
 
 /*
+ * Sequence-parallel prefill: one long sequence cut along T across several GPUs (the affine form of Appendix B: every
+ * chunk step, hence every span of tokens, maps the incoming state S to Phi S + N).  Each GPU holds one span of the
+ * sequence and (1) calls kla_chunk_span_map on it, (2) exchanges (Phi, N) with the other GPUs (one all-gather of
+ * 2 x B x H x d_k x d_k fp32 per GPU; the library has no communication of its own), (3) calls kla_state_chain on the
+ * gathered maps to get the state at the start of its span, (4) calls kla_chunk_fwd on its span with that state.
+ *
+ * kla_chunk_span_map: transition map of the whole input (head dimension 128 or 64, bf16, chunk 64, fixed length).
+ *   q is not read (no outputs are formed) and may be NULL.
+ *   phi_out [B, H, d_k, d_k] fp32: the state reached from the identity with v = 0 (S_end = phi_out . S_start + n_out)
+ *   n_out   [B, H, d_k, d_v] fp32: the state reached from zero
+ *   desc->workspace: at least kla_chunk_span_map_workspace_bytes(desc) bytes.
+ *
+ * kla_state_chain: start states of R consecutive spans from their maps, in fp32:
+ *   start[b, 0] = init_state[b] (or 0);  start[b, r + 1] = phi[b, r] . start[b, r] + n[b, r]
+ *   phi, n [B, R, H, d, d] fp32 (the maps of spans 0 .. R-2 are read); start_out [B, R, H, d, d] fp32.
+ *   Uses desc->B, H, d_k, stream only.
+ */
+size_t kla_chunk_span_map_workspace_bytes(const kla_desc *desc);
+kla_status kla_chunk_span_map(const kla_desc *desc, const void *k, const void *v, const float *log_alpha, const float *eta,
+                              float eps, float *phi_out, float *n_out);
+kla_status kla_state_chain(const kla_desc *desc, int32_t n_spans, const float *init_state, const float *phi, const float *n,
+                           float *start_out);
+
+/*
  * One recurrent decode step (Algorithm 1 left) for B sequences x H heads; desc->T must be 1 and
  * desc->cu_seqlens NULL.
  *

@@ -22,7 +22,8 @@ def KLA_FLAG_SEGMENTS(g: int) -> int:
     return int(g) << 8
 
 
-EXPORTS = ["kla_chunk_fwd_workspace_bytes", "kla_chunk_fwd", "kla_chunk_fwd_timed", "kla_chunk_fwd_static_scratch", "kla_decode_step", "kla_decode_steps",
+EXPORTS = ["kla_chunk_fwd_workspace_bytes", "kla_chunk_fwd", "kla_chunk_fwd_timed", "kla_chunk_fwd_static_scratch",
+           "kla_chunk_span_map_workspace_bytes", "kla_chunk_span_map", "kla_state_chain", "kla_decode_step", "kla_decode_steps",
            "kla_status_str", "kla_launch_count"]
 
 
@@ -62,6 +63,12 @@ def load():
     lib.kla_chunk_fwd_timed.argtypes = lib.kla_chunk_fwd.argtypes + [ctypes.POINTER(ctypes.c_float)]
     lib.kla_chunk_fwd_static_scratch.restype = ctypes.c_int
     lib.kla_chunk_fwd_static_scratch.argtypes = lib.kla_chunk_fwd.argtypes
+    lib.kla_chunk_span_map_workspace_bytes.restype = ctypes.c_size_t
+    lib.kla_chunk_span_map_workspace_bytes.argtypes = [dp]
+    lib.kla_chunk_span_map.restype = ctypes.c_int
+    lib.kla_chunk_span_map.argtypes = [dp, vp, vp, fp, fp, ctypes.c_float, fp, fp]
+    lib.kla_state_chain.restype = ctypes.c_int
+    lib.kla_state_chain.argtypes = [dp, ctypes.c_int32, fp, fp, fp, fp]
     lib.kla_decode_step.restype = ctypes.c_int
     lib.kla_decode_step.argtypes = [dp, vp, vp, vp, fp, fp, ctypes.c_float, fp, vp]
     lib.kla_decode_steps.restype = ctypes.c_int
@@ -202,6 +209,41 @@ def kla_chunk_fwd_static_scratch(q, k, v, log_alpha, eta, eps, out, final_state=
             _dev(out, "out"), _dev(final_state, "final_state", torch.float32))
     _check(code)
     return out, final_state
+
+
+def kla_chunk_span_map(k, v, log_alpha, eta, eps, flags=KLA_FLAG_NONE):
+    """Transition map of a span of tokens (include/kla.h: kla_chunk_span_map): S_end = phi . S_start + n.
+    k [B, T, H, d]; v [B, T, H, d]; log_alpha, eta [B, T, H]; bf16 inputs.  Returns (phi, n), both [B, H, d, d] fp32."""
+    lib = load()
+    B, T, H, d = k.shape
+    phi = torch.empty((B, H, d, d), device=k.device, dtype=torch.float32)
+    n = torch.empty((B, H, d, d), device=k.device, dtype=torch.float32)
+    desc = KlaDesc(B=B, T=T, H=H, d_k=d, d_v=v.shape[-1], n_seq=B, cu_seqlens=None, host_seqlens=None, io_dtype=_dt(k),
+                   out_dtype=KLA_F32, flags=flags, workspace=None, workspace_bytes=0, status_word=None, stream=_stream(k.device))
+    need = lib.kla_chunk_span_map_workspace_bytes(ctypes.byref(desc))
+    ws = torch.empty(max(need, 16), device=k.device, dtype=torch.uint8)
+    desc.workspace, desc.workspace_bytes = ws.data_ptr(), need
+    with torch.cuda.device(k.device):
+        code = lib.kla_chunk_span_map(ctypes.byref(desc), _dev(k, "k"), _dev(v, "v"), _dev(log_alpha, "log_alpha", torch.float32),
+                                      _dev(eta, "eta", torch.float32), float(eps), phi.data_ptr(), n.data_ptr())
+    _check(code)
+    return phi, n
+
+
+def kla_state_chain(phi, n, init_state=None):
+    """Start states of R consecutive spans from their maps (include/kla.h: kla_state_chain).
+    phi, n [B, R, H, d, d] fp32; init_state [B, H, d, d] fp32 or None (zeros).  Returns start [B, R, H, d, d] fp32 with
+    start[:, 0] = init_state and start[:, r + 1] = phi[:, r] . start[:, r] + n[:, r]."""
+    lib = load()
+    B, R, H, d, _ = phi.shape
+    start = torch.empty_like(phi)
+    desc = KlaDesc(B=B, T=1, H=H, d_k=d, d_v=d, n_seq=B, cu_seqlens=None, host_seqlens=None, io_dtype=KLA_BF16, out_dtype=KLA_F32,
+                   flags=0, workspace=None, workspace_bytes=0, status_word=None, stream=_stream(phi.device))
+    with torch.cuda.device(phi.device):
+        code = lib.kla_state_chain(ctypes.byref(desc), R, _dev(init_state, "init_state", torch.float32), _dev(phi, "phi", torch.float32),
+                                   _dev(n, "n", torch.float32), start.data_ptr())
+    _check(code)
+    return start
 
 
 def _decode_desc(q, v, out, B, H, d_k, d_v, flags=0):

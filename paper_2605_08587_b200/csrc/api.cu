@@ -269,6 +269,79 @@ kla_status kla_chunk_fwd_timed(const kla_desc *desc, const void *q, const void *
 }
 
 
+// ---- sequence-parallel prefill: the pieces around the exchange ------------------------------------------------------------
+size_t kla_chunk_span_map_workspace_bytes(const kla_desc *desc)
+{
+    if (check_common(desc) != KLA_OK) return 0;
+    // segment bounds of a two-segment cut whose second segment is empty, then both halves of the segment arrays
+    const size_t cu_bytes = (((size_t)desc->B * 2 + 1) * sizeof(int32_t) + 255) & ~(size_t)255;
+    return cu_bytes + 2 * (size_t)desc->B * 2 * desc->H * desc->d_k * desc->d_v * sizeof(float);
+}
+
+kla_status kla_chunk_span_map(const kla_desc *desc, const void *k, const void *v, const float *log_alpha, const float *eta,
+                              float eps, float *phi_out, float *n_out)
+{
+    kla_status st = check_common(desc);
+    if (st != KLA_OK) return st;
+    if (!k || !v || !log_alpha || !eta || !phi_out || !n_out) return KLA_ERR_NULL;
+    if (!(eps >= 0.f) || !std::isfinite(eps)) return KLA_ERR_EPS;
+    if (desc->cu_seqlens || desc->n_seq != desc->B || desc->T < 1) return KLA_ERR_SHAPE;
+    if (desc->io_dtype != KLA_BF16) return KLA_ERR_DTYPE;
+    if ((int64_t)desc->B * desc->T >= (int64_t)1 << 31) return KLA_ERR_SHAPE;
+    if (!aligned16(k) || !aligned16(v) || !aligned16(log_alpha) || !aligned16(eta) || !aligned16(phi_out) || !aligned16(n_out))
+        return KLA_ERR_ALIGN;
+    const size_t need = kla_chunk_span_map_workspace_bytes(desc);
+    if (!desc->workspace || desc->workspace_bytes < need) return KLA_ERR_WORKSPACE;
+    if (!aligned16(desc->workspace)) return KLA_ERR_ALIGN;
+    st = check_arch();
+    if (st != KLA_OK) return st;
+    cudaStream_t stream = (cudaStream_t)desc->stream;
+    // The whole input as the first of two segments per sequence (the second is empty): segment pass 1 of the chunk
+    // kernel then gives the map and the zero-start state of exactly that span.
+    char *ws = (char *)desc->workspace;
+    int32_t *cu_seg = (int32_t *)ws;
+    const size_t cu_bytes = (((size_t)desc->B * 2 + 1) * sizeof(int32_t) + 255) & ~(size_t)255;
+    const size_t half = (size_t)desc->B * 2 * desc->H * desc->d_k * desc->d_v;
+    float *map = (float *)(ws + cu_bytes), *local = map + half;
+    if (launch_seg_bounds(cu_seg, desc->B, desc->T, 2, ((desc->T + 63) / 64) * 64, stream) != cudaSuccess) return KLA_ERR_LAUNCH;
+    ChunkParams p;
+    p.q = k;   // never read out: pass 1 forms no outputs (the tensor map only needs a valid address)
+    p.k = k; p.v = v;
+    p.log_alpha = log_alpha; p.eta = eta;
+    p.init_state = nullptr;
+    p.out = nullptr;
+    p.final_state = local;
+    p.cu_seqlens = cu_seg;
+    p.status_word = desc->status_word;
+    p.B = desc->B; p.T = desc->T; p.H = desc->H; p.n_seq = desc->B * 2;
+    p.eps = eps;
+    p.seg_pass = 1; p.seg_G = 2;
+    p.variant = ((desc->flags & KLA_FLAG_COEFF_ETA) ? VARIANT_COEFF_ETA : 0) | ((desc->flags & KLA_FLAG_NO_PAIR) ? VARIANT_NO_PAIR : 0) |
+                ((desc->flags & KLA_FLAG_WY_FORM) ? VARIANT_WY : 0);
+    p.map_state = map;
+    if (launch_chunk_tc(p, desc->d_k, desc->io_dtype, KLA_F32, stream) != cudaSuccess) return KLA_ERR_LAUNCH;
+    // segment 0 of sequence b sits at index 2 b of the segment arrays
+    const size_t one = (size_t)desc->H * desc->d_k * desc->d_v * sizeof(float);
+    if (cudaMemcpy2DAsync(phi_out, one, map, 2 * one, one, (size_t)desc->B, cudaMemcpyDeviceToDevice, stream) != cudaSuccess ||
+        cudaMemcpy2DAsync(n_out, one, local, 2 * one, one, (size_t)desc->B, cudaMemcpyDeviceToDevice, stream) != cudaSuccess)
+        return KLA_ERR_LAUNCH;
+    return KLA_OK;
+}
+
+kla_status kla_state_chain(const kla_desc *desc, int32_t n_spans, const float *init_state, const float *phi, const float *n,
+                           float *start_out)
+{
+    kla_status st = check_common(desc);
+    if (st != KLA_OK) return st;
+    if (!phi || !n || !start_out) return KLA_ERR_NULL;
+    if (n_spans < 1) return KLA_ERR_SHAPE;
+    if (!aligned16(phi) || !aligned16(n) || !aligned16(start_out) || !aligned16(init_state)) return KLA_ERR_ALIGN;
+    st = check_arch();
+    if (st != KLA_OK) return st;
+    return launch_seg_combine(init_state, phi, n, start_out, desc->B, desc->H, n_spans, desc->d_k, (cudaStream_t)desc->stream) == cudaSuccess
+               ? KLA_OK : KLA_ERR_LAUNCH;
+}
+
 static kla_status check_decode(const kla_desc *d, const void *q, const void *k, const void *v,
                                const float *log_alpha, const float *eta, float eps,
                                float *state, void *out)

@@ -8,6 +8,8 @@ the coefficient of Eq. (3) in fp64 (C, `kla_oracle.c`).  `chunkwise.forward_chun
 Algorithm 1 (right panel, Eqs. 7-9) in numpy fp64; the tests use it to pin the reading of the
 chunk formulas against the recurrence.
 
+`forward(..., diagonal_gates=True)` is the diagonal-gated extension of Appendix B.5 (a decay per row of the state).
+
 Pins (tests/test_oracle_pins.py): Kaczmarz projection (Theorem 1), residual contraction (Eq. 5),
 proximal stationarity (Prop. 1), minimum-norm change, pure decay at eta=0, chunkwise == tokenwise
 for several chunk sizes, brute force over the unrolled product form (Table 7) on T<=8, reduction
@@ -31,6 +33,8 @@ def _load():
         lib.kla_oracle_forward.argtypes = [ctypes.c_int, ctypes.POINTER(ctypes.c_int64),
                                            ctypes.c_int, ctypes.c_int, ctypes.c_int,
                                            dp, dp, dp, dp, dp, ctypes.c_double, dp, dp, dp]
+        lib.kla_oracle_forward_dg.restype = ctypes.c_int
+        lib.kla_oracle_forward_dg.argtypes = lib.kla_oracle_forward.argtypes
         lib.kla_oracle_decode_step.restype = ctypes.c_int
         lib.kla_oracle_decode_step.argtypes = [ctypes.c_int] * 4 + [dp] * 5 + [ctypes.c_double, dp, dp]
         lib.kla_oracle_set_variant.restype = None
@@ -69,11 +73,12 @@ def set_threads(n: int) -> None:
     _load().kla_oracle_set_threads(int(n))
 
 
-def forward_packed(q, k, v, log_alpha, eta, eps, cu_seqlens, init_state=None, want_final=True):
+def forward_packed(q, k, v, log_alpha, eta, eps, cu_seqlens, init_state=None, want_final=True, diagonal_gates=False):
     """Packed variable-length forward.
 
     q, k [n_tok, H, d_k]; v [n_tok, H, d_v]; log_alpha, eta [n_tok, H];
     cu_seqlens int[n_seq+1]; init_state [n_seq, H, d_k, d_v] or None (zeros).
+    `diagonal_gates`: log_alpha is [n_tok, H, d_k], one decay per row of the state (Appendix B.5).
     Returns (out [n_tok, H, d_v], final_state [n_seq, H, d_k, d_v] or None, threads_used).
     """
     lib = _load()
@@ -81,7 +86,7 @@ def forward_packed(q, k, v, log_alpha, eta, eps, cu_seqlens, init_state=None, wa
     n_tok, H, d_k = q.shape
     d_v = v.shape[-1]
     assert k.shape == (n_tok, H, d_k) and v.shape == (n_tok, H, d_v)
-    assert la.shape == (n_tok, H) and et.shape == (n_tok, H)
+    assert la.shape == ((n_tok, H, d_k) if diagonal_gates else (n_tok, H)) and et.shape == (n_tok, H)
     cu = np.ascontiguousarray(np.asarray(cu_seqlens, dtype=np.int64))
     n_seq = cu.shape[0] - 1
     assert cu[0] == 0 and cu[-1] == n_tok and np.all(np.diff(cu) >= 0)
@@ -91,22 +96,25 @@ def forward_packed(q, k, v, log_alpha, eta, eps, cu_seqlens, init_state=None, wa
         assert s0.shape == (n_seq, H, d_k, d_v)
     out = np.zeros((n_tok, H, d_v), dtype=np.float64)
     fin = np.zeros((n_seq, H, d_k, d_v), dtype=np.float64) if want_final else None
-    thr = lib.kla_oracle_forward(n_seq, cu.ctypes.data_as(ctypes.POINTER(ctypes.c_int64)), H, d_k, d_v,
+    fn = lib.kla_oracle_forward_dg if diagonal_gates else lib.kla_oracle_forward
+    thr = fn(n_seq, cu.ctypes.data_as(ctypes.POINTER(ctypes.c_int64)), H, d_k, d_v,
                                  _ptr(q), _ptr(k), _ptr(v), _ptr(la), _ptr(et), float(eps),
                                  _ptr(s0), _ptr(out), _ptr(fin))
     return out, fin, thr
 
 
-def forward(q, k, v, log_alpha, eta, eps, init_state=None, want_final=True):
-    """Fixed-length forward: q, k [B, T, H, d_k]; v [B, T, H, d_v]; log_alpha, eta [B, T, H];
-    init_state [B, H, d_k, d_v] or None.  Returns (out [B, T, H, d_v], final_state, threads)."""
+def forward(q, k, v, log_alpha, eta, eps, init_state=None, want_final=True, diagonal_gates=False):
+    """Fixed-length forward: q, k [B, T, H, d_k]; v [B, T, H, d_v]; log_alpha, eta [B, T, H] (log_alpha
+    [B, T, H, d_k] with `diagonal_gates`); init_state [B, H, d_k, d_v] or None.
+    Returns (out [B, T, H, d_v], final_state, threads)."""
     q = np.asarray(q)
     B, T, H, d_k = q.shape
     d_v = np.asarray(v).shape[-1]
     cu = np.arange(B + 1, dtype=np.int64) * T
+    la = _f64(log_alpha).reshape((B * T, H, d_k) if diagonal_gates else (B * T, H))
     out, fin, thr = forward_packed(_f64(q).reshape(B * T, H, d_k), _f64(k).reshape(B * T, H, d_k),
-                                   _f64(v).reshape(B * T, H, d_v), _f64(log_alpha).reshape(B * T, H),
-                                   _f64(eta).reshape(B * T, H), eps, cu, init_state, want_final)
+                                   _f64(v).reshape(B * T, H, d_v), la,
+                                   _f64(eta).reshape(B * T, H), eps, cu, init_state, want_final, diagonal_gates)
     return out.reshape(B, T, H, d_v), fin, thr
 
 

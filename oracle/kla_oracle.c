@@ -144,6 +144,60 @@ int kla_oracle_decode_step(int B, int H, int d_k, int d_v, const double *q, cons
     return threads;
 }
 
+/*
+ * Diagonal-gated KLA (Appendix B.5, "Extension to diagonal gating"; the decay-agnostic remark of the proofs): the decay
+ * operator is D_t = diag(alpha_t) with alpha_t a vector over d_k, so the decay scales the ROWS of S,
+ *
+ *     S~ = diag(exp(log_alpha_t)) S_{t-1},
+ *
+ * and everything after it (residual, coefficient of Eq. 3, rank-one write, read-out) is the loop body above unchanged:
+ * the Kaczmarz coefficient depends on S~ and k_t only, not on how S~ was produced.  Same layouts as kla_oracle_forward
+ * except log_alpha [n_tok, H, d_k].
+ */
+static void kla_token_update_dg(double *S, int d_k, int d_v, const double *q, const double *k, const double *v,
+                                const double *log_alpha, double eta, double eps, double *e, double *o)
+{
+    /* row-wise decay, then the scalar-gated update with alpha = 1 (log_alpha = 0) */
+    for (int i = 0; i < d_k; ++i) {
+        const double a = exp(log_alpha[i]);
+        for (int j = 0; j < d_v; ++j) S[(size_t)i * d_v + j] *= a;
+    }
+    kla_token_update(S, d_k, d_v, q, k, v, 0.0, eta, eps, e, o);
+}
+
+int kla_oracle_forward_dg(int n_seq, const int64_t *cu_seqlens, int H, int d_k, int d_v,
+                          const double *q, const double *k, const double *v,
+                          const double *log_alpha, const double *eta, double eps,
+                          const double *init_state, double *out, double *final_state)
+{
+    int threads = 1;
+#ifdef _OPENMP
+    threads = omp_get_max_threads();
+#endif
+    const size_t ss = (size_t)d_k * d_v;
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+    for (int n = 0; n < n_seq; ++n) {
+        for (int h = 0; h < H; ++h) {
+            double *S = (double *)malloc(ss * sizeof(double));
+            double *e = (double *)malloc((size_t)d_v * sizeof(double));
+            if (init_state)
+                memcpy(S, init_state + ((size_t)n * H + h) * ss, ss * sizeof(double));
+            else
+                memset(S, 0, ss * sizeof(double));
+            for (int64_t t = cu_seqlens[n]; t < cu_seqlens[n + 1]; ++t) {
+                const size_t th = (size_t)t * H + h;
+                kla_token_update_dg(S, d_k, d_v, q + th * d_k, k + th * d_k, v + th * d_v,
+                                    log_alpha + th * d_k, eta[th], eps, e, out + th * d_v);
+            }
+            if (final_state)
+                memcpy(final_state + ((size_t)n * H + h) * ss, S, ss * sizeof(double));
+            free(S);
+            free(e);
+        }
+    }
+    return threads;
+}
+
 void kla_oracle_set_threads(int n)
 {
 #ifdef _OPENMP

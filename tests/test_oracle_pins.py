@@ -294,3 +294,79 @@ def test_variant_qnorm_divides_the_readout_only():
     # and the default is restored on leaving the context
     o3, _, _ = oracle.forward(q, k, v, la, eta, 1e-3, s0)
     np.testing.assert_array_equal(o3, o0)
+
+
+# ---- diagonal-gated extension (Appendix B.5; decay-agnostic remark): a decay per row of the state ----------------------
+def _rand_dg(rng, B=1, T=7, H=2, d_k=4, d_v=3, eta=None):
+    q, k, v, _, eta, s0 = _rand_problem(rng, B=B, T=T, H=H, d_k=d_k, d_v=d_v, eta=eta)
+    la = -np.log1p(np.exp(rng.standard_normal((B, T, H, d_k))))
+    return q, k, v, la, eta, s0
+
+
+def _dg_states(q, k, v, la, eta, eps, s0):
+    return [oracle.forward(q[:, :t], k[:, :t], v[:, :t], la[:, :t], eta[:, :t], eps, s0, diagonal_gates=True)[1]
+            for t in range(1, q.shape[1] + 1)]
+
+
+def test_dg_constant_gate_vector_is_the_scalar_gate():
+    rng = RNG(31)
+    q, k, v, la, eta, s0 = _rand_problem(rng)
+    o1, f1, _ = oracle.forward(q, k, v, la, eta, 0.2, s0)
+    o2, f2, _ = oracle.forward(q, k, v, np.repeat(la[..., None], q.shape[-1], -1), eta, 0.2, s0, diagonal_gates=True)
+    np.testing.assert_allclose(o2, o1, rtol=0, atol=1e-13)
+    np.testing.assert_allclose(f2, f1, rtol=0, atol=1e-13)
+
+
+def test_dg_brute_force_with_explicit_transition_matrices():
+    """S_t = (I - beta k k^T) diag(alpha_t) S_{t-1} + beta k v^T with explicit d_k x d_k matrices, d_k != d_v so that a
+    decay applied to the wrong index of the state cannot pass; the read-out is taken from the post-write state."""
+    rng = RNG(32)
+    q, k, v, la, eta, s0 = _rand_dg(rng, T=6, d_k=4, d_v=2)
+    eps = 0.05
+    out, fin, _ = oracle.forward(q, k, v, la, eta, eps, s0, diagonal_gates=True)
+    for b in range(q.shape[0]):
+        for h in range(q.shape[2]):
+            S = s0[b, h].copy()
+            for t in range(q.shape[1]):
+                kt, vt = k[b, t, h], v[b, t, h]
+                beta = eta[b, t, h] / (kt @ kt + eps)
+                M = (np.eye(4) - beta * np.outer(kt, kt)) @ np.diag(np.exp(la[b, t, h]))
+                S = M @ S + beta * np.outer(kt, vt)
+                np.testing.assert_allclose(out[b, t, h], S.T @ q[b, t, h], rtol=0, atol=1e-12)
+            np.testing.assert_allclose(fin[b, h], S, rtol=0, atol=1e-12)
+
+
+def test_dg_eta_zero_is_pure_row_decay():
+    rng = RNG(33)
+    q, k, v, la, eta, s0 = _rand_dg(rng, eta=0.0)
+    out, fin, _ = oracle.forward(q, k, v, la, eta, 1e-6, s0, diagonal_gates=True)
+    gam = np.exp(np.cumsum(la, axis=1))                       # [B, T, H, d_k]
+    np.testing.assert_allclose(fin, gam[:, -1][..., None] * s0, rtol=0, atol=1e-13)
+    np.testing.assert_allclose(out, np.einsum("bhkv,bthk->bthv", s0, gam * q), rtol=0, atol=1e-12)
+
+
+def test_dg_projection_and_contraction_hold_for_any_decay_operator():
+    """Theorem 1 and Eq. 5 use only the decayed state S~ and k_t (decay-agnostic remark)."""
+    rng = RNG(34)
+    q, k, v, la, eta, s0 = _rand_dg(rng, eta=1.0)
+    for t, S in enumerate(_dg_states(q, k, v, la, eta, 0.0, s0)):
+        np.testing.assert_allclose(np.einsum("bhkv,bhk->bhv", S, k[:, t]), v[:, t], rtol=0, atol=1e-12)
+    q, k, v, la, eta, s0 = _rand_dg(rng)
+    eps, prev = 0.4, s0
+    for t, S in enumerate(_dg_states(q, k, v, la, eta, eps, s0)):
+        decayed = np.exp(la[:, t])[..., None] * prev
+        e_before = v[:, t] - np.einsum("bhkv,bhk->bhv", decayed, k[:, t])
+        e_after = v[:, t] - np.einsum("bhkv,bhk->bhv", S, k[:, t])
+        nk = np.sum(k[:, t] ** 2, axis=-1)
+        np.testing.assert_allclose(e_after, (1.0 - eta[:, t] * nk / (nk + eps))[..., None] * e_before, rtol=0, atol=1e-12)
+        prev = S
+
+
+def test_dg_state_handoff():
+    rng = RNG(35)
+    q, k, v, la, eta, s0 = _rand_dg(rng, T=9)
+    o, f, _ = oracle.forward(q, k, v, la, eta, 0.1, s0, diagonal_gates=True)
+    o1, f1, _ = oracle.forward(q[:, :4], k[:, :4], v[:, :4], la[:, :4], eta[:, :4], 0.1, s0, diagonal_gates=True)
+    o2, f2, _ = oracle.forward(q[:, 4:], k[:, 4:], v[:, 4:], la[:, 4:], eta[:, 4:], 0.1, f1, diagonal_gates=True)
+    np.testing.assert_allclose(np.concatenate([o1, o2], 1), o, rtol=0, atol=1e-13)
+    np.testing.assert_allclose(f2, f, rtol=0, atol=1e-13)

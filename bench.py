@@ -297,6 +297,24 @@ def wy_leg(w, t, dev, steps, warmup):
     return {"workload": w.name, "ms": ms, **stats, "mtok_per_s": B * T / (ms * 1e-3) / 1e6}
 
 
+def dg_leg(dev, steps, warmup, peaks):
+    """Diagonal-gated extension (Appendix B.5) on the headline shape: token-recurrent CUDA-core kernel."""
+    import torch
+    from paper_2605_08587_b200 import kla_dg_fwd, workloads as W
+    w = W.config_dg()
+    t = [x.to(dev) for x in (w.q, w.k, w.v, w.log_alpha, w.eta)]
+    s0 = w.init_state.to(dev)
+    B, T, H, d = w.q.shape
+    out = torch.empty((B, T, H, d), device=dev, dtype=torch.bfloat16)
+    fin = torch.empty((B, H, d, d), device=dev, dtype=torch.float32)
+    stats = {}
+    ms = time_launches(lambda: kla_dg_fwd(*t, w.eps, init_state=s0, out=out, final_state=fin), steps, warmup,
+                       torch.cuda.current_stream(), stats)
+    nbytes = B * T * H * (3 * d * 2 + d * 2 + d * 4 + 4) + 2 * B * H * d * d * 4   # q, k, v, out, the gate vector, eta; states
+    return {"workload": w.name, "ms": ms, **stats, "mtok_per_s": B * T / (ms * 1e-3) / 1e6, "algorithmic_bytes": nbytes,
+            "achieved_gbs": nbytes / (ms * 1e-3) / 1e9, "roofline_frac": nbytes / (peaks["hbm_gbs"] * 1e9) / (ms * 1e-3), "bound": "hbm"}
+
+
 def e2e_leg(w, dev, steps, warmup, groups=8):
     """Same step, host buffers: pinned host -> device copies of every input, the launches, and the
     device -> host read of out and final state, all inside the timed region.  The batch is cut into `groups`
@@ -441,6 +459,7 @@ def run_ours(args):
         extras["chunk_cfg3_long_context"] = chunk_leg(W.config3(), dev, 20, 3, peaks, torch.bfloat16)
         extras["chunk_cfg5_varlen"] = chunk_leg(W.config5(), dev, 20, 3, peaks, torch.bfloat16)
         extras["chunk_cfg2_wy_form"] = wy_leg(w, t, dev, 20, 3)
+        extras["dg_fwd_layer_shape"] = dg_leg(dev, 10, 3, peaks)
         if not args.no_cpu_baseline:
             extras["chunk_cfg3_long_context"]["cpu_baseline"] = oracle_chunk_workload(W.config3())
             extras["chunk_cfg5_varlen"]["cpu_baseline"] = oracle_chunk_workload(W.config5())

@@ -233,6 +233,26 @@ kla_status kla_decode_steps(const kla_desc *desc, int32_t n_steps, const void *q
                             const void *v, const float *log_alpha, const float *eta, float eps,
                             float *state_inout, void *out);
 
+/*
+ * Diagonal-gated KLA (Appendix B.5, "Extension to diagonal gating"; the decay-agnostic remark of Appendix A): the decay
+ * of the recurrence at the top of this file becomes a vector over d_k,
+ *
+ *     S~ = diag(exp(log_alpha_t)) S_{t-1}         (row i of the state decays by exp(log_alpha_t[i])),
+ *
+ * and the residual, the coefficient of Eq. 3, the write and the read-out are unchanged.  Arguments as kla_chunk_fwd /
+ * kla_decode_step except
+ *   log_alpha   [B, T, H, d_k] fp32 (decode: [B, H, d_k])
+ * and no chunk length, workspace or segment flags: the recurrence is evaluated token by token on CUDA cores, in fp32,
+ * with the state of every (sequence, head) in registers (the chunkwise form with elementwise decay products is not
+ * built).  Packed input (cu_seqlens), KLA_FLAG_COEFF_ETA and KLA_FLAG_QNORM are supported; fp32 or bf16 q, k, v.
+ */
+kla_status kla_dg_fwd(const kla_desc *desc, const void *q, const void *k, const void *v,
+                      const float *log_alpha, const float *eta, float eps,
+                      const float *init_state, void *out, float *final_state);
+kla_status kla_dg_decode_step(const kla_desc *desc, const void *q, const void *k, const void *v,
+                              const float *log_alpha, const float *eta, float eps,
+                              float *state_inout, void *out);
+
 /* Static, NUL-terminated description of a status code. */
 const char *kla_status_str(kla_status s);
 

@@ -23,7 +23,7 @@ def KLA_FLAG_SEGMENTS(g: int) -> int:
 
 
 EXPORTS = ["kla_chunk_fwd_workspace_bytes", "kla_chunk_fwd", "kla_chunk_fwd_timed", "kla_chunk_fwd_static_scratch",
-           "kla_chunk_span_map_workspace_bytes", "kla_chunk_span_map", "kla_state_chain", "kla_decode_step", "kla_decode_steps",
+           "kla_chunk_span_map_workspace_bytes", "kla_chunk_span_map", "kla_state_chain", "kla_dg_fwd", "kla_dg_decode_step", "kla_decode_step", "kla_decode_steps",
            "kla_status_str", "kla_launch_count"]
 
 
@@ -71,6 +71,10 @@ def load():
     lib.kla_state_chain.argtypes = [dp, ctypes.c_int32, fp, fp, fp, fp]
     lib.kla_decode_step.restype = ctypes.c_int
     lib.kla_decode_step.argtypes = [dp, vp, vp, vp, fp, fp, ctypes.c_float, fp, vp]
+    lib.kla_dg_fwd.restype = ctypes.c_int
+    lib.kla_dg_fwd.argtypes = [dp, vp, vp, vp, fp, fp, ctypes.c_float, fp, vp, fp]
+    lib.kla_dg_decode_step.restype = ctypes.c_int
+    lib.kla_dg_decode_step.argtypes = lib.kla_decode_step.argtypes
     lib.kla_decode_steps.restype = ctypes.c_int
     lib.kla_decode_steps.argtypes = [dp, ctypes.c_int32, vp, vp, vp, fp, fp, ctypes.c_float, fp, vp]
     lib.kla_status_str.restype = ctypes.c_char_p
@@ -282,5 +286,49 @@ def kla_decode_steps(q, k, v, log_alpha, eta, eps, state_inout, out=None, out_dt
         code = lib.kla_decode_steps(ctypes.byref(desc), n, _dev(q, "q"), _dev(k, "k"), _dev(v, "v"),
                                     _dev(log_alpha, "log_alpha", torch.float32), _dev(eta, "eta", torch.float32),
                                     float(eps), _dev(state_inout, "state_inout", torch.float32), _dev(out, "out"))
+    _check(code)
+    return out
+
+
+def kla_dg_fwd(q, k, v, log_alpha, eta, eps, init_state=None, out=None, final_state=None, cu_seqlens=None, host_seqlens=None,
+               out_dtype=None, flags=KLA_FLAG_NONE, want_final_state=True):
+    """Diagonal-gated forward (include/kla.h: kla_dg_fwd): as kla_chunk_fwd with log_alpha [B, T, H, d_k], one decay per
+    row of the state.  Returns (out, final_state)."""
+    lib = load()
+    B, T, H, d_k = q.shape
+    d_v = v.shape[-1]
+    if tuple(log_alpha.shape) != (B, T, H, d_k) or tuple(eta.shape) != (B, T, H):
+        raise ValueError("log_alpha must be [B, T, H, d_k] and eta [B, T, H]")
+    n_seq, hs = B, None
+    if cu_seqlens is not None:
+        hs = (cu_seqlens.cpu() if host_seqlens is None else host_seqlens).contiguous()
+        n_seq = cu_seqlens.numel() - 1
+    if out is None:
+        out = torch.empty((B, T, H, d_v), device=q.device, dtype=out_dtype or q.dtype)
+    if final_state is None and want_final_state:
+        final_state = torch.empty((n_seq, H, d_k, d_v), device=q.device, dtype=torch.float32)
+    desc = KlaDesc(B=B, T=T, H=H, d_k=d_k, d_v=d_v, n_seq=n_seq, cu_seqlens=_dev(cu_seqlens, "cu_seqlens"),
+                   host_seqlens=hs.data_ptr() if hs is not None else None, io_dtype=_dt(q), out_dtype=_dt(out), flags=flags,
+                   workspace=None, workspace_bytes=0, status_word=None, stream=_stream(q.device))
+    with torch.cuda.device(q.device):
+        code = lib.kla_dg_fwd(ctypes.byref(desc), _dev(q, "q"), _dev(k, "k"), _dev(v, "v"), _dev(log_alpha, "log_alpha", torch.float32),
+                              _dev(eta, "eta", torch.float32), float(eps), _dev(init_state, "init_state", torch.float32),
+                              _dev(out, "out"), _dev(final_state, "final_state", torch.float32))
+    _check(code)
+    return out, final_state
+
+
+def kla_dg_decode_step(q, k, v, log_alpha, eta, eps, state_inout, out=None, out_dtype=None, flags=KLA_FLAG_NONE):
+    """One diagonal-gated decode step (include/kla.h: kla_dg_decode_step): log_alpha [B, H, d_k]; state updated in place."""
+    lib = load()
+    B, H, d_k = q.shape
+    d_v = v.shape[-1]
+    if out is None:
+        out = torch.empty((B, H, d_v), device=q.device, dtype=out_dtype or q.dtype)
+    desc = _decode_desc(q, v, out, B, H, d_k, d_v, flags)
+    with torch.cuda.device(q.device):
+        code = lib.kla_dg_decode_step(ctypes.byref(desc), _dev(q, "q"), _dev(k, "k"), _dev(v, "v"),
+                                      _dev(log_alpha, "log_alpha", torch.float32), _dev(eta, "eta", torch.float32), float(eps),
+                                      _dev(state_inout, "state_inout", torch.float32), _dev(out, "out"))
     _check(code)
     return out

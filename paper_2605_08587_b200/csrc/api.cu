@@ -397,6 +397,44 @@ kla_status kla_decode_step(const kla_desc *desc, const void *q, const void *k, c
     return kla_decode_steps(desc, 1, q, k, v, log_alpha, eta, eps, state_inout, out);
 }
 
+kla_status kla_dg_fwd(const kla_desc *desc, const void *q, const void *k, const void *v,
+                      const float *log_alpha, const float *eta, float eps,
+                      const float *init_state, void *out, float *final_state)
+{
+    // the same host-side checks as the chunk forward (chunk 64 stands in: there is no chunk length here)
+    kla_status st = check_chunk_args(desc, q, k, v, log_alpha, eta, eps, 64, init_state, out, final_state, false);
+    if (st != KLA_OK) return st;
+    st = check_arch();
+    if (st != KLA_OK) return st;
+    cudaStream_t stream = (cudaStream_t)desc->stream;
+    if (desc->T == 0) {
+        if (final_state) {
+            const size_t bytes = (size_t)desc->n_seq * desc->H * desc->d_k * desc->d_v * sizeof(float);
+            cudaError_t e = init_state ? cudaMemcpyAsync(final_state, init_state, bytes, cudaMemcpyDeviceToDevice, stream)
+                                       : cudaMemsetAsync(final_state, 0, bytes, stream);
+            if (e != cudaSuccess) return KLA_ERR_LAUNCH;
+        }
+        return KLA_OK;
+    }
+    return launch_dg_scan(q, k, v, log_alpha, eta, init_state, out, final_state, desc->cu_seqlens, desc->T, desc->H, desc->n_seq,
+                          desc->d_k, eps, (desc->flags & KLA_FLAG_COEFF_ETA) ? 1 : 0, (desc->flags & KLA_FLAG_QNORM) ? 1 : 0,
+                          desc->io_dtype, desc->out_dtype, stream) == cudaSuccess ? KLA_OK : KLA_ERR_LAUNCH;
+}
+
+kla_status kla_dg_decode_step(const kla_desc *desc, const void *q, const void *k, const void *v,
+                              const float *log_alpha, const float *eta, float eps,
+                              float *state_inout, void *out)
+{
+    kla_status st = check_decode(desc, q, k, v, log_alpha, eta, eps, state_inout, out);
+    if (st != KLA_OK) return st;
+    st = check_arch();
+    if (st != KLA_OK) return st;
+    // one token per sequence; every warp reads its columns of the state before it writes them, so the update is in place
+    return launch_dg_scan(q, k, v, log_alpha, eta, state_inout, out, state_inout, nullptr, 1, desc->H, desc->B, desc->d_k, eps,
+                          (desc->flags & KLA_FLAG_COEFF_ETA) ? 1 : 0, (desc->flags & KLA_FLAG_QNORM) ? 1 : 0, desc->io_dtype,
+                          desc->out_dtype, (cudaStream_t)desc->stream) == cudaSuccess ? KLA_OK : KLA_ERR_LAUNCH;
+}
+
 const char *kla_status_str(kla_status s)
 {
     switch (s) {

@@ -66,6 +66,10 @@ cudaError_t launch_seq_order(const int32_t *cu_seqlens, int n_seq, int32_t *orde
 // start[b, 0] = init (or 0); start[b, g + 1] = map[b, g] . start[b, g] + local[b, g]   (d x d products, fp32)
 cudaError_t launch_seg_combine(const float *init_state, const float *map, const float *local, float *start, int B, int H,
                                int G, int d, cudaStream_t stream);
+// Diagonal-gated recurrence, token by token on CUDA cores (dg_scan.cu); log_alpha [n_tok, H, d].
+cudaError_t launch_dg_scan(const void *q, const void *k, const void *v, const float *log_alpha, const float *eta,
+                           const float *init_state, void *out, float *final_state, const int32_t *cu_seqlens, int T, int H,
+                           int n_seq, int d, float eps, int coeff_eta, int qnorm, int io_dtype, int out_dtype, cudaStream_t stream);
 // True when the tensor-core kernel covers this case.
 bool chunk_tc_supported(int d, int chunk, int io_dtype);
 

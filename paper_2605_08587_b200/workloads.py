@@ -125,3 +125,14 @@ def config5(n_seq=32, max_len=8192, H=16, d=64, chunk=64, seed=4, lengths=None):
     return ChunkWorkload("cfg5_varlen_n%d_tok%d_H%d_d%d" % (n_seq, n_tok, H, d), q.bfloat16(),
                          k.bfloat16(), v.bfloat16(), log_alpha, eta, 1e-6, chunk, cu_seqlens=cu,
                          meta={"dtype": "bf16", "lengths": lens.tolist()})
+
+
+def config_dg(B=8, H=8, T=4096, d=128, seed=5, dtype=torch.bfloat16, init_state=True):
+    """Diagonal-gated variant of the layer-shaped workload (Appendix B.5): as config 2, with one decay per key dimension,
+    log_alpha [B, T, H, d] = -softplus(N(0,1)) / 8 drawn independently per dimension (drawn last, after the initial state)."""
+    gen = torch.Generator().manual_seed(seed)
+    q, k, v, eta, _ = _layer_shaped(gen, B, T, H, d, 0.5)
+    s0 = (0.02 * torch.randn(B, H, d, d, generator=gen)).float().contiguous() if init_state else None
+    log_alpha = (-torch.nn.functional.softplus(torch.randn(B, T, H, d, generator=gen)) / 8.0).float().contiguous()
+    return ChunkWorkload("dg_%s_B%d_H%d_T%d_d%d" % ("bf16" if dtype == torch.bfloat16 else "f32", B, H, T, d), q.to(dtype),
+                         k.to(dtype), v.to(dtype), log_alpha, eta, 1e-6, 0, init_state=s0, meta={"dtype": str(dtype), "diagonal_gates": True})

@@ -31,7 +31,7 @@ UNIT = "Mtok/s"
 WORKLOAD = "cfg2_bf16_B8_H8_T4096_d128_chunk64"   # the same string in both arms
 # dram__bytes_read.sum + dram__bytes_write.sum of one headline launch of the chunk kernel, from the ncu capture
 # summarised under profiles/; None while the kernel has changed since the counters were taken.
-CHUNK_TC_DRAM_BYTES_PER_LAUNCH = None
+CHUNK_TC_DRAM_BYTES_PER_LAUNCH = 253634560   # 203.79 MB read + 49.85 MB written
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -451,6 +451,10 @@ def run_ours(args):
             extras["chunk_cfg3_long_context"] = chunk_leg(W.config3(), dev, 2, 1, peaks, torch.bfloat16)
         elif args.also == "varlen":
             extras["chunk_cfg5_varlen"] = chunk_leg(W.config5(), dev, 2, 1, peaks, torch.bfloat16)
+        elif args.also == "wy":
+            extras["chunk_cfg2_wy_form"] = wy_leg(w, t, dev, 2, 1)
+        elif args.also == "dg":
+            extras["dg_fwd_layer_shape"] = dg_leg(dev, 2, 1, peaks)
     if not args.quick:
         # decode: calls of 1024 consecutive steps on 1024 distinct token vectors, state carried in place
         extras["decode_cfg4"] = decode_leg(dev, 1024, 5, 1, peaks)
@@ -497,7 +501,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--quick", action="store_true", help="profiling mode: headline kernel only (no e2e, decode, long-context, varlen or CPU legs)")
-    ap.add_argument("--also", default="", choices=["", "decode", "decode64", "long", "varlen"],
+    ap.add_argument("--also", default="", choices=["", "decode", "decode64", "long", "varlen", "wy", "dg"],
                     help="with --quick: run one more leg after the headline kernel (used for profiling)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

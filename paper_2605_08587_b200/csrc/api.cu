@@ -108,7 +108,9 @@ static SegPlan plan_segments(const kla_desc *d, int32_t chunk)
         for (int G = 2; G <= 32 && chunks / G >= 8; ++G) {
             const int len = (chunks + G - 1) / G, Ge = (chunks + len - 1) / len;
             if (Ge < 2) continue;
-            const double cost = 0.8 * waves(units * 2 * (Ge - 1)) * len + (double)waves(units * Ge) * len + 2.0 * Ge;
+            // measured on the 65K single-sequence workload (per-pass device times): a chunk of pass 1 (no outputs) takes 0.86 of a
+            // main-pass chunk, and chaining the maps costs 2.2 chunk periods per segment
+            const double cost = 0.86 * waves(units * 2 * (Ge - 1)) * len + (double)waves(units * Ge) * len + 2.2 * Ge;
             if (cost < best) {
                 best = cost;
                 best_len = len;

@@ -167,77 +167,6 @@ __device__ __forceinline__ void split2h(float a, float b, uint32_t &hi, uint32_t
 }
 
 
-// ---- the blocked inverse of I + B X on the warp-level tensor instruction ------------------------------------------------------
-// The block products T_10 = -T_11 (B_1 X_10 T_00) at block sizes 16 and 32 are small dense products whose operands sit
-// in shared memory in fp32.  With CUDA-core FMAs every multiply-add fetches its operands from shared memory again (the
-// products then take most of the pre group's time and most of the SM's shared-memory bandwidth, which the tcgen05 products
-// need for their operand tiles); mma.sync m16n8k16 takes whole fragments into registers once.  Operands are split into
-// bf16 hi/lo pairs in registers and multiplied in three terms, accumulated in fp32.
-__device__ __forceinline__ void mma_16816(float (&c)[4], const uint32_t (&a)[4], const uint32_t (&b)[2])
-{
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
-                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
-}
-// c (16 x 8) += A (16 x K, rows lda floats apart) . B (K x 8, rows ldb floats apart), both fp32 in shared memory.  Fragment
-// layout of the instruction (g = lane / 4, t = lane % 4): c[0,1] = C[g][2t, 2t+1], c[2,3] = C[g+8][2t, 2t+1].
-__device__ __forceinline__ void warp_tile_product(float (&c)[4], int K, const float *Ap, int lda, const float *Bp, int ldb, int lane)
-{
-    const int g = lane >> 2, t = lane & 3;
-    float c1[4] = {0.f, 0.f, 0.f, 0.f}, c2[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll 1
-    for (int k0 = 0; k0 < K; k0 += 16) {
-        const float2 a00 = *reinterpret_cast<const float2 *>(Ap + g * lda + k0 + 2 * t);
-        const float2 a10 = *reinterpret_cast<const float2 *>(Ap + (g + 8) * lda + k0 + 2 * t);
-        const float2 a01 = *reinterpret_cast<const float2 *>(Ap + g * lda + k0 + 2 * t + 8);
-        const float2 a11 = *reinterpret_cast<const float2 *>(Ap + (g + 8) * lda + k0 + 2 * t + 8);
-        const float b0 = Bp[(k0 + 2 * t) * ldb + g], b1 = Bp[(k0 + 2 * t + 1) * ldb + g];
-        const float b2 = Bp[(k0 + 2 * t + 8) * ldb + g], b3 = Bp[(k0 + 2 * t + 9) * ldb + g];
-        uint32_t ah[4], al[4], bh[2], bl[2];
-        split2(a00.x, a00.y, ah[0], al[0]);
-        split2(a10.x, a10.y, ah[1], al[1]);
-        split2(a01.x, a01.y, ah[2], al[2]);
-        split2(a11.x, a11.y, ah[3], al[3]);
-        split2(b0, b1, bh[0], bl[0]);
-        split2(b2, b3, bh[1], bl[1]);
-        mma_16816(c, ah, bh);     // three accumulators: the instruction's latency is long, so the terms must not queue
-        mma_16816(c1, ah, bl);    // behind one another
-        mma_16816(c2, al, bh);
-    }
-#pragma unroll
-    for (int e = 0; e < 4; ++e) c[e] += c1[e] + c2[e];
-}
-// One level of the inverse (see merge_level in chunk_pieces.cuh for the algebra), block size BS = 16 or 32: every warp of
-// the pre group takes one 16 x 8 tile of the result (BS = 16: four tiles, warps 0..3; BS = 32: eight).  `mm` (rows LDT
-// floats apart) holds the intermediate product.  Out of line, one copy for both sizes: the pre group's code has to stay
-// small (instruction fetch is what the whole CTA stalls on first when the roles' loops outgrow the instruction cache).
-__device__ __noinline__ void merge_level_mma(int BS, float *tl, float *mm, const float *bet, int pw, int lane)
-{
-    const int NTL = BS / 8;                        // column tiles per block
-    const bool act = pw < (32 / BS) * (BS / 16) * NTL;
-    const int nt = pw % NTL, mt = (pw / NTL) % (BS / 16), pr = pw / (NTL * (BS / 16));
-    const int rb = (2 * pr + 1) * BS, cb = 2 * pr * BS;
-    const int g = lane >> 2, t = lane & 3;
-    if (act) {
-        // M = B_1 X_10 T_00
-        float c[4] = {0.f, 0.f, 0.f, 0.f};
-        warp_tile_product(c, BS, tl + (rb + 16 * mt) * LDT + cb, LDT, tl + cb * LDT + cb + 8 * nt, LDT, lane);
-        const float s0 = bet[rb + 16 * mt + g], s1 = bet[rb + 16 * mt + g + 8];
-        float *d = mm + (pr * BS + 16 * mt + g) * LDT + 8 * nt + 2 * t;
-        *reinterpret_cast<float2 *>(d) = make_float2(s0 * c[0], s0 * c[1]);
-        *reinterpret_cast<float2 *>(d + 8 * LDT) = make_float2(s1 * c[2], s1 * c[3]);
-    }
-    pg_sync();
-    if (act) {
-        // T_10 = -T_11 M
-        float c[4] = {0.f, 0.f, 0.f, 0.f};
-        warp_tile_product(c, BS, tl + (rb + 16 * mt) * LDT + rb, LDT, mm + (pr * BS) * LDT + 8 * nt, LDT, lane);
-        float *d = tl + (rb + 16 * mt + g) * LDT + cb + 8 * nt + 2 * t;
-        *reinterpret_cast<float2 *>(d) = make_float2(-c[0], -c[1]);
-        *reinterpret_cast<float2 *>(d + 8 * LDT) = make_float2(-c[2], -c[3]);
-    }
-    pg_sync();
-}
 // X = A^- o K K^T: this thread's row i, columns chh * 32 .. + 31 of the K K^T accumulator at tbase (two loads of 16
 // columns: four loads of eight paid the TMEM latency four times, one of 32 doubled the code), into the solve matrix.
 // Returns the diagonal element G_ii = ||k_i||^2 if it lies in these columns (else 0).
@@ -859,9 +788,12 @@ kla_chunk_wy_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             const float *bet = sm.beta[sc];
             if (pt < 64) substitute_diag_blocks(sm.tl, bet, pt);
             pg_sync();
+            // (CUDA-core FMAs: block products on the warp-level tensor instruction, mma.sync with bf16 hi/lo register fragments,
+            // were measured too -- they slow every tcgen05 product of the CTA down, 272 -> 420 us when tried in the default
+            // kernel, so the two tensor paths are not mixed)
             merge_level<8>(sm.tl, mm, LDT, bet, pt);
-            merge_level_mma(16, sm.tl, mm, bet, pt >> 5, lane);
-            merge_level_mma(32, sm.tl, mm, bet, pt >> 5, lane);
+            merge_level<16>(sm.tl, mm, LDT, bet, pt);
+            merge_level<32>(sm.tl, mm, LDT, bet, pt);
             // ---- T B D_gamma tiles (this CTA only); the W product of this CTA's previous chunk has read the old ones -----------
             bool okd = true;
             if (o > 0 && pt >= PG_T - 32) okd = wait(B_W_DONE, (uint32_t)((o - 1) & 1));

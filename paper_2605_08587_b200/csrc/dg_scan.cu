@@ -12,38 +12,44 @@
 // in registers for the whole sequence (columns never interact: the write is k e^T).  Per token: the decayed state is
 // never stored -- a_c = sum_j alpha_j S_jc k_j is reduced over the warp with a reduce-scatter butterfly (9 shuffles for
 // the 8 columns instead of 40), the residuals are gathered back (8 shuffles), S_jc <- alpha_j S_jc + beta k_j e_c is one
-// FMA on top of the decay, and the read-out is a second reduce-scatter.  The next token's operands are loaded while
-// the current one is processed.
+// FMA on top of the decay, and the read-out is a second reduce-scatter.  Operands are requested three tokens ahead and
+// prepared one token ahead (see the loop).
 #include "common.cuh"
 
 namespace kla {
 
 namespace {
 
-constexpr int WC = 8;          // state columns per warp
+#ifndef DG_WC
+#define DG_WC 8   // state columns per warp (4: twice the warps, but every warp prepares every token: 3.4 ms against 3.0 ms)
+#endif
 constexpr int WARPS = 4;       // warps (column groups) per block
 
-// Sums over the warp of x[0..7], by halving: afterwards every lane holds the complete sum of column (lane >> 2) & 7.
-__device__ __forceinline__ float reduce_scatter8(const float (&x)[WC], int lane)
+// Sums over the warp of x[0..WC-1] (WC = 4 or 8 state columns per warp), by halving: afterwards every lane holds the
+// complete sum of column col_of_lane<WC>(lane).
+template <int WC>
+__device__ __forceinline__ int col_of_lane(int lane) { return WC == 8 ? (lane >> 2) & 7 : (lane >> 3) & 3; }
+template <int WC>
+__device__ __forceinline__ int lane_of_col(int c) { return WC == 8 ? c << 2 : c << 3; }
+template <int WC>
+__device__ __forceinline__ float reduce_scatter(const float (&x)[WC], int lane)
 {
-    float y[4], z[2], w;
-    const bool b4 = lane & 16, b3 = lane & 8, b2 = lane & 4;
+    float y[WC];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const float keep = b4 ? x[4 + i] : x[i], give = b4 ? x[i] : x[4 + i];
-        y[i] = keep + __shfl_xor_sync(0xffffffffu, give, 16);
-    }
+    for (int i = 0; i < WC; ++i) y[i] = x[i];
+    int n = WC, off = 16;
 #pragma unroll
-    for (int i = 0; i < 2; ++i) {
-        const float keep = b3 ? y[2 + i] : y[i], give = b3 ? y[i] : y[2 + i];
-        z[i] = keep + __shfl_xor_sync(0xffffffffu, give, 8);
+    for (; n > 1; n >>= 1, off >>= 1) {   // halve the number of columns held, summing with the partner that keeps the other half
+        const bool hi = lane & off;
+#pragma unroll
+        for (int i = 0; i < n / 2; ++i) {
+            const float keep = hi ? y[n / 2 + i] : y[i], give = hi ? y[i] : y[n / 2 + i];
+            y[i] = keep + __shfl_xor_sync(0xffffffffu, give, off);
+        }
     }
-    {
-        const float keep = b2 ? z[1] : z[0], give = b2 ? z[0] : z[1];
-        w = keep + __shfl_xor_sync(0xffffffffu, give, 4);
-    }
-    w += __shfl_xor_sync(0xffffffffu, w, 2);
-    w += __shfl_xor_sync(0xffffffffu, w, 1);
+    float w = y[0];
+#pragma unroll
+    for (; off > 0; off >>= 1) w += __shfl_xor_sync(0xffffffffu, w, off);
     return w;
 }
 __device__ __forceinline__ float warp_sum(float x)
@@ -66,7 +72,7 @@ struct DgParams {
     int32_t coeff_eta, qnorm;
 };
 
-template <int D, typename IO, typename OUT>
+template <int D, int WC, typename IO, typename OUT>
 __global__ void __launch_bounds__(32 * WARPS) kla_dg_scan_kernel(DgParams p)
 {
     constexpr int J = D / 32;              // rows per lane
@@ -83,102 +89,120 @@ __global__ void __launch_bounds__(32 * WARPS) kla_dg_scan_kernel(DgParams p)
         tok0 = n * p.T;
         len = p.T;
     }
-    const int c0 = cg * WC;                 // first column of this warp
-    const int myc = (lane >> 2) & 7;        // the column whose sums this lane ends up with
+    const int c0 = cg * WC;                    // first column of this warp
+    const int myc = col_of_lane<WC>(lane);     // the column whose sums this lane ends up with
     const size_t sbase = ((size_t)n * p.H + h) * D * D;
 
     float S[J][WC];
 #pragma unroll
     for (int j = 0; j < J; ++j) {
-        if (p.init_state) {
-            const float4 a = *reinterpret_cast<const float4 *>(p.init_state + sbase + (size_t)(lane + 32 * j) * D + c0);
-            const float4 b = *reinterpret_cast<const float4 *>(p.init_state + sbase + (size_t)(lane + 32 * j) * D + c0 + 4);
-            S[j][0] = a.x; S[j][1] = a.y; S[j][2] = a.z; S[j][3] = a.w;
-            S[j][4] = b.x; S[j][5] = b.y; S[j][6] = b.z; S[j][7] = b.w;
-        } else {
 #pragma unroll
-            for (int c = 0; c < WC; ++c) S[j][c] = 0.f;
+        for (int c = 0; c < WC; c += 4) {
+            float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (p.init_state) a = *reinterpret_cast<const float4 *>(p.init_state + sbase + (size_t)(lane + 32 * j) * D + c0 + c);
+            S[j][c] = a.x; S[j][c + 1] = a.y; S[j][c + 2] = a.z; S[j][c + 3] = a.w;
         }
     }
 
     const IO *qp = reinterpret_cast<const IO *>(p.q), *kp = reinterpret_cast<const IO *>(p.k), *vp = reinterpret_cast<const IO *>(p.v);
     OUT *op = reinterpret_cast<OUT *>(p.out);
-    // operands of one token: this lane's rows of q, k and of the decay; the value of this lane's column; the gate
-    struct Tok { float q[J], k[J], a[J], v, eta; };
-    auto load = [&](int t) {
-        Tok x;
-        const size_t th = (size_t)(tok0 + t) * p.H + h;
+    // Three-stage software pipeline per warp.  Raw operands of token t + 3 are requested from global memory and not touched
+    // (any use, even a conversion, would wait for them); the operands of token t + 1 are prepared from raw values requested two
+    // iterations earlier -- everything that does not depend on the state: alpha_j, alpha_j k_j, beta k_j (Eq. 3), 1 / ||q||;
+    // token t is applied to the state.
+    struct Raw { IO q[J], k[J], v; float la[J], eta; };
+    struct Tok { float q[J], a[J], ak[J], bk[J], v, qinv; };
+    auto request = [&](int t) {
+        Raw r;
+        const size_t th = (size_t)(tok0 + min(t, len - 1)) * p.H + h;   // (past the end: the last token again, never used)
 #pragma unroll
         for (int j = 0; j < J; ++j) {
-            x.q[j] = to_f32(qp[th * D + lane + 32 * j]);
-            x.k[j] = to_f32(kp[th * D + lane + 32 * j]);
-            x.a[j] = __expf(p.log_alpha[th * D + lane + 32 * j]);
+            r.q[j] = qp[th * D + lane + 32 * j];
+            r.k[j] = kp[th * D + lane + 32 * j];
+            r.la[j] = p.log_alpha[th * D + lane + 32 * j];
         }
-        x.v = to_f32(vp[th * D + c0 + myc]);
-        x.eta = p.eta[th];
+        r.v = vp[th * D + c0 + myc];
+        r.eta = p.eta[th];
+        return r;
+    };
+    auto prepare = [&](const Raw &r) {
+        Tok x;
+        float k[J], nk = 0.f, nq = 0.f;
+#pragma unroll
+        for (int j = 0; j < J; ++j) {
+            x.q[j] = to_f32(r.q[j]);
+            k[j] = to_f32(r.k[j]);
+            x.a[j] = __expf(r.la[j]);
+            nk += k[j] * k[j];
+            nq += x.q[j] * x.q[j];
+        }
+        x.v = to_f32(r.v);
+        nk = warp_sum(nk);
+        const float beta = p.coeff_eta ? r.eta : r.eta / (nk + p.eps);   // Eq. 3
+        x.qinv = p.qnorm ? rsqrtf(warp_sum(nq)) : 1.f;
+#pragma unroll
+        for (int j = 0; j < J; ++j) {
+            x.ak[j] = x.a[j] * k[j];
+            x.bk[j] = beta * k[j];
+        }
         return x;
     };
-    Tok cur;
-    if (len > 0) cur = load(0);
-    for (int t = 0; t < len; ++t) {
-        Tok nxt = cur;
-        if (t + 1 < len) nxt = load(t + 1);
-        // ||k||^2 (and ||q||^2 for the normalised read-out)
-        float nk = 0.f, nq = 0.f;
+    if (len > 0) {
+        Raw r1 = request(1), r2 = request(2);
+        Tok cur = prepare(request(0));
+        for (int t = 0; t < len; ++t) {
+            const Raw r3 = request(t + 3);
+            const Tok nxt = prepare(r1);
+            // a_c = sum_j alpha_j S_jc k_j, residual e_c = v_c - a_c
+            float part[WC];
 #pragma unroll
-        for (int j = 0; j < J; ++j) {
-            nk += cur.k[j] * cur.k[j];
-            nq += cur.q[j] * cur.q[j];
-        }
-        nk = warp_sum(nk);
-        const float beta = p.coeff_eta ? cur.eta : cur.eta / (nk + p.eps);
-        // a_c = sum_j alpha_j S_jc k_j
-        float part[WC];
+            for (int c = 0; c < WC; ++c) {
+                float s = 0.f;
 #pragma unroll
-        for (int c = 0; c < WC; ++c) {
-            float s = 0.f;
-#pragma unroll
-            for (int j = 0; j < J; ++j) s += (cur.a[j] * cur.k[j]) * S[j][c];
-            part[c] = s;
-        }
-        const float e_mine = cur.v - reduce_scatter8(part, lane);   // residual of column myc
-        // S_jc <- alpha_j S_jc + beta k_j e_c;  o_c = sum_j S_jc q_j
-#pragma unroll
-        for (int c = 0; c < WC; ++c) {
-            const float e = __shfl_sync(0xffffffffu, e_mine, c << 2);
-            float s = 0.f;
-#pragma unroll
-            for (int j = 0; j < J; ++j) {
-                S[j][c] = cur.a[j] * S[j][c] + (beta * cur.k[j]) * e;
-                s += S[j][c] * cur.q[j];
+                for (int j = 0; j < J; ++j) s += cur.ak[j] * S[j][c];
+                part[c] = s;
             }
-            part[c] = s;
+            const float e_mine = cur.v - reduce_scatter<WC>(part, lane);   // residual of column myc
+            // S_jc <- alpha_j S_jc + beta k_j e_c;  o_c = sum_j S_jc q_j
+#pragma unroll
+            for (int c = 0; c < WC; ++c) {
+                const float e = __shfl_sync(0xffffffffu, e_mine, lane_of_col<WC>(c));
+                float s = 0.f;
+#pragma unroll
+                for (int j = 0; j < J; ++j) {
+                    S[j][c] = cur.a[j] * S[j][c] + cur.bk[j] * e;
+                    s += S[j][c] * cur.q[j];
+                }
+                part[c] = s;
+            }
+            const float o = reduce_scatter<WC>(part, lane) * cur.qinv;
+            if ((lane & (WC == 8 ? 3 : 7)) == 0) op[((size_t)(tok0 + t) * p.H + h) * D + c0 + myc] = from_f32<OUT>(o);
+            cur = nxt;
+            r1 = r2;
+            r2 = r3;
         }
-        float o = reduce_scatter8(part, lane);
-        if (p.qnorm) o *= rsqrtf(warp_sum(nq));
-        if ((lane & 3) == 0) op[((size_t)(tok0 + t) * p.H + h) * D + c0 + myc] = from_f32<OUT>(o);
-        cur = nxt;
     }
     if (p.final_state) {
 #pragma unroll
-        for (int j = 0; j < J; ++j) {
-            float *d = p.final_state + sbase + (size_t)(lane + 32 * j) * D + c0;
-            *reinterpret_cast<float4 *>(d) = make_float4(S[j][0], S[j][1], S[j][2], S[j][3]);
-            *reinterpret_cast<float4 *>(d + 4) = make_float4(S[j][4], S[j][5], S[j][6], S[j][7]);
-        }
+        for (int j = 0; j < J; ++j)
+#pragma unroll
+            for (int c = 0; c < WC; c += 4)
+                *reinterpret_cast<float4 *>(p.final_state + sbase + (size_t)(lane + 32 * j) * D + c0 + c) =
+                    make_float4(S[j][c], S[j][c + 1], S[j][c + 2], S[j][c + 3]);
     }
 }
 
 template <int D, typename IO>
 cudaError_t launch_io(const DgParams &p, int out_dtype, cudaStream_t stream)
 {
+    constexpr int WC = DG_WC;   // state columns per warp
     const int units = p.n_seq * p.H * (D / WC);
     if (units == 0) return cudaSuccess;
     const int blocks = (units + WARPS - 1) / WARPS;
     if (out_dtype == KLA_BF16)
-        kla_dg_scan_kernel<D, IO, __nv_bfloat16><<<blocks, 32 * WARPS, 0, stream>>>(p);
+        kla_dg_scan_kernel<D, WC, IO, __nv_bfloat16><<<blocks, 32 * WARPS, 0, stream>>>(p);
     else
-        kla_dg_scan_kernel<D, IO, float><<<blocks, 32 * WARPS, 0, stream>>>(p);
+        kla_dg_scan_kernel<D, WC, IO, float><<<blocks, 32 * WARPS, 0, stream>>>(p);
     count_launch(1);
     return cudaGetLastError();
 }

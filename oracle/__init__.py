@@ -9,6 +9,8 @@ Algorithm 1 (right panel, Eqs. 7-9) in numpy fp64; the tests use it to pin the r
 chunk formulas against the recurrence.
 
 `forward(..., diagonal_gates=True)` is the diagonal-gated extension of Appendix B.5 (a decay per row of the state).
+`backward` / `backward_packed` are the reverse-mode derivative of the recurrence (the training pass of Section 5.1),
+pinned by central differences of `forward`, closed forms and a library autograd run.
 
 Pins (tests/test_oracle_pins.py): Kaczmarz projection (Theorem 1), residual contraction (Eq. 5),
 proximal stationarity (Prop. 1), minimum-norm change, pure decay at eta=0, chunkwise == tokenwise
@@ -35,6 +37,10 @@ def _load():
                                            dp, dp, dp, dp, dp, ctypes.c_double, dp, dp, dp]
         lib.kla_oracle_forward_dg.restype = ctypes.c_int
         lib.kla_oracle_forward_dg.argtypes = lib.kla_oracle_forward.argtypes
+        lib.kla_oracle_backward.restype = ctypes.c_int
+        lib.kla_oracle_backward.argtypes = [ctypes.c_int, ctypes.POINTER(ctypes.c_int64),
+                                            ctypes.c_int, ctypes.c_int, ctypes.c_int,
+                                            dp, dp, dp, dp, dp, ctypes.c_double, dp, dp, dp] + [dp] * 6
         lib.kla_oracle_decode_step.restype = ctypes.c_int
         lib.kla_oracle_decode_step.argtypes = [ctypes.c_int] * 4 + [dp] * 5 + [ctypes.c_double, dp, dp]
         lib.kla_oracle_set_variant.restype = None
@@ -116,6 +122,48 @@ def forward(q, k, v, log_alpha, eta, eps, init_state=None, want_final=True, diag
                                    _f64(v).reshape(B * T, H, d_v), la,
                                    _f64(eta).reshape(B * T, H), eps, cu, init_state, want_final, diagonal_gates)
     return out.reshape(B, T, H, d_v), fin, thr
+
+
+def backward_packed(q, k, v, log_alpha, eta, eps, cu_seqlens, dout, init_state=None, dfinal=None):
+    """Gradients of a scalar loss through the packed forward, given dout = dL/dout [n_tok, H, d_v] and
+    dfinal = dL/dfinal_state [n_seq, H, d_k, d_v] or None (zeros).  Layouts as `forward_packed`.
+    Returns a dict with dq, dk, dv, dlog_alpha, deta, dinit (dL/dinit_state) and threads."""
+    lib = _load()
+    q, k, v, la, et, do = _f64(q), _f64(k), _f64(v), _f64(log_alpha), _f64(eta), _f64(dout)
+    n_tok, H, d_k = q.shape
+    d_v = v.shape[-1]
+    assert k.shape == (n_tok, H, d_k) and v.shape == (n_tok, H, d_v) and do.shape == (n_tok, H, d_v)
+    assert la.shape == (n_tok, H) and et.shape == (n_tok, H)
+    cu = np.ascontiguousarray(np.asarray(cu_seqlens, dtype=np.int64))
+    n_seq = cu.shape[0] - 1
+    assert cu[0] == 0 and cu[-1] == n_tok and np.all(np.diff(cu) >= 0)
+    s0 = _f64(init_state) if init_state is not None else None
+    df = _f64(dfinal) if dfinal is not None else None
+    for a in (s0, df):
+        assert a is None or a.shape == (n_seq, H, d_k, d_v)
+    g = dict(dq=np.zeros((n_tok, H, d_k)), dk=np.zeros((n_tok, H, d_k)), dv=np.zeros((n_tok, H, d_v)),
+             dlog_alpha=np.zeros((n_tok, H)), deta=np.zeros((n_tok, H)), dinit=np.zeros((n_seq, H, d_k, d_v)))
+    g["threads"] = lib.kla_oracle_backward(n_seq, cu.ctypes.data_as(ctypes.POINTER(ctypes.c_int64)), H, d_k, d_v,
+                                           _ptr(q), _ptr(k), _ptr(v), _ptr(la), _ptr(et), float(eps),
+                                           _ptr(s0), _ptr(do), _ptr(df), _ptr(g["dq"]), _ptr(g["dk"]), _ptr(g["dv"]),
+                                           _ptr(g["dlog_alpha"]), _ptr(g["deta"]), _ptr(g["dinit"]))
+    return g
+
+
+def backward(q, k, v, log_alpha, eta, eps, dout, init_state=None, dfinal=None):
+    """Fixed-length form of `backward_packed`: q, k [B, T, H, d_k]; v, dout [B, T, H, d_v]; log_alpha, eta [B, T, H]."""
+    q = np.asarray(q)
+    B, T, H, d_k = q.shape
+    d_v = np.asarray(v).shape[-1]
+    cu = np.arange(B + 1, dtype=np.int64) * T
+    g = backward_packed(_f64(q).reshape(B * T, H, d_k), _f64(k).reshape(B * T, H, d_k), _f64(v).reshape(B * T, H, d_v),
+                        _f64(log_alpha).reshape(B * T, H), _f64(eta).reshape(B * T, H), eps, cu,
+                        _f64(dout).reshape(B * T, H, d_v), init_state, dfinal)
+    for name, last in (("dq", d_k), ("dk", d_k), ("dv", d_v)):
+        g[name] = g[name].reshape(B, T, H, last)
+    for name in ("dlog_alpha", "deta"):
+        g[name] = g[name].reshape(B, T, H)
+    return g
 
 
 def decode_step(q, k, v, log_alpha, eta, eps, state):

@@ -198,6 +198,174 @@ int kla_oracle_forward_dg(int n_seq, const int64_t *cu_seqlens, int H, int d_k, 
     return threads;
 }
 
+/*
+ * Reverse-mode derivative of the recurrence above (the models of Section 5.1 are trained through it; the paper prints no
+ * backward pass, so this is the chain rule applied to the five lines of the loop body, last line first).  For a scalar
+ * loss L with dO_t = dL/do_t given for every token and dS_T = dL/dS_T given for the final state:
+ *
+ *   read-out   o = S_t^T qh  (qh = q, or q / ||q|| with the qnorm variant)
+ *                  G  += qh dO^T                 (G holds dL/dS_t)
+ *                  dqh = S_t dO ;  dq = dqh, or (dqh - qh (qh . dqh)) / ||q||
+ *   write      S_t = S~ + beta k e^T
+ *                  dbeta = k^T G e ;  dk = beta G e ;  de = beta G^T k
+ *   residual   e = v - S~^T k
+ *                  dv = de ;  dk -= S~ de ;  G -= k de^T   (G now holds dL/dS~)
+ *   coefficient  beta = eta / n, n = ||k||^2 + eps  (Eq. 3)
+ *                  deta = dbeta / n ;  dk += 2 k (-dbeta eta / n^2)        (beta = eta: deta = dbeta)
+ *   decay      S~ = exp(log_alpha) S_{t-1}
+ *                  dlog_alpha = <G, S~> ;  G <- exp(log_alpha) G            (G now holds dL/dS_{t-1})
+ *
+ * `Sprev` is S_{t-1}; the forward quantities of the token are recomputed from it.  `work` holds 2 d_k d_v + 2 d_v doubles.
+ */
+static void kla_token_backward(const double *Sprev, int d_k, int d_v, const double *q, const double *k,
+                               const double *v, double log_alpha, double eta, double eps, const double *dout,
+                               double *G, double *dq, double *dk, double *dv, double *dlog_alpha, double *deta,
+                               double *work)
+{
+    const size_t ss = (size_t)d_k * d_v;
+    double *St = work;          /* S~ = alpha S_{t-1} */
+    double *Sn = work + ss;     /* S_t */
+    double *e = work + 2 * ss;
+    double *de = e + d_v;
+    const double alpha = exp(log_alpha);
+    /* forward quantities of this token */
+    for (size_t x = 0; x < ss; ++x) St[x] = alpha * Sprev[x];
+    for (int j = 0; j < d_v; ++j) e[j] = v[j];
+    for (int i = 0; i < d_k; ++i)
+        for (int j = 0; j < d_v; ++j) e[j] -= St[(size_t)i * d_v + j] * k[i];
+    double nk = 0.0;
+    for (int i = 0; i < d_k; ++i) nk += k[i] * k[i];
+    const double n = nk + eps;
+    const double beta = g_coeff_eta ? eta : eta / n;
+    for (int i = 0; i < d_k; ++i)
+        for (int j = 0; j < d_v; ++j) Sn[(size_t)i * d_v + j] = St[(size_t)i * d_v + j] + beta * k[i] * e[j];
+    /* read-out */
+    double qnrm = 1.0;
+    if (g_qnorm) {
+        double nq = 0.0;
+        for (int i = 0; i < d_k; ++i) nq += q[i] * q[i];
+        qnrm = sqrt(nq);
+    }
+    double proj = 0.0;   /* qh . dqh */
+    for (int i = 0; i < d_k; ++i) {
+        const double qh = q[i] / qnrm;
+        double s = 0.0;
+        for (int j = 0; j < d_v; ++j) {
+            G[(size_t)i * d_v + j] += qh * dout[j];
+            s += Sn[(size_t)i * d_v + j] * dout[j];
+        }
+        dq[i] = s;       /* dqh for now */
+        proj += qh * s;
+    }
+    if (g_qnorm)
+        for (int i = 0; i < d_k; ++i) dq[i] = (dq[i] - (q[i] / qnrm) * proj) / qnrm;
+    /* rank-one write */
+    double dbeta = 0.0;
+    for (int j = 0; j < d_v; ++j) de[j] = 0.0;
+    for (int i = 0; i < d_k; ++i) {
+        double ge = 0.0;
+        for (int j = 0; j < d_v; ++j) {
+            ge += G[(size_t)i * d_v + j] * e[j];
+            de[j] += beta * G[(size_t)i * d_v + j] * k[i];
+        }
+        dbeta += k[i] * ge;
+        dk[i] = beta * ge;
+    }
+    /* residual */
+    for (int j = 0; j < d_v; ++j) dv[j] = de[j];
+    for (int i = 0; i < d_k; ++i) {
+        double s = 0.0;
+        for (int j = 0; j < d_v; ++j) {
+            s += St[(size_t)i * d_v + j] * de[j];
+            G[(size_t)i * d_v + j] -= k[i] * de[j];
+        }
+        dk[i] -= s;
+    }
+    /* coefficient, Eq. 3 */
+    if (g_coeff_eta) {
+        *deta = dbeta;
+    } else {
+        *deta = dbeta / n;
+        const double dn = -dbeta * eta / (n * n);
+        for (int i = 0; i < d_k; ++i) dk[i] += 2.0 * k[i] * dn;
+    }
+    /* decay */
+    double dla = 0.0;
+    for (size_t x = 0; x < ss; ++x) {
+        dla += G[x] * St[x];
+        G[x] *= alpha;
+    }
+    *dlog_alpha = dla;
+}
+
+/*
+ * Packed backward.  Inputs as kla_oracle_forward, plus dout [n_tok, H, d_v] and dfinal [n_seq, H, d_k, d_v] or NULL
+ * (zeros).  Outputs dq, dk [n_tok, H, d_k], dv [n_tok, H, d_v], dlog_alpha, deta [n_tok, H], dinit [n_seq, H, d_k, d_v]
+ * or NULL (skipped).  The reverse sweep needs S_{t-1} of every token: the forward sweep keeps the state at the start of
+ * every block of 64 tokens, and the states inside one block are recomputed from its start when the sweep reaches it.
+ */
+#define KLA_ORACLE_BWD_BLOCK 64
+int kla_oracle_backward(int n_seq, const int64_t *cu_seqlens, int H, int d_k, int d_v,
+                        const double *q, const double *k, const double *v,
+                        const double *log_alpha, const double *eta, double eps,
+                        const double *init_state, const double *dout, const double *dfinal,
+                        double *dq, double *dk, double *dv, double *dlog_alpha, double *deta, double *dinit)
+{
+    int threads = 1;
+#ifdef _OPENMP
+    threads = omp_get_max_threads();
+#endif
+    const size_t ss = (size_t)d_k * d_v;
+    const int L = KLA_ORACLE_BWD_BLOCK;
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+    for (int n = 0; n < n_seq; ++n) {
+        for (int h = 0; h < H; ++h) {
+            const int64_t t0 = cu_seqlens[n], len = cu_seqlens[n + 1] - t0;
+            const int64_t n_blocks = (len + L - 1) / L;
+            double *starts = (double *)malloc((size_t)(n_blocks + 1) * ss * sizeof(double));  /* state at each block start */
+            double *inside = (double *)malloc((size_t)(L + 1) * ss * sizeof(double));         /* S_{t-1} of a block's tokens */
+            double *G = (double *)malloc(ss * sizeof(double));
+            double *work = (double *)malloc((2 * ss + 2 * (size_t)d_v) * sizeof(double));
+            double *o = (double *)malloc((size_t)d_v * sizeof(double));
+            double *S = inside;   /* running state of the forward sweep */
+            if (init_state)
+                memcpy(S, init_state + ((size_t)n * H + h) * ss, ss * sizeof(double));
+            else
+                memset(S, 0, ss * sizeof(double));
+            for (int64_t i = 0; i < len; ++i) {
+                if (i % L == 0) memcpy(starts + (size_t)(i / L) * ss, S, ss * sizeof(double));
+                const size_t th = (size_t)(t0 + i) * H + h;
+                kla_token_update(S, d_k, d_v, q + th * d_k, k + th * d_k, v + th * d_v, log_alpha[th], eta[th], eps,
+                                 work, o);
+            }
+            if (dfinal)
+                memcpy(G, dfinal + ((size_t)n * H + h) * ss, ss * sizeof(double));
+            else
+                memset(G, 0, ss * sizeof(double));
+            for (int64_t b = n_blocks - 1; b >= 0; --b) {
+                const int64_t i0 = b * L, i1 = (i0 + L < len) ? i0 + L : len;
+                memcpy(inside, starts + (size_t)b * ss, ss * sizeof(double));
+                for (int64_t i = i0; i + 1 < i1; ++i) {   /* inside[j] = state before token i0 + j */
+                    double *nxt = inside + (size_t)(i - i0 + 1) * ss;
+                    memcpy(nxt, inside + (size_t)(i - i0) * ss, ss * sizeof(double));
+                    const size_t th = (size_t)(t0 + i) * H + h;
+                    kla_token_update(nxt, d_k, d_v, q + th * d_k, k + th * d_k, v + th * d_v, log_alpha[th], eta[th],
+                                     eps, work, o);
+                }
+                for (int64_t i = i1 - 1; i >= i0; --i) {
+                    const size_t th = (size_t)(t0 + i) * H + h;
+                    kla_token_backward(inside + (size_t)(i - i0) * ss, d_k, d_v, q + th * d_k, k + th * d_k, v + th * d_v,
+                                       log_alpha[th], eta[th], eps, dout + th * d_v, G, dq + th * d_k, dk + th * d_k,
+                                       dv + th * d_v, dlog_alpha + th, deta + th, work);
+                }
+            }
+            if (dinit) memcpy(dinit + ((size_t)n * H + h) * ss, G, ss * sizeof(double));
+            free(starts); free(inside); free(G); free(work); free(o);
+        }
+    }
+    return threads;
+}
+
 void kla_oracle_set_threads(int n)
 {
 #ifdef _OPENMP

@@ -370,3 +370,153 @@ def test_dg_state_handoff():
     o2, f2, _ = oracle.forward(q[:, 4:], k[:, 4:], v[:, 4:], la[:, 4:], eta[:, 4:], 0.1, f1, diagonal_gates=True)
     np.testing.assert_allclose(np.concatenate([o1, o2], 1), o, rtol=0, atol=1e-13)
     np.testing.assert_allclose(f2, f, rtol=0, atol=1e-13)
+
+
+# ---- reverse-mode derivative of the recurrence (training pass, Section 5.1) --------------------------------------------------
+# The backward oracle is pinned against things it does not compute itself: central differences of the (pinned) forward
+# oracle, closed forms worked out by hand for one token and for eta = 0, the composition rule of reverse mode over a split
+# sequence, and a library autograd run over a forward written with tensor operations.
+
+GRADS = ("dq", "dk", "dv", "dlog_alpha", "deta", "dinit")
+
+
+def _central_differences(loss, args, h=1e-6):
+    out = []
+    for x in args:
+        fd = np.zeros_like(x)
+        it = np.nditer(x, flags=["multi_index"])
+        for _ in it:
+            i = it.multi_index
+            old = x[i]
+            x[i] = old + h
+            lp = loss(*args)
+            x[i] = old - h
+            lm = loss(*args)
+            x[i] = old
+            fd[i] = (lp - lm) / (2 * h)
+        out.append(fd)
+    return out
+
+
+@pytest.mark.parametrize("coeff_eta,qnorm", [(False, False), (True, False), (False, True), (True, True)])
+def test_bwd_central_differences_of_the_forward_oracle(coeff_eta, qnorm):
+    rng = RNG(31)
+    q, k, v, la, eta, s0 = _rand_problem(rng, B=2, T=6, H=2, d_k=4, d_v=3)
+    la = 0.4 * la
+    do = rng.standard_normal(v.shape)
+    df = rng.standard_normal(s0.shape)
+    eps = 1e-2
+
+    def loss(q, k, v, la, eta, s0):
+        o, f, _ = oracle.forward(q, k, v, la, eta, eps, s0)
+        return float((o * do).sum() + (f * df).sum())
+
+    with oracle.variant(coeff_eta=coeff_eta, qnorm=qnorm):
+        g = oracle.backward(q, k, v, la, eta, eps, do, s0, df)
+        fd = _central_differences(loss, [q, k, v, la, eta, s0])
+    for name, ref in zip(GRADS, fd):
+        np.testing.assert_allclose(g[name], ref, rtol=0, atol=2e-8 * max(1.0, np.abs(ref).max()), err_msg=name)
+
+
+def test_bwd_one_token_from_an_empty_state_closed_form():
+    # S_0 = 0: o = beta (k.q) v with beta = eta / (|k|^2 + eps); L = dO . o, differentiated by hand.
+    rng = RNG(32)
+    d = 5
+    q, k, v, do = (rng.standard_normal(d) for _ in range(4))
+    eta, eps, la = 0.7, 0.05, -0.3
+    n = k @ k + eps
+    kq, vd = k @ q, v @ do
+    want = dict(dq=eta / n * vd * k, dk=eta / n * vd * q - 2 * eta * kq * vd / n ** 2 * k, dv=eta / n * kq * do,
+                deta=kq * vd / n, dlog_alpha=0.0)
+    g = oracle.backward(q[None, None, None], k[None, None, None], v[None, None, None], np.full((1, 1, 1), la),
+                        np.full((1, 1, 1), eta), eps, do[None, None, None])
+    for name, ref in want.items():
+        np.testing.assert_allclose(np.squeeze(g[name]), ref, rtol=0, atol=1e-13, err_msg=name)
+    # the initial state enters decayed: dL/dS_0 = alpha (I - beta k k^T) q dO^T
+    ref = np.exp(la) * np.outer(q - eta / n * kq * k, do)
+    np.testing.assert_allclose(g["dinit"][0, 0], ref, rtol=0, atol=1e-13)
+
+
+def test_bwd_eta_zero_is_the_derivative_of_pure_decay():
+    # eta = 0: S_t = Gamma_t S_0 with Gamma_t = exp(sum_{s<=t} log_alpha_s), o_t = Gamma_t S_0^T q_t.
+    rng = RNG(33)
+    q, k, v, la, eta, s0 = _rand_problem(rng, B=1, T=9, H=1, d_k=4, d_v=3, eta=0.0)
+    do = rng.standard_normal(v.shape)
+    g = oracle.backward(q, k, v, la, eta, 1e-6, do, s0)
+    Gam = np.exp(np.cumsum(la[0, :, 0]))
+    S0 = s0[0, 0]
+    Q, DO = q[0, :, 0], do[0, :, 0]
+    np.testing.assert_allclose(g["dq"][0, :, 0], Gam[:, None] * (DO @ S0.T), rtol=0, atol=1e-13)
+    np.testing.assert_allclose(g["dinit"][0, 0], np.einsum("t,ti,tj->ij", Gam, Q, DO), rtol=0, atol=1e-13)
+    per_tok = Gam * np.einsum("ti,ij,tj->t", Q, S0, DO)            # d o_t . dO_t / d log Gamma_t
+    np.testing.assert_allclose(g["dlog_alpha"][0, :, 0], np.cumsum(per_tok[::-1])[::-1], rtol=0, atol=1e-13)
+    np.testing.assert_allclose(g["dv"], 0.0, atol=0)               # nothing is written, so v is never read
+    assert np.abs(g["deta"]).max() > 1e-3                          # but the loss does depend on eta at eta = 0
+
+
+def test_bwd_composes_over_a_split_sequence_and_over_recompute_blocks():
+    # Reverse mode over [0, T) = reverse mode over [m, T) followed by [0, m) fed with the gradient of the hand-over state.
+    # T = 150 also crosses the 64-token blocks the oracle recomputes its states in, at a split (70) that is not a boundary.
+    rng = RNG(34)
+    T, m = 150, 70
+    q, k, v, la, eta, s0 = _rand_problem(rng, B=1, T=T, H=2, d_k=4, d_v=3)
+    la = 0.2 * la
+    do = rng.standard_normal(v.shape)
+    df = rng.standard_normal(s0.shape)
+    eps = 1e-3
+    whole = oracle.backward(q, k, v, la, eta, eps, do, s0, df)
+    _, mid, _ = oracle.forward(q[:, :m], k[:, :m], v[:, :m], la[:, :m], eta[:, :m], eps, s0)
+    late = oracle.backward(q[:, m:], k[:, m:], v[:, m:], la[:, m:], eta[:, m:], eps, do[:, m:], mid, df)
+    early = oracle.backward(q[:, :m], k[:, :m], v[:, :m], la[:, :m], eta[:, :m], eps, do[:, :m], s0, late["dinit"])
+    for name in GRADS[:-1]:
+        np.testing.assert_allclose(np.concatenate([early[name], late[name]], axis=1), whole[name], rtol=0, atol=1e-11)
+    np.testing.assert_allclose(early["dinit"], whole["dinit"], rtol=0, atol=1e-11)
+
+
+def test_bwd_matches_library_autograd():
+    torch = pytest.importorskip("torch")
+    rng = RNG(35)
+    T, d_k, d_v = 70, 6, 5
+    q, k, v, la, eta, s0 = _rand_problem(rng, B=1, T=T, H=1, d_k=d_k, d_v=d_v)
+    la = 0.3 * la
+    do = rng.standard_normal(v.shape)
+    df = rng.standard_normal(s0.shape)
+    eps = 1e-3
+    leaves = [torch.tensor(a, dtype=torch.float64, requires_grad=True)
+              for a in (q[0, :, 0], k[0, :, 0], v[0, :, 0], la[0, :, 0], eta[0, :, 0], s0[0, 0])]
+    tq, tk, tv, tla, teta, ts0 = leaves
+    S = ts0
+    outs = []
+    for t in range(T):
+        S = torch.exp(tla[t]) * S
+        e = tv[t] - S.T @ tk[t]
+        S = S + (teta[t] / (tk[t] @ tk[t] + eps)) * torch.outer(tk[t], e)
+        outs.append(S.T @ tq[t])
+    out = torch.stack(outs)
+    ref_o, ref_f, _ = oracle.forward(q, k, v, la, eta, eps, s0)
+    np.testing.assert_allclose(out.detach().numpy(), ref_o[0, :, 0], rtol=0, atol=1e-12)   # same function first
+    loss = (out * torch.tensor(do[0, :, 0])).sum() + (S * torch.tensor(df[0, 0])).sum()
+    loss.backward()
+    g = oracle.backward(q, k, v, la, eta, eps, do, s0, df)
+    got = [g["dq"][0, :, 0], g["dk"][0, :, 0], g["dv"][0, :, 0], g["dlog_alpha"][0, :, 0], g["deta"][0, :, 0], g["dinit"][0, 0]]
+    for name, a, leaf in zip(GRADS, got, leaves):
+        np.testing.assert_allclose(a, leaf.grad.numpy(), rtol=0, atol=1e-11, err_msg=name)
+
+
+def test_bwd_packed_equals_per_sequence_and_zero_length():
+    rng = RNG(36)
+    lens = [5, 0, 9]
+    cu = np.concatenate([[0], np.cumsum(lens)])
+    q, k, v, la, eta, _ = _rand_problem(rng, B=1, T=sum(lens), H=2, d_k=4, d_v=3)
+    s0 = rng.standard_normal((3, 2, 4, 3))
+    df = rng.standard_normal((3, 2, 4, 3))
+    do = rng.standard_normal(v.shape)
+    g = oracle.backward_packed(q[0], k[0], v[0], la[0], eta[0], 1e-3, cu, do[0], s0, df)
+    for n, (a, b) in enumerate(zip(cu[:-1], cu[1:])):
+        if a == b:
+            np.testing.assert_array_equal(g["dinit"][n], df[n])    # an empty sequence hands the gradient straight through
+            continue
+        one = oracle.backward(q[:, a:b], k[:, a:b], v[:, a:b], la[:, a:b], eta[:, a:b], 1e-3, do[:, a:b], s0[n:n + 1], df[n:n + 1])
+        for name in GRADS[:-1]:
+            np.testing.assert_array_equal(g[name][a:b], one[name][0])
+        np.testing.assert_array_equal(g["dinit"][n], one["dinit"][0])

@@ -253,6 +253,34 @@ kla_status kla_dg_decode_step(const kla_desc *desc, const void *q, const void *k
                               const float *log_alpha, const float *eta, float eps,
                               float *state_inout, void *out);
 
+/*
+ * Backward pass (training, Section 5.1): gradients of a scalar loss L through the recurrence at the top of this file.
+ * The paper prints no backward; this is reverse-mode differentiation of Algorithm 1 (left) with the coefficient of
+ * Eq. 3, token by token in reverse order (G = dL/dS_t carried backwards):
+ *
+ *     G += q dO_t^T ;  dq_t = S_t dO_t                                   (read-out)
+ *     dbeta = k^T G e ;  dk_t = beta G e ;  de = beta G^T k              (write)
+ *     dv_t = de ;  dk_t -= S~ de ;  G -= k de^T                          (residual)
+ *     deta_t = dbeta / n ;  dk_t -= 2 k dbeta beta / n, n = ||k||^2+eps  (coefficient, Eq. 3)
+ *     dlog_alpha_t = <G, S~> ;  G <- alpha_t G                           (decay)
+ *
+ * Inputs q, k, v, log_alpha, eta, eps, init_state: as kla_chunk_fwd (fixed-length or packed through desc->cu_seqlens /
+ * host_seqlens; desc->io_dtype; KLA_FLAG_COEFF_ETA and KLA_FLAG_QNORM are honoured, other flags ignored).
+ *   d_out          [B, T, H, d_v] io_dtype, dL/dout
+ *   d_final_state  [n_seq, H, d_k, d_v] fp32, dL/dfinal_state, or NULL for zeros
+ *   dq, dk         [B, T, H, d_k] fp32; dv [B, T, H, d_v] fp32; dlog_alpha, deta [B, T, H] fp32: fully overwritten
+ *   dinit_state    [n_seq, H, d_k, d_v] fp32, dL/dinit_state, or NULL to skip; an empty sequence gets d_final_state
+ * All arithmetic is fp32 on CUDA cores.  The forward states are not an input: they are recomputed (a state is kept every
+ * 16 tokens on a forward sweep, the ones in between are re-run when the reverse sweep reaches them), which needs
+ * desc->workspace of kla_bwd_workspace_bytes(desc) bytes: (B T / 16 + n_seq + 16 n_seq) x H x d_k x d_v fp32
+ * (host function; 0 for an invalid descriptor).  Errors as kla_chunk_fwd.
+ */
+size_t kla_bwd_workspace_bytes(const kla_desc *desc);
+kla_status kla_bwd(const kla_desc *desc, const void *q, const void *k, const void *v,
+                   const float *log_alpha, const float *eta, float eps, const float *init_state,
+                   const void *d_out, const float *d_final_state,
+                   float *dq, float *dk, float *dv, float *dlog_alpha, float *deta, float *dinit_state);
+
 /* Static, NUL-terminated description of a status code. */
 const char *kla_status_str(kla_status s);
 

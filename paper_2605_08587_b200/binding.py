@@ -23,7 +23,7 @@ def KLA_FLAG_SEGMENTS(g: int) -> int:
 
 
 EXPORTS = ["kla_chunk_fwd_workspace_bytes", "kla_chunk_fwd", "kla_chunk_fwd_timed", "kla_chunk_fwd_static_scratch",
-           "kla_chunk_span_map_workspace_bytes", "kla_chunk_span_map", "kla_state_chain", "kla_dg_fwd", "kla_dg_decode_step", "kla_decode_step", "kla_decode_steps",
+           "kla_chunk_span_map_workspace_bytes", "kla_chunk_span_map", "kla_state_chain", "kla_dg_fwd", "kla_dg_decode_step", "kla_bwd_workspace_bytes", "kla_bwd", "kla_decode_step", "kla_decode_steps",
            "kla_status_str", "kla_launch_count"]
 
 
@@ -75,6 +75,10 @@ def load():
     lib.kla_dg_fwd.argtypes = [dp, vp, vp, vp, fp, fp, ctypes.c_float, fp, vp, fp]
     lib.kla_dg_decode_step.restype = ctypes.c_int
     lib.kla_dg_decode_step.argtypes = lib.kla_decode_step.argtypes
+    lib.kla_bwd_workspace_bytes.restype = ctypes.c_size_t
+    lib.kla_bwd_workspace_bytes.argtypes = [dp]
+    lib.kla_bwd.restype = ctypes.c_int
+    lib.kla_bwd.argtypes = [dp, vp, vp, vp, fp, fp, ctypes.c_float, fp, vp, fp] + [fp] * 6
     lib.kla_decode_steps.restype = ctypes.c_int
     lib.kla_decode_steps.argtypes = [dp, ctypes.c_int32, vp, vp, vp, fp, fp, ctypes.c_float, fp, vp]
     lib.kla_status_str.restype = ctypes.c_char_p
@@ -316,6 +320,44 @@ def kla_dg_fwd(q, k, v, log_alpha, eta, eps, init_state=None, out=None, final_st
                               _dev(out, "out"), _dev(final_state, "final_state", torch.float32))
     _check(code)
     return out, final_state
+
+
+def kla_bwd(q, k, v, log_alpha, eta, eps, d_out, init_state=None, d_final_state=None, cu_seqlens=None, host_seqlens=None,
+            flags=KLA_FLAG_NONE, want_dinit_state=True, workspace=None):
+    """Backward pass (include/kla.h: kla_bwd): gradients of a scalar loss given d_out = dL/dout (dtype of q) and
+    d_final_state = dL/dfinal_state (or None).  Returns a dict of fp32 tensors dq, dk, dv, dlog_alpha, deta and
+    dinit_state (None unless asked for).  `workspace`: a uint8 CUDA tensor of at least kla_bwd_workspace_bytes, else
+    one is allocated here."""
+    lib = load()
+    B, T, H, d_k = q.shape
+    d_v = v.shape[-1]
+    if tuple(d_out.shape) != (B, T, H, d_v) or d_out.dtype != q.dtype:
+        raise ValueError("d_out must be [B, T, H, d_v] with the dtype of q")
+    n_seq, hs = B, None
+    if cu_seqlens is not None:
+        hs = (cu_seqlens.cpu() if host_seqlens is None else host_seqlens).contiguous()
+        n_seq = cu_seqlens.numel() - 1
+    f32 = dict(device=q.device, dtype=torch.float32)
+    g = dict(dq=torch.empty((B, T, H, d_k), **f32), dk=torch.empty((B, T, H, d_k), **f32), dv=torch.empty((B, T, H, d_v), **f32),
+             dlog_alpha=torch.empty((B, T, H), **f32), deta=torch.empty((B, T, H), **f32),
+             dinit_state=torch.empty((n_seq, H, d_k, d_v), **f32) if want_dinit_state else None)
+    desc = KlaDesc(B=B, T=T, H=H, d_k=d_k, d_v=d_v, n_seq=n_seq, cu_seqlens=_dev(cu_seqlens, "cu_seqlens"),
+                   host_seqlens=hs.data_ptr() if hs is not None else None, io_dtype=_dt(q), out_dtype=KLA_F32, flags=flags,
+                   workspace=None, workspace_bytes=0, status_word=None, stream=_stream(q.device))
+    need = int(lib.kla_bwd_workspace_bytes(ctypes.byref(desc)))
+    if workspace is None and need > 0:
+        workspace = torch.empty(need, device=q.device, dtype=torch.uint8)
+    if workspace is not None:
+        desc.workspace = _dev(workspace, "workspace")
+        desc.workspace_bytes = workspace.numel() * workspace.element_size()
+    with torch.cuda.device(q.device):
+        code = lib.kla_bwd(ctypes.byref(desc), _dev(q, "q"), _dev(k, "k"), _dev(v, "v"), _dev(log_alpha, "log_alpha", torch.float32),
+                           _dev(eta, "eta", torch.float32), float(eps), _dev(init_state, "init_state", torch.float32),
+                           _dev(d_out, "d_out"), _dev(d_final_state, "d_final_state", torch.float32),
+                           _dev(g["dq"], "dq"), _dev(g["dk"], "dk"), _dev(g["dv"], "dv"), _dev(g["dlog_alpha"], "dlog_alpha"),
+                           _dev(g["deta"], "deta"), _dev(g["dinit_state"], "dinit_state"))
+    _check(code)
+    return g
 
 
 def kla_dg_decode_step(q, k, v, log_alpha, eta, eps, state_inout, out=None, out_dtype=None, flags=KLA_FLAG_NONE):

@@ -7,8 +7,8 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libkla_b200.so")
-SOURCES = ["api.cu", "decode.cu", "chunk_simt.cu", "chunk_tc.cu", "chunk_wy.cu", "segscan.cu", "static_scratch.cu", "dg_scan.cu"]
-HEADERS = [os.path.join(CSRC, "common.cuh"), os.path.join(CSRC, "umma.cuh"), os.path.join(CSRC, "chunk_pieces.cuh"), os.path.join(ROOT, "include", "kla.h")]
+SOURCES = ["api.cu", "decode.cu", "chunk_simt.cu", "chunk_tc.cu", "chunk_wy.cu", "segscan.cu", "static_scratch.cu", "dg_scan.cu", "bwd_scan.cu"]
+HEADERS = [os.path.join(CSRC, "common.cuh"), os.path.join(CSRC, "umma.cuh"), os.path.join(CSRC, "chunk_pieces.cuh"), os.path.join(CSRC, "scan_pieces.cuh"), os.path.join(ROOT, "include", "kla.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I" + os.path.join(ROOT, "include"), "-I" + CSRC]
 

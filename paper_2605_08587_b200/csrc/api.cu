@@ -437,6 +437,36 @@ kla_status kla_dg_decode_step(const kla_desc *desc, const void *q, const void *k
                           desc->out_dtype, (cudaStream_t)desc->stream) == cudaSuccess ? KLA_OK : KLA_ERR_LAUNCH;
 }
 
+size_t kla_bwd_workspace_bytes(const kla_desc *desc)
+{
+    if (check_common(desc) != KLA_OK || desc->n_seq < 1) return 0;
+    return bwd_workspace_bytes(desc->n_seq, (long long)desc->B * desc->T, desc->H, desc->d_k);
+}
+
+kla_status kla_bwd(const kla_desc *desc, const void *q, const void *k, const void *v,
+                   const float *log_alpha, const float *eta, float eps, const float *init_state,
+                   const void *d_out, const float *d_final_state,
+                   float *dq, float *dk, float *dv, float *dlog_alpha, float *deta, float *dinit_state)
+{
+    // the forward's host-side checks (d_out stands where out does: same shape, required, aligned)
+    kla_status st = check_chunk_args(desc, q, k, v, log_alpha, eta, eps, 64, init_state, const_cast<void *>(d_out), nullptr, false);
+    if (st != KLA_OK) return st;
+    if (!dq || !dk || !dv || !dlog_alpha || !deta) return KLA_ERR_NULL;
+    if (!aligned16(dq) || !aligned16(dk) || !aligned16(dv) || !aligned16(dlog_alpha) || !aligned16(deta) ||
+        !aligned16(d_final_state) || !aligned16(dinit_state))
+        return KLA_ERR_ALIGN;
+    const size_t need = kla_bwd_workspace_bytes(desc);
+    if (need > 0 && (!desc->workspace || desc->workspace_bytes < need)) return KLA_ERR_WORKSPACE;
+    if (!aligned16(desc->workspace)) return KLA_ERR_ALIGN;
+    st = check_arch();
+    if (st != KLA_OK) return st;
+    cudaStream_t stream = (cudaStream_t)desc->stream;
+    return launch_bwd_scan(q, k, v, log_alpha, eta, init_state, d_out, d_final_state, dq, dk, dv, dlog_alpha, deta, dinit_state,
+                           desc->workspace, desc->cu_seqlens, desc->T, (long long)desc->B * desc->T, desc->H, desc->n_seq,
+                           desc->d_k, eps, (desc->flags & KLA_FLAG_COEFF_ETA) ? 1 : 0, (desc->flags & KLA_FLAG_QNORM) ? 1 : 0,
+                           desc->io_dtype, stream) == cudaSuccess ? KLA_OK : KLA_ERR_LAUNCH;
+}
+
 const char *kla_status_str(kla_status s)
 {
     switch (s) {

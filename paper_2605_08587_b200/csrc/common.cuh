@@ -70,6 +70,13 @@ cudaError_t launch_seg_combine(const float *init_state, const float *map, const 
 cudaError_t launch_dg_scan(const void *q, const void *k, const void *v, const float *log_alpha, const float *eta,
                            const float *init_state, void *out, float *final_state, const int32_t *cu_seqlens, int T, int H,
                            int n_seq, int d, float eps, int coeff_eta, int qnorm, int io_dtype, int out_dtype, cudaStream_t stream);
+// Reverse-mode derivative of the recurrence, token by token on CUDA cores (bwd_scan.cu); gradients in fp32.
+size_t bwd_workspace_bytes(int n_seq, long long n_tok, int H, int d);
+cudaError_t launch_bwd_scan(const void *q, const void *k, const void *v, const float *log_alpha, const float *eta,
+                            const float *init_state, const void *dout, const float *dfinal, float *dq, float *dk, float *dv,
+                            float *dlog_alpha, float *deta, float *dinit, void *workspace, const int32_t *cu_seqlens, int T,
+                            long long n_tok, int H, int n_seq, int d, float eps, int coeff_eta, int qnorm, int io_dtype,
+                            cudaStream_t stream);
 // True when the tensor-core kernel covers this case.
 bool chunk_tc_supported(int d, int chunk, int io_dtype);
 

@@ -15,6 +15,7 @@
 // FMA on top of the decay, and the read-out is a second reduce-scatter.  Operands are requested three tokens ahead and
 // prepared one token ahead (see the loop).
 #include "common.cuh"
+#include "scan_pieces.cuh"
 
 namespace kla {
 
@@ -24,40 +25,6 @@ namespace {
 #define DG_WC 8   // state columns per warp (4: twice the warps, but every warp prepares every token: 3.4 ms against 3.0 ms)
 #endif
 constexpr int WARPS = 4;       // warps (column groups) per block
-
-// Sums over the warp of x[0..WC-1] (WC = 4 or 8 state columns per warp), by halving: afterwards every lane holds the
-// complete sum of column col_of_lane<WC>(lane).
-template <int WC>
-__device__ __forceinline__ int col_of_lane(int lane) { return WC == 8 ? (lane >> 2) & 7 : (lane >> 3) & 3; }
-template <int WC>
-__device__ __forceinline__ int lane_of_col(int c) { return WC == 8 ? c << 2 : c << 3; }
-template <int WC>
-__device__ __forceinline__ float reduce_scatter(const float (&x)[WC], int lane)
-{
-    float y[WC];
-#pragma unroll
-    for (int i = 0; i < WC; ++i) y[i] = x[i];
-    int n = WC, off = 16;
-#pragma unroll
-    for (; n > 1; n >>= 1, off >>= 1) {   // halve the number of columns held, summing with the partner that keeps the other half
-        const bool hi = lane & off;
-#pragma unroll
-        for (int i = 0; i < n / 2; ++i) {
-            const float keep = hi ? y[n / 2 + i] : y[i], give = hi ? y[i] : y[n / 2 + i];
-            y[i] = keep + __shfl_xor_sync(0xffffffffu, give, off);
-        }
-    }
-    float w = y[0];
-#pragma unroll
-    for (; off > 0; off >>= 1) w += __shfl_xor_sync(0xffffffffu, w, off);
-    return w;
-}
-__device__ __forceinline__ float warp_sum(float x)
-{
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
-    return x;
-}
 
 struct DgParams {
     const void *q, *k, *v;

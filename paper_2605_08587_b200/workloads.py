@@ -136,3 +136,13 @@ def config_dg(B=8, H=8, T=4096, d=128, seed=5, dtype=torch.bfloat16, init_state=
     log_alpha = (-torch.nn.functional.softplus(torch.randn(B, T, H, d, generator=gen)) / 8.0).float().contiguous()
     return ChunkWorkload("dg_%s_B%d_H%d_T%d_d%d" % ("bf16" if dtype == torch.bfloat16 else "f32", B, H, T, d), q.to(dtype),
                          k.to(dtype), v.to(dtype), log_alpha, eta, 1e-6, 0, init_state=s0, meta={"dtype": str(dtype), "diagonal_gates": True})
+
+
+def upstream_grads(w: ChunkWorkload, seed=6, final=True):
+    """Seeded upstream gradients for a backward pass over workload `w`: d_out ~ N(0,1) in the dtype of v (shape of v)
+    and, with `final`, d_final_state ~ N(0,1) fp32 [n_seq, H, d_k, d_v] (else None)."""
+    gen = torch.Generator().manual_seed(seed)
+    d_out = torch.randn(w.v.shape, generator=gen).to(w.v.dtype).contiguous()
+    H, d_k, d_v = w.q.shape[2], w.q.shape[3], w.v.shape[3]
+    d_final = torch.randn((w.n_seq, H, d_k, d_v), generator=gen).float().contiguous() if final else None
+    return d_out, d_final

@@ -17,7 +17,7 @@
 // Work split: columns of S and G never interact, so a block owns 64 columns of one (sequence, head), one warp 8 of them,
 // lane l rows l, l + 32, ... (S_{t-1}, G and the prefetched next S_{t-1} in registers).  Sums over rows (S~^T k, G^T k)
 // are reduce-scatter butterflies inside the warp; sums over columns (dq, dk, dbeta, dlog_alpha) are per-warp partials
-// added up through shared memory once per token.  With d = 128 the two blocks of a head add their halves into
+// added up through shared memory once per block of 16 tokens.  With d = 128 the two blocks of a head add their halves into
 // zero-initialised outputs with one atomic each: two commutative additions, so the result does not depend on their order.
 #include "common.cuh"
 #include "scan_pieces.cuh"
@@ -26,10 +26,14 @@ namespace kla {
 
 namespace {
 
-constexpr int WC = 8;         // state columns per warp
-constexpr int WARPS = 8;      // warps per block (64 columns)
+#ifndef BWD_WC
+#define BWD_WC 4
+#endif
+constexpr int WC = BWD_WC;    // state columns per warp
+constexpr int WARPS = 64 / WC;   // warps per block (64 columns)
 constexpr int NT = 32 * WARPS;
-constexpr int L = 16;         // tokens between stored states (kla_bwd_workspace_bytes in api.cu uses the same figure)
+constexpr int L = 16;         // tokens between stored states
+constexpr int RL = WC == 8 ? 16 : 8;   // tokens between two additions of the warps' partial sums (shared memory: RL x WARPS x (2 d + 2) floats)
 
 struct BwdParams {
     const void *q, *k, *v, *dout;
@@ -46,13 +50,24 @@ struct BwdParams {
     int32_t coeff_eta;
 };
 
+// One block of L tokens as the steps read it.
+template <int D>
+struct Stage {
+    float k[L][D], q[L][D];       // q already divided by ||q|| when the read-out is normalised
+    float v[L][64], dout[L][64];  // the 64 columns of this thread block
+    float alpha[L], beta[L], nrm[L], qinv[L];
+};
+
 template <int D, typename IO, bool QN>
 __global__ void __launch_bounds__(NT, 1) kla_bwd_scan_kernel(BwdParams p)
 {
     constexpr int J = D / 32;            // rows per lane
     constexpr int SPLIT = D / 64;        // blocks per head
     constexpr int NRED = 2 * D + 2;      // per-token sums over columns: dq, dk, dlog_alpha, deta
-    __shared__ float red[2][WARPS][NRED];
+    extern __shared__ __align__(16) float smem_all[];
+    Stage<D> *const stage = reinterpret_cast<Stage<D> *>(smem_all);                    // two buffers
+    float *const red_all = smem_all + 2 * sizeof(Stage<D>) / sizeof(float);            // [RL][WARPS][NRED]: the warps' partial sums over their columns
+    auto red = [&](int slot, int w) { return red_all + ((size_t)slot * WARPS + w) * NRED; };
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int split = blockIdx.x % SPLIT, h = (blockIdx.x / SPLIT) % p.H, n = blockIdx.x / (SPLIT * p.H);
     int tok0, len;
@@ -67,24 +82,25 @@ __global__ void __launch_bounds__(NT, 1) kla_bwd_scan_kernel(BwdParams p)
     const int c0 = cg * WC;                      // first column of this warp
     const int myc = col_of_lane<WC>(lane);       // the column whose row sums this lane ends up with
     const size_t sbase = ((size_t)n * p.H + h) * D * D;
-    // Stored states use a layout of their own, [column group][j][half][lane] float4, so that every access is 512 contiguous bytes.
-    const size_t soff = ((size_t)cg * J * 2) * 128 + lane * 4;
+    // Stored states use a layout of their own, [column group][j][quad of columns][lane] float4, so that every access is 512 contiguous bytes.
+    const size_t soff = ((size_t)cg * J * (WC / 4)) * 128 + lane * 4;
     float *const stored = p.stored + ((size_t)(tok0 / L + n) * p.H + h) * D * D + soff;
     float *const scratch = p.scratch + ((size_t)n * p.H + h) * L * D * D + soff;
     auto put = [&](float *dst, const float (&S)[J][WC]) {
 #pragma unroll
-        for (int j = 0; j < J; ++j) {
-            store4(dst + (j * 2) * 128, make_float4(S[j][0], S[j][1], S[j][2], S[j][3]));
-            store4(dst + (j * 2 + 1) * 128, make_float4(S[j][4], S[j][5], S[j][6], S[j][7]));
-        }
+        for (int j = 0; j < J; ++j)
+#pragma unroll
+            for (int c = 0; c < WC; c += 4)
+                store4(dst + (j * (WC / 4) + c / 4) * 128, make_float4(S[j][c], S[j][c + 1], S[j][c + 2], S[j][c + 3]));
     };
     auto get = [&](const float *src, float (&S)[J][WC]) {
 #pragma unroll
-        for (int j = 0; j < J; ++j) {
-            const float4 a = load4(src + (j * 2) * 128), b = load4(src + (j * 2 + 1) * 128);
-            S[j][0] = a.x; S[j][1] = a.y; S[j][2] = a.z; S[j][3] = a.w;
-            S[j][4] = b.x; S[j][5] = b.y; S[j][6] = b.z; S[j][7] = b.w;
-        }
+        for (int j = 0; j < J; ++j)
+#pragma unroll
+            for (int c = 0; c < WC; c += 4) {
+                const float4 a = load4(src + (j * (WC / 4) + c / 4) * 128);
+                S[j][c] = a.x; S[j][c + 1] = a.y; S[j][c + 2] = a.z; S[j][c + 3] = a.w;
+            }
     };
     // the caller's states are [row][column]
     auto get_natural = [&](const float *src, float (&S)[J][WC]) {
@@ -101,28 +117,78 @@ __global__ void __launch_bounds__(NT, 1) kla_bwd_scan_kernel(BwdParams p)
     const IO *qp = reinterpret_cast<const IO *>(p.q), *kp = reinterpret_cast<const IO *>(p.k), *vp = reinterpret_cast<const IO *>(p.v);
     const IO *dop = reinterpret_cast<const IO *>(p.dout);
 
-    // ---- forward steps (no read-out): operands of the next token are requested while this one is applied ----
-    struct FRaw { IO k[J], v; float la, eta; };
-    auto frequest = [&](int i) {
-        FRaw r;
-        const size_t th = (size_t)(tok0 + max(min(i, len - 1), 0)) * p.H + h;
+    float S[J][WC], G[J][WC];
+    get_natural(p.init_state, S);
+    get_natural(p.dfinal, G);
+    const int n_blocks = (len + L - 1) / L;
+
+    // ---- operands of one block of L tokens, staged in shared memory as fp32 together with the per-token scalars ----
+    // Each warp fetches whole tokens (TPW of them): the raw values are requested into registers before the block in hand
+    // is processed and touched only after it (a use, even a conversion, would wait for them), then converted, reduced to
+    // alpha, beta (Eq. 3), ||k||^2 + eps and 1 / ||q||, and written to the buffer that is not being read.
+    constexpr int TPW = L / WARPS;
+    struct Pre { IO k[J], q[J]; IO v[2], dout[2]; float la, eta; };
+    Pre pre[TPW];
+    auto request_block = [&](int b, bool full) {
 #pragma unroll
-        for (int j = 0; j < J; ++j) r.k[j] = kp[th * D + lane + 32 * j];
-        r.v = vp[th * D + c0 + myc];
-        r.la = p.log_alpha[th];
-        r.eta = p.eta[th];
-        return r;
-    };
-    auto fstep = [&](float (&S)[J][WC], const FRaw &r) {
-        float k[J], nk = 0.f;
+        for (int u = 0; u < TPW; ++u) {
+            const int i = min(b * L + warp + u * WARPS, len - 1);
+            const size_t th = (size_t)(tok0 + i) * p.H + h;
 #pragma unroll
-        for (int j = 0; j < J; ++j) {
-            k[j] = to_f32(r.k[j]);
-            nk += k[j] * k[j];
+            for (int j = 0; j < J; ++j) {
+                pre[u].k[j] = kp[th * D + lane + 32 * j];
+                if (full) pre[u].q[j] = qp[th * D + lane + 32 * j];
+            }
+            const size_t col = th * D + split * 64 + 2 * lane;   // this block's 64 columns, two per lane
+            if constexpr (sizeof(IO) == 2) {
+                *reinterpret_cast<uint32_t *>(pre[u].v) = *reinterpret_cast<const uint32_t *>(vp + col);
+                if (full) *reinterpret_cast<uint32_t *>(pre[u].dout) = *reinterpret_cast<const uint32_t *>(dop + col);
+            } else {
+                *reinterpret_cast<float2 *>(pre[u].v) = *reinterpret_cast<const float2 *>(vp + col);
+                if (full) *reinterpret_cast<float2 *>(pre[u].dout) = *reinterpret_cast<const float2 *>(dop + col);
+            }
+            pre[u].la = p.log_alpha[th];
+            pre[u].eta = p.eta[th];
         }
-        const float alpha = __expf(r.la);
-        const float beta = p.coeff_eta ? r.eta : r.eta / (warp_sum(nk) + p.eps);   // Eq. 3
-        float part[WC];
+    };
+    auto commit_block = [&](Stage<D> &st, bool full) {
+#pragma unroll
+        for (int u = 0; u < TPW; ++u) {
+            const int tok = warp + u * WARPS;
+            float nk = 0.f, nq = 0.f, q[J];
+#pragma unroll
+            for (int j = 0; j < J; ++j) {
+                const float k = to_f32(pre[u].k[j]);
+                st.k[tok][lane + 32 * j] = k;
+                nk += k * k;
+                if (full) {
+                    q[j] = to_f32(pre[u].q[j]);
+                    nq += q[j] * q[j];
+                }
+            }
+            const float nrm = warp_sum(nk) + p.eps;
+            float qinv = 1.f;
+            if (QN && full) qinv = rsqrtf(warp_sum(nq));
+            store2(&st.v[tok][2 * lane], to_f32(pre[u].v[0]), to_f32(pre[u].v[1]));
+            if (full) {
+#pragma unroll
+                for (int j = 0; j < J; ++j) st.q[tok][lane + 32 * j] = q[j] * qinv;   // qh
+                store2(&st.dout[tok][2 * lane], to_f32(pre[u].dout[0]), to_f32(pre[u].dout[1]));
+            }
+            if (lane == 0) {
+                st.alpha[tok] = __expf(pre[u].la);
+                st.beta[tok] = p.coeff_eta ? pre[u].eta : pre[u].eta / nrm;   // Eq. 3
+                st.nrm[tok] = nrm;
+                st.qinv[tok] = qinv;
+            }
+        }
+    };
+    // one forward step without read-out
+    auto fstep = [&](const Stage<D> &st, int tok) {
+        float k[J], part[WC];
+#pragma unroll
+        for (int j = 0; j < J; ++j) k[j] = st.k[tok][lane + 32 * j];
+        const float alpha = st.alpha[tok], beta = st.beta[tok];
 #pragma unroll
         for (int c = 0; c < WC; ++c) {
             float s = 0.f;
@@ -130,7 +196,7 @@ __global__ void __launch_bounds__(NT, 1) kla_bwd_scan_kernel(BwdParams p)
             for (int j = 0; j < J; ++j) s += k[j] * S[j][c];
             part[c] = s;
         }
-        const float e_mine = to_f32(r.v) - alpha * reduce_scatter<WC>(part, lane);
+        const float e_mine = st.v[tok][warp * WC + myc] - alpha * reduce_scatter<WC>(part, lane);
 #pragma unroll
         for (int c = 0; c < WC; ++c) {
             const float be = beta * __shfl_sync(0xffffffffu, e_mine, lane_of_col<WC>(c));
@@ -139,179 +205,154 @@ __global__ void __launch_bounds__(NT, 1) kla_bwd_scan_kernel(BwdParams p)
         }
     };
 
-    float S[J][WC], G[J][WC];
-    get_natural(p.init_state, S);
-    get_natural(p.dfinal, G);
-    const int n_blocks = (len + L - 1) / L;
-    // forward sweep up to the start of the last block, keeping the state at the start of every block
-    if (n_blocks > 1) {
-        FRaw r = frequest(0);
-        for (int i = 0; i < (n_blocks - 1) * L; ++i) {
-            if (i % L == 0) put(stored + (size_t)(i / L) * p.H * D * D, S);
-            const FRaw rn = frequest(i + 1);
-            fstep(S, r);
-            r = rn;
+    if (n_blocks > 0) {
+        int cur = 0;
+        request_block(0, n_blocks == 1);
+        commit_block(stage[0], n_blocks == 1);
+        __syncthreads();
+        // forward sweep up to the start of the last block, keeping the state at the start of every block
+        for (int b = 0; b + 1 < n_blocks; ++b) {
+            const bool next_full = b + 2 == n_blocks;   // the last block is the first one the reverse sweep works on
+            request_block(b + 1, next_full);
+            put(stored + (size_t)b * p.H * D * D, S);
+            for (int tok = 0; tok < L; ++tok) fstep(stage[cur], tok);
+            commit_block(stage[cur ^ 1], next_full);
+            __syncthreads();   // one barrier per block: the buffer written is the one nobody reads
+            cur ^= 1;
         }
-    }
-
-    // ---- reverse sweep, block by block ----
-    struct BRaw { alignas(16) IO dout[WC]; IO q[J], k[J], v; float la, eta; };
-    auto brequest = [&](int i) {
-        BRaw r;
-        const size_t th = (size_t)(tok0 + max(i, 0)) * p.H + h;
-#pragma unroll
-        for (int j = 0; j < J; ++j) {
-            r.q[j] = qp[th * D + lane + 32 * j];
-            r.k[j] = kp[th * D + lane + 32 * j];
-        }
-        r.v = vp[th * D + c0 + myc];
-        r.la = p.log_alpha[th];
-        r.eta = p.eta[th];
-#pragma unroll
-        for (int c = 0; c < WC; c += 4) {   // the same WC values for every lane
-            if constexpr (sizeof(IO) == 2) {
-                const uint2 raw = *reinterpret_cast<const uint2 *>(dop + th * D + c0 + c);
-                *reinterpret_cast<uint2 *>(&r.dout[c]) = raw;
-            } else {
-                const float4 raw = *reinterpret_cast<const float4 *>(dop + th * D + c0 + c);
-                *reinterpret_cast<float4 *>(&r.dout[c]) = raw;
+        // ---- reverse sweep, block by block ----
+        for (int b = n_blocks - 1; b >= 0; --b) {
+            const int i0 = b * L, cnt = min(L, len - i0);
+            const Stage<D> &st = stage[cur];
+            if (b > 0) request_block(b - 1, true);
+            if (b != n_blocks - 1) get(stored + (size_t)b * p.H * D * D, S);
+            // the state before every token of the block (the last one stays in registers)
+            for (int tok = 0; tok + 1 < cnt; ++tok) {
+                put(scratch + (size_t)tok * D * D, S);
+                fstep(st, tok);
             }
-        }
-        return r;
-    };
-    for (int b = n_blocks - 1; b >= 0; --b) {
-        const int i0 = b * L, i1 = min(i0 + L, len);
-        if (b != n_blocks - 1) get(stored + (size_t)b * p.H * D * D, S);
-        {   // the state before every token of the block (the last one stays in registers)
-            FRaw r = frequest(i0);
-            for (int i = i0; i + 1 < i1; ++i) {
-                put(scratch + (size_t)(i - i0) * D * D, S);
-                const FRaw rn = frequest(i + 1);
-                fstep(S, r);
-                r = rn;
-            }
-        }
-        BRaw raw = brequest(i1 - 1);
-        for (int i = i1 - 1; i >= i0; --i) {
-            // S holds S_{i-1}; the state and the operands of the token before are requested now and used next iteration
-            float Sn[J][WC];
-            if (i > i0) get(scratch + (size_t)(i - 1 - i0) * D * D, Sn);
-            const BRaw rawn = brequest(i - 1);
-            const size_t th = (size_t)(tok0 + i) * p.H + h;
-            float q[J], k[J], dout[WC], nk = 0.f, nq = 0.f;
-#pragma unroll
-            for (int j = 0; j < J; ++j) {
-                q[j] = to_f32(raw.q[j]);
-                k[j] = to_f32(raw.k[j]);
-                nk += k[j] * k[j];
-                nq += q[j] * q[j];
-            }
-#pragma unroll
-            for (int c = 0; c < WC; ++c) dout[c] = to_f32(raw.dout[c]);
-            const float alpha = __expf(raw.la);
-            const float nrm = warp_sum(nk) + p.eps;
-            const float beta = p.coeff_eta ? raw.eta : raw.eta / nrm;   // Eq. 3
-            float qinv = 1.f;
-            if (QN) {
-                qinv = rsqrtf(warp_sum(nq));
-#pragma unroll
-                for (int j = 0; j < J; ++j) q[j] *= qinv;   // qh
-            }
-            // forward quantities of the token: S~ = alpha S_{i-1} (in place), e = v - S~^T k
-            float part[WC], e[WC], de[WC];
-#pragma unroll
-            for (int c = 0; c < WC; ++c) {
-                float s = 0.f;
+            for (int tok = cnt - 1; tok >= 0; --tok) {
+                // S holds the state before this token; the one before the previous token is requested now, used next iteration
+                float Sn[J][WC];
+                if (tok > 0) get(scratch + (size_t)(tok - 1) * D * D, Sn);
+                const size_t th = (size_t)(tok0 + i0 + tok) * p.H + h;
+                float q[J], k[J], dout[WC];
 #pragma unroll
                 for (int j = 0; j < J; ++j) {
-                    S[j][c] *= alpha;
-                    s += k[j] * S[j][c];
+                    q[j] = st.q[tok][lane + 32 * j];   // qh
+                    k[j] = st.k[tok][lane + 32 * j];
                 }
-                part[c] = s;
-            }
-            const float e_mine = to_f32(raw.v) - reduce_scatter<WC>(part, lane);
 #pragma unroll
-            for (int c = 0; c < WC; ++c) e[c] = __shfl_sync(0xffffffffu, e_mine, lane_of_col<WC>(c));
-            // read-out: dqh = S_t dO with S_t = S~ + beta k e^T formed on the fly; G += qh dO^T; then u = G^T k
-            float dq[J], dk[J];
-#pragma unroll
-            for (int j = 0; j < J; ++j) dq[j] = 0.f;
-#pragma unroll
-            for (int c = 0; c < WC; ++c) {
-                const float be = beta * e[c];
-                float s = 0.f;
-#pragma unroll
-                for (int j = 0; j < J; ++j) {
-                    dq[j] += (S[j][c] + k[j] * be) * dout[c];
-                    G[j][c] += q[j] * dout[c];
-                    s += G[j][c] * k[j];
+                for (int c = 0; c < WC; c += 4) {
+                    const float4 x = load4(&st.dout[tok][warp * WC + c]);
+                    dout[c] = x.x; dout[c + 1] = x.y; dout[c + 2] = x.z; dout[c + 3] = x.w;
                 }
-                part[c] = s;
-            }
-            const float u_mine = reduce_scatter<WC>(part, lane);
-            const float de_mine = beta * u_mine;                                      // de = beta G^T k  (= dv)
-            const float dbeta = warp_sum((lane & 3) == 0 ? u_mine * e_mine : 0.f);   // this warp's columns of k^T G e
-#pragma unroll
-            for (int c = 0; c < WC; ++c) de[c] = __shfl_sync(0xffffffffu, de_mine, lane_of_col<WC>(c));
-            // dk = beta G e - S~ de;  G <- alpha (G - k de^T);  dlog_alpha = <G - k de^T, S~>
-            float dla = 0.f;
-#pragma unroll
-            for (int j = 0; j < J; ++j) {
-                float ge = 0.f, sd = 0.f;
+                const float alpha = st.alpha[tok], beta = st.beta[tok], nrm = st.nrm[tok];
+                // forward quantities of the token: S~ = alpha S_{t-1} (in place), e = v - S~^T k
+                float part[WC], e[WC], de[WC];
 #pragma unroll
                 for (int c = 0; c < WC; ++c) {
-                    ge += G[j][c] * e[c];
-                    sd += S[j][c] * de[c];
-                    const float g = G[j][c] - k[j] * de[c];
-                    dla += g * S[j][c];
-                    G[j][c] = alpha * g;
+                    float s = 0.f;
+#pragma unroll
+                    for (int j = 0; j < J; ++j) {
+                        S[j][c] *= alpha;
+                        s += k[j] * S[j][c];
+                    }
+                    part[c] = s;
                 }
-                dk[j] = beta * ge - sd;
-            }
-            dla = warp_sum(dla);
-            float deta = dbeta;
-            if (!p.coeff_eta) {   // beta = eta / n: deta = dbeta / n, dn = -dbeta eta / n^2 = -dbeta beta / n, dk += 2 k dn
-                deta = dbeta / nrm;
-                const float dn2 = -2.f * dbeta * beta / nrm;
+                const float e_mine = st.v[tok][warp * WC + myc] - reduce_scatter<WC>(part, lane);
 #pragma unroll
-                for (int j = 0; j < J; ++j) dk[j] += k[j] * dn2;
-            }
-            if (QN) {   // o = S^T q / ||q||: dq = (dqh - qh (qh . dqh)) / ||q||, a linear map, applied to this warp's part
-                float pr = 0.f;
+                for (int c = 0; c < WC; ++c) e[c] = __shfl_sync(0xffffffffu, e_mine, lane_of_col<WC>(c));
+                // read-out: dqh = S_t dO with S_t = S~ + beta k e^T formed on the fly; G += qh dO^T; then u = G^T k
+                float dq[J], dk[J];
 #pragma unroll
-                for (int j = 0; j < J; ++j) pr += q[j] * dq[j];
-                pr = warp_sum(pr);
+                for (int j = 0; j < J; ++j) dq[j] = 0.f;
 #pragma unroll
-                for (int j = 0; j < J; ++j) dq[j] = (dq[j] - q[j] * pr) * qinv;
-            }
-            if ((lane & 3) == 0) p.dv[th * D + c0 + myc] = de_mine;
-            // sums over the block's columns
-            float *mine = red[i & 1][warp];
+                for (int c = 0; c < WC; ++c) {
+                    const float be = beta * e[c];
+                    float s = 0.f;
 #pragma unroll
-            for (int j = 0; j < J; ++j) {
-                mine[lane + 32 * j] = dq[j];
-                mine[D + lane + 32 * j] = dk[j];
-            }
-            if (lane == 0) {
-                mine[2 * D] = dla;
-                mine[2 * D + 1] = deta;
-            }
-            __syncthreads();   // one barrier per token: the buffers alternate, and nobody is two tokens ahead of anybody
-            for (int x = threadIdx.x; x < NRED; x += NT) {
-                float s = 0.f;
+                    for (int j = 0; j < J; ++j) {
+                        dq[j] += (S[j][c] + k[j] * be) * dout[c];
+                        G[j][c] += q[j] * dout[c];
+                        s += G[j][c] * k[j];
+                    }
+                    part[c] = s;
+                }
+                const float u_mine = reduce_scatter<WC>(part, lane);
+                const float de_mine = beta * u_mine;                                                   // de = beta G^T k  (= dv)
+                const float dbeta = warp_sum((lane & (32 / WC - 1)) == 0 ? u_mine * e_mine : 0.f);   // this warp's columns of k^T G e
 #pragma unroll
-                for (int w = 0; w < WARPS; ++w) s += red[i & 1][w][x];
-                float *dst = x < D ? p.dq + th * D + x : x < 2 * D ? p.dk + th * D + (x - D) : x == 2 * D ? p.dlog_alpha + th : p.deta + th;
-                if (SPLIT == 1) *dst = s;
-                else atomicAdd(dst, s);
-            }
-            if (i > i0) {
+                for (int c = 0; c < WC; ++c) de[c] = __shfl_sync(0xffffffffu, de_mine, lane_of_col<WC>(c));
+                // dk = beta G e - S~ de;  G <- alpha (G - k de^T);  dlog_alpha = <G - k de^T, S~>
+                float dla = 0.f;
 #pragma unroll
-                for (int j = 0; j < J; ++j)
+                for (int j = 0; j < J; ++j) {
+                    float ge = 0.f, sd = 0.f;
 #pragma unroll
-                    for (int c = 0; c < WC; ++c) S[j][c] = Sn[j][c];
+                    for (int c = 0; c < WC; ++c) {
+                        ge += G[j][c] * e[c];
+                        sd += S[j][c] * de[c];
+                        const float g = G[j][c] - k[j] * de[c];
+                        dla += g * S[j][c];
+                        G[j][c] = alpha * g;
+                    }
+                    dk[j] = beta * ge - sd;
+                }
+                dla = warp_sum(dla);
+                float deta = dbeta;
+                if (!p.coeff_eta) {   // beta = eta / n: deta = dbeta / n, dn = -dbeta eta / n^2 = -dbeta beta / n, dk += 2 k dn
+                    deta = dbeta / nrm;
+                    const float dn2 = -2.f * dbeta * beta / nrm;
+#pragma unroll
+                    for (int j = 0; j < J; ++j) dk[j] += k[j] * dn2;
+                }
+                if (QN) {   // o = S^T q / ||q||: dq = (dqh - qh (qh . dqh)) / ||q||, a linear map, applied to this warp's part
+                    float pr = 0.f;
+#pragma unroll
+                    for (int j = 0; j < J; ++j) pr += q[j] * dq[j];
+                    pr = warp_sum(pr);
+                    const float qinv = st.qinv[tok];
+#pragma unroll
+                    for (int j = 0; j < J; ++j) dq[j] = (dq[j] - q[j] * pr) * qinv;
+                }
+                if ((lane & (32 / WC - 1)) == 0) p.dv[th * D + c0 + myc] = de_mine;
+                // this warp's part of the sums over columns; added up every RL tokens
+                float *mine = red(tok % RL, warp);
+#pragma unroll
+                for (int j = 0; j < J; ++j) {
+                    mine[lane + 32 * j] = dq[j];
+                    mine[D + lane + 32 * j] = dk[j];
+                }
+                if (lane == 0) {
+                    mine[2 * D] = dla;
+                    mine[2 * D + 1] = deta;
+                }
+                if (tok > 0) {
+#pragma unroll
+                    for (int j = 0; j < J; ++j)
+#pragma unroll
+                        for (int c = 0; c < WC; ++c) S[j][c] = Sn[j][c];
+                }
+                if (tok % RL == 0) {   // add up the partial sums of tokens tok .. tok + RL - 1 (fewer at the end of the sequence)
+                    __syncthreads();
+                    const int n_sum = min(RL, cnt - tok);
+                    for (int idx = threadIdx.x; idx < n_sum * NRED; idx += NT) {
+                        const int slot = idx / NRED, x = idx - slot * NRED;
+                        float s = 0.f;
+#pragma unroll
+                        for (int w = 0; w < WARPS; ++w) s += red(slot, w)[x];
+                        const size_t tq = th + (size_t)slot * p.H;
+                        float *dst = x < D ? p.dq + tq * D + x : x < 2 * D ? p.dk + tq * D + (x - D) : x == 2 * D ? p.dlog_alpha + tq : p.deta + tq;
+                        if (SPLIT == 1) *dst = s;
+                        else atomicAdd(dst, s);
+                    }
+                    __syncthreads();
+                }
             }
-            raw = rawn;
+            if (b > 0) commit_block(stage[cur ^ 1], true);
+            __syncthreads();
+            cur ^= 1;
         }
     }
     if (p.dinit) {
@@ -328,10 +369,11 @@ cudaError_t launch_io(const BwdParams &p, int qnorm, cudaStream_t stream)
 {
     const int blocks = p.n_seq * p.H * (D / 64);
     if (blocks == 0) return cudaSuccess;
-    if (qnorm)
-        kla_bwd_scan_kernel<D, IO, true><<<blocks, NT, 0, stream>>>(p);
-    else
-        kla_bwd_scan_kernel<D, IO, false><<<blocks, NT, 0, stream>>>(p);
+    constexpr int smem = 2 * (int)sizeof(Stage<D>) + RL * WARPS * (2 * D + 2) * (int)sizeof(float);
+    auto kern = qnorm ? kla_bwd_scan_kernel<D, IO, true> : kla_bwd_scan_kernel<D, IO, false>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    kern<<<blocks, NT, smem, stream>>>(p);
     count_launch(1);
     return cudaGetLastError();
 }

@@ -315,6 +315,36 @@ def dg_leg(dev, steps, warmup, peaks):
             "achieved_gbs": nbytes / (ms * 1e-3) / 1e9, "roofline_frac": nbytes / (peaks["hbm_gbs"] * 1e9) / (ms * 1e-3), "bound": "hbm"}
 
 
+def bwd_leg(w, dev, steps, warmup, peaks, cpu_baseline):
+    """Backward pass (training, Section 5.1) on the headline shape: reverse sweep over recomputed states, fp32 on CUDA cores."""
+    import torch
+    from paper_2605_08587_b200 import binding, kla_bwd, workloads as W
+    do, df = W.upstream_grads(w)
+    t = [x.to(dev) for x in (w.q, w.k, w.v, w.log_alpha, w.eta)]
+    dod, dfd = do.to(dev), df.to(dev)
+    B, T, H, d = w.q.shape
+    desc = binding.KlaDesc(B=B, T=T, H=H, d_k=d, d_v=d, n_seq=B, io_dtype=binding.KLA_BF16, out_dtype=binding.KLA_F32)
+    import ctypes
+    ws = torch.empty(int(binding.load().kla_bwd_workspace_bytes(ctypes.byref(desc))), device=dev, dtype=torch.uint8)
+    stats = {}
+    ms = time_launches(lambda: kla_bwd(*t, w.eps, dod, d_final_state=dfd, workspace=ws), steps, warmup,
+                       torch.cuda.current_stream(), stats)
+    # q, k, v, d_out bf16 and the two gates read; dq, dk, dv and the two gate gradients written in fp32; dS_T read, dS_0 written
+    nbytes = B * T * H * (4 * d * 2 + 8 + 3 * d * 4 + 8) + 2 * B * H * d * d * 4
+    r = {"workload": w.name, "ms": ms, **stats, "mtok_per_s": B * T / (ms * 1e-3) / 1e6, "algorithmic_bytes": nbytes,
+         "workspace_bytes": ws.numel(), "achieved_gbs": nbytes / (ms * 1e-3) / 1e9,
+         "roofline_frac": nbytes / (peaks["hbm_gbs"] * 1e9) / (ms * 1e-3), "bound": "hbm"}
+    if cpu_baseline:
+        import oracle
+        a = [x.float().numpy() for x in (w.q, w.k, w.v)] + [w.log_alpha.numpy(), w.eta.numpy()]
+        t0 = time.perf_counter()
+        thr = oracle.backward(*a, w.eps, do.float().numpy(), None, df.numpy())["threads"]
+        dt = time.perf_counter() - t0
+        r["cpu_baseline"] = {"value": B * T / dt / 1e6, "unit": UNIT, "cores": thr, "kind": "oracle",
+                             "sample": "the whole backward of %s, one run, %.1f s" % (w.name, dt)}
+    return r
+
+
 def e2e_leg(w, dev, steps, warmup, groups=8):
     """Same step, host buffers: pinned host -> device copies of every input, the launches, and the
     device -> host read of out and final state, all inside the timed region.  The batch is cut into `groups`
@@ -455,6 +485,8 @@ def run_ours(args):
             extras["chunk_cfg2_wy_form"] = wy_leg(w, t, dev, 2, 1)
         elif args.also == "dg":
             extras["dg_fwd_layer_shape"] = dg_leg(dev, 2, 1, peaks)
+        elif args.also == "bwd":
+            extras["bwd_layer_shape"] = bwd_leg(W.config2(T=512), dev, 2, 1, peaks, False)
     if not args.quick:
         # decode: calls of 1024 consecutive steps on 1024 distinct token vectors, state carried in place
         extras["decode_cfg4"] = decode_leg(dev, 1024, 5, 1, peaks)
@@ -464,6 +496,7 @@ def run_ours(args):
         extras["chunk_cfg5_varlen"] = chunk_leg(W.config5(), dev, 20, 3, peaks, torch.bfloat16)
         extras["chunk_cfg2_wy_form"] = wy_leg(w, t, dev, 20, 3)
         extras["dg_fwd_layer_shape"] = dg_leg(dev, 10, 3, peaks)
+        extras["bwd_layer_shape"] = bwd_leg(w, dev, 10, 3, peaks, not args.no_cpu_baseline)
         if not args.no_cpu_baseline:
             extras["chunk_cfg3_long_context"]["cpu_baseline"] = oracle_chunk_workload(W.config3())
             extras["chunk_cfg5_varlen"]["cpu_baseline"] = oracle_chunk_workload(W.config5())
@@ -501,7 +534,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--quick", action="store_true", help="profiling mode: headline kernel only (no e2e, decode, long-context, varlen or CPU legs)")
-    ap.add_argument("--also", default="", choices=["", "decode", "decode64", "long", "varlen", "wy", "dg"],
+    ap.add_argument("--also", default="", choices=["", "decode", "decode64", "long", "varlen", "wy", "dg", "bwd"],
                     help="with --quick: run one more leg after the headline kernel (used for profiling)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -89,7 +89,16 @@ typedef enum { KLA_F32 = 0, KLA_BF16 = 1 } kla_dtype;
  * parallel, chained, and the segments then run in parallel from their true start states: the same result up
  * to rounding, about three times the state work, G times the parallelism.  By default the library decides
  * from the shape (few long sequences -> segments) and the workspace query returns what that decision needs. */
+/* When the decay is strong enough the segments need no transition maps at all: the map over a run of tokens has norm
+ * at most exp(sum of log_alpha) (every factor alpha (I - beta k k^T) has norm <= alpha when 0 <= eta <= 2, Eq. 3), so a
+ * segment run from the zero state, started so many chunks early that this bound is below exp(-40), reaches its first
+ * token with the exact state to fp32 accuracy.  A small kernel checks both conditions on the device (eta in [0, 2]
+ * everywhere; for every segment and head a warm-up of at most min(half a segment, 2048 tokens)); if they hold, one pass
+ * over the segments (plus their warm-up chunks) does the work, otherwise the transition-map passes do.  The decision is
+ * taken on the device, the call stays asynchronous; the workspace need is the same either way.  Not attempted with
+ * KLA_FLAG_COEFF_ETA (no bound on beta ||k||^2), KLA_FLAG_WY_FORM or KLA_FLAG_EXACT_SEGMENTS. */
 #define KLA_FLAG_NO_SEGMENTS 2            /* never cut sequences into segments                              */
+#define KLA_FLAG_EXACT_SEGMENTS 128       /* segments always from chained transition maps, never from warm-up runs */
 #define KLA_FLAG_SEGMENTS(g) ((g) << 8)   /* force g segments per sequence, 2 <= g <= 255 (fewer if T is short) */
 
 typedef struct {
@@ -116,12 +125,20 @@ typedef struct {
 
 /*
  * Scratch needed by kla_chunk_fwd for this descriptor (shape, dtypes, flags) and chunk length; 0 unless the
- * segment-parallel scan applies (then: per-segment transition maps and states, 3 x B x G x H x d_k x d_v fp32) or the
+ * segment-parallel scan applies (then: per-segment transition maps and states, 3 x B x G x H x d_k x d_v fp32, after a block of
+ * B G (H + 1) + 2 int32 padded to 256 bytes: segment bounds, plan word, warm-up lengths) or the
  * input is packed and goes to the tensor-core kernel (then: one int32 per sequence, for a longest-first order).
  * Computed on the host (it reads the current device's SM count when a device is present); returns 0 for an
  * invalid descriptor.  The same descriptor must be passed to kla_chunk_fwd with a workspace of at least this size.
  */
 size_t kla_chunk_fwd_workspace_bytes(const kla_desc *desc, int32_t chunk);
+
+/*
+ * Byte offset, inside the workspace of a call with this descriptor and chunk length, of an int32 that holds after the
+ * call 1 if the segments were started from decay-bounded warm-up runs and 0 if from chained transition maps (see
+ * KLA_FLAG_EXACT_SEGMENTS); (size_t)-1 when the call does not cut its sequences into segments.  Host function.
+ */
+size_t kla_chunk_fwd_plan_word_offset(const kla_desc *desc, int32_t chunk);
 
 /*
  * Chunkwise-parallel forward (Algorithm 1 right; Eqs. 7-9; Props. 3-4).

@@ -15,6 +15,7 @@ LIB_PATH = os.path.join(_HERE, "libkla_b200.so")
 KLA_F32, KLA_BF16 = 0, 1
 KLA_FLAG_NONE, KLA_FLAG_FORCE_SIMT, KLA_FLAG_NO_SEGMENTS = 0, 1, 2
 KLA_FLAG_COEFF_ETA, KLA_FLAG_QNORM, KLA_INTERNAL_FLAG_TEST_TIMEOUT, KLA_FLAG_NO_PAIR, KLA_FLAG_WY_FORM = 4, 8, 16, 32, 64
+KLA_FLAG_EXACT_SEGMENTS = 128
 
 
 def KLA_FLAG_SEGMENTS(g: int) -> int:
@@ -22,7 +23,7 @@ def KLA_FLAG_SEGMENTS(g: int) -> int:
     return int(g) << 8
 
 
-EXPORTS = ["kla_chunk_fwd_workspace_bytes", "kla_chunk_fwd", "kla_chunk_fwd_timed", "kla_chunk_fwd_static_scratch",
+EXPORTS = ["kla_chunk_fwd_workspace_bytes", "kla_chunk_fwd_plan_word_offset", "kla_chunk_fwd", "kla_chunk_fwd_timed", "kla_chunk_fwd_static_scratch",
            "kla_chunk_span_map_workspace_bytes", "kla_chunk_span_map", "kla_state_chain", "kla_dg_fwd", "kla_dg_decode_step", "kla_bwd_workspace_bytes", "kla_bwd", "kla_decode_step", "kla_decode_steps",
            "kla_status_str", "kla_launch_count"]
 
@@ -57,6 +58,8 @@ def load():
     vp, fp, dp = ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(KlaDesc)
     lib.kla_chunk_fwd_workspace_bytes.restype = ctypes.c_size_t
     lib.kla_chunk_fwd_workspace_bytes.argtypes = [dp, ctypes.c_int32]
+    lib.kla_chunk_fwd_plan_word_offset.restype = ctypes.c_size_t
+    lib.kla_chunk_fwd_plan_word_offset.argtypes = [dp, ctypes.c_int32]
     lib.kla_chunk_fwd.restype = ctypes.c_int
     lib.kla_chunk_fwd.argtypes = [dp, vp, vp, vp, fp, fp, ctypes.c_float, ctypes.c_int32, fp, vp, fp]
     lib.kla_chunk_fwd_timed.restype = ctypes.c_int
@@ -126,13 +129,15 @@ def _stream(dev):
 
 def kla_chunk_fwd(q, k, v, log_alpha, eta, eps, chunk=64, init_state=None, out=None, final_state=None,
                   cu_seqlens=None, host_seqlens=None, out_dtype=None, flags=KLA_FLAG_NONE,
-                  want_final_state=True, status_word=None, pass_ms=None):
+                  want_final_state=True, status_word=None, pass_ms=None, plan_word=None):
     """Chunkwise forward (include/kla.h: kla_chunk_fwd).
 
     q, k [B, T, H, d_k]; v [B, T, H, d_v]; log_alpha, eta [B, T, H] fp32; all CUDA, contiguous.
     Packed input: B = 1, cu_seqlens int32 CUDA [n_seq + 1] plus `host_seqlens` (CPU int32 copy;
     made from cu_seqlens with one D2H copy if omitted).
     Returns (out, final_state); buffers are allocated here unless passed in.
+    `plan_word`: a list; if given, the int32 of kla_chunk_fwd_plan_word_offset is read back after the call (which
+    waits for the device) and appended: 1 = segments started from warm-up runs, 0 = from chained maps, None = no segments.
     `pass_ms`: a list; if given the call goes through kla_chunk_fwd_timed (which waits for the stream) and the four
     per-pass device times in ms (set-up, segment pass 1, chaining, main pass) are appended to it.
     """
@@ -181,6 +186,9 @@ def kla_chunk_fwd(q, k, v, log_alpha, eta, eps, chunk=64, init_state=None, out=N
             code = lib.kla_chunk_fwd_timed(*args, ms)
             pass_ms.extend(float(x) for x in ms)
     _check(code)
+    if plan_word is not None:
+        off = lib.kla_chunk_fwd_plan_word_offset(ctypes.byref(desc), chunk)
+        plan_word.append(None if off == ctypes.c_size_t(-1).value or ws is None else int(ws[off:off + 4].view(torch.int32).item()))
     return out, final_state
 
 

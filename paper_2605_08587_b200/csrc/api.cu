@@ -121,7 +121,7 @@ static SegPlan plan_segments(const kla_desc *d, int32_t chunk)
     pl.seg_len = best_len * 64;
     pl.G = (d->T + pl.seg_len - 1) / pl.seg_len;
     if (pl.G < 2) return SegPlan();
-    const size_t cu_bytes = (((size_t)d->B * pl.G + 1) * sizeof(int32_t) + 255) & ~(size_t)255;
+    const size_t cu_bytes = (seg_plan_ints(d->B, pl.G, d->H) * sizeof(int32_t) + 255) & ~(size_t)255;
     const size_t st = (size_t)d->B * pl.G * d->H * d->d_k * d->d_v * sizeof(float);
     pl.off_map = cu_bytes;
     pl.off_local = cu_bytes + st;
@@ -143,6 +143,13 @@ size_t kla_chunk_fwd_workspace_bytes(const kla_desc *desc, int32_t chunk)
     // packed input on the tensor-core path, by the longest-first order of the sequences
     if (order_bytes(desc, chunk)) return order_bytes(desc, chunk);
     return plan_segments(desc, chunk).bytes;
+}
+
+size_t kla_chunk_fwd_plan_word_offset(const kla_desc *desc, int32_t chunk)
+{
+    if (check_common(desc) != KLA_OK) return (size_t)-1;
+    const SegPlan pl = plan_segments(desc, chunk);
+    return pl.G >= 2 ? ((size_t)desc->B * pl.G + 1) * sizeof(int32_t) : (size_t)-1;
 }
 
 }  // extern "C"
@@ -193,7 +200,14 @@ static kla_status chunk_fwd_impl(const kla_desc *desc, const void *q, const void
         char *ws = (char *)desc->workspace;
         int32_t *cu_seg = (int32_t *)ws;
         float *map = (float *)(ws + pl.off_map), *local = (float *)(ws + pl.off_local), *start = (float *)(ws + pl.off_start);
-        if (launch_seg_bounds(cu_seg, desc->B, desc->T, pl.G, pl.seg_len, stream) != cudaSuccess) return KLA_ERR_LAUNCH;
+        // Decay-bounded segment starts (seg_warm_plan_kernel): tried unless the caller forbids it, the coefficient is not
+        // Eq. 3's (beta = eta: no bound on beta ||k||^2) or the WY-form kernel is asked for (it has no such pass).  Both
+        // kinds of passes are enqueued; a device word decides which of them does the work, so nothing waits for the host.
+        const bool try_warm = !(desc->flags & (KLA_FLAG_EXACT_SEGMENTS | KLA_FLAG_COEFF_ETA)) &&
+                              !((desc->flags & KLA_FLAG_WY_FORM) && desc->d_k == 128);
+        if (launch_seg_bounds(cu_seg, desc->B, desc->T, pl.G, pl.seg_len, try_warm ? 1 : 0, stream) != cudaSuccess) return KLA_ERR_LAUNCH;
+        if (try_warm && launch_seg_warm_plan(cu_seg, log_alpha, eta, desc->B, desc->T, desc->H, pl.G, pl.seg_len, stream) != cudaSuccess)
+            return KLA_ERR_LAUNCH;
         mark(1);
         ChunkParams p1 = p;   // pass 1: transition map and zero-start state of every segment but the last
         p1.cu_seqlens = cu_seg; p1.n_seq = desc->B * pl.G;
@@ -201,7 +215,7 @@ static kla_status chunk_fwd_impl(const kla_desc *desc, const void *q, const void
         p1.seg_pass = 1; p1.seg_G = pl.G;
         if (launch_chunk_tc(p1, desc->d_k, desc->io_dtype, desc->out_dtype, stream) != cudaSuccess) return KLA_ERR_LAUNCH;
         mark(2);
-        if (launch_seg_combine(init_state, map, local, start, desc->B, desc->H, pl.G, desc->d_k, stream) != cudaSuccess)
+        if (launch_seg_combine(init_state, map, local, start, desc->B, desc->H, pl.G, desc->d_k, cu_seg + desc->B * pl.G + 1, stream) != cudaSuccess)
             return KLA_ERR_LAUNCH;
         mark(3);
         ChunkParams p3 = p;   // pass 3: every segment from its true start state
@@ -209,6 +223,12 @@ static kla_status chunk_fwd_impl(const kla_desc *desc, const void *q, const void
         p3.init_state = start;
         p3.seg_pass = 3; p3.seg_G = pl.G;
         err = launch_chunk_tc(p3, desc->d_k, desc->io_dtype, desc->out_dtype, stream);
+        if (err == cudaSuccess && try_warm) {
+            ChunkParams p4 = p;   // pass 4: every segment from a warm-up run (the sequence's first from its initial state)
+            p4.cu_seqlens = cu_seg; p4.n_seq = desc->B * pl.G;
+            p4.seg_pass = 4; p4.seg_G = pl.G;
+            err = launch_chunk_tc(p4, desc->d_k, desc->io_dtype, desc->out_dtype, stream);
+        }
         mark(4);
         return err == cudaSuccess ? KLA_OK : KLA_ERR_LAUNCH;
     }
@@ -276,7 +296,7 @@ size_t kla_chunk_span_map_workspace_bytes(const kla_desc *desc)
 {
     if (check_common(desc) != KLA_OK) return 0;
     // segment bounds of a two-segment cut whose second segment is empty, then both halves of the segment arrays
-    const size_t cu_bytes = (((size_t)desc->B * 2 + 1) * sizeof(int32_t) + 255) & ~(size_t)255;
+    const size_t cu_bytes = (seg_plan_ints(desc->B, 2, desc->H) * sizeof(int32_t) + 255) & ~(size_t)255;
     return cu_bytes + 2 * (size_t)desc->B * 2 * desc->H * desc->d_k * desc->d_v * sizeof(float);
 }
 
@@ -302,10 +322,10 @@ kla_status kla_chunk_span_map(const kla_desc *desc, const void *k, const void *v
     // kernel then gives the map and the zero-start state of exactly that span.
     char *ws = (char *)desc->workspace;
     int32_t *cu_seg = (int32_t *)ws;
-    const size_t cu_bytes = (((size_t)desc->B * 2 + 1) * sizeof(int32_t) + 255) & ~(size_t)255;
+    const size_t cu_bytes = (seg_plan_ints(desc->B, 2, desc->H) * sizeof(int32_t) + 255) & ~(size_t)255;
     const size_t half = (size_t)desc->B * 2 * desc->H * desc->d_k * desc->d_v;
     float *map = (float *)(ws + cu_bytes), *local = map + half;
-    if (launch_seg_bounds(cu_seg, desc->B, desc->T, 2, ((desc->T + 63) / 64) * 64, stream) != cudaSuccess) return KLA_ERR_LAUNCH;
+    if (launch_seg_bounds(cu_seg, desc->B, desc->T, 2, ((desc->T + 63) / 64) * 64, 0, stream) != cudaSuccess) return KLA_ERR_LAUNCH;
     ChunkParams p;
     p.q = k;   // never read out: pass 1 forms no outputs (the tensor map only needs a valid address)
     p.k = k; p.v = v;
@@ -340,7 +360,7 @@ kla_status kla_state_chain(const kla_desc *desc, int32_t n_spans, const float *i
     if (!aligned16(phi) || !aligned16(n) || !aligned16(start_out) || !aligned16(init_state)) return KLA_ERR_ALIGN;
     st = check_arch();
     if (st != KLA_OK) return st;
-    return launch_seg_combine(init_state, phi, n, start_out, desc->B, desc->H, n_spans, desc->d_k, (cudaStream_t)desc->stream) == cudaSuccess
+    return launch_seg_combine(init_state, phi, n, start_out, desc->B, desc->H, n_spans, desc->d_k, nullptr, (cudaStream_t)desc->stream) == cudaSuccess
                ? KLA_OK : KLA_ERR_LAUNCH;
 }
 

@@ -419,6 +419,9 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     if (p.seg_pass == 1) n = (n / (p.seg_G - 1)) * p.seg_G + n % (p.seg_G - 1);
     else if (p.seg_pass == 0 && p.seq_order) n = p.seq_order[n];   // packed input: longest sequences first
     const bool no_out = p.seg_pass == 1;
+    // Segment passes: the word after the segment bounds says whether the segments start from decay-bounded warm-up runs
+    // (pass 4 alone does the work) or from chained transition maps (passes 1 and 3 do); the other kind returns at once.
+    if (p.seg_pass != 0 && (p.seg_pass == 4) != (p.cu_seqlens[p.n_seq + 1] == 1)) return;
 
     int tok0, len;
     if (p.cu_seqlens) {
@@ -429,10 +432,24 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         len = p.T;
     }
     const size_t state_off = (((size_t)n * p.H + h) * D) * D + (size_t)sl * NS;
+    // the state before the first token (null: zero) and the number of leading chunks whose outputs are not stored
+    const float *init = p.init_state;
+    size_t init_off = state_off;
+    int first_out = 0;
+    if (p.seg_pass == 4) {
+        if (n % p.seg_G == 0) {   // first segment: the sequence's own initial state
+            init_off = (((size_t)(n / p.seg_G) * p.H + h) * D) * D + (size_t)sl * NS;
+        } else {                  // later segments: from zero, so many chunks before the segment (see seg_warm_plan_kernel)
+            init = nullptr;
+            first_out = p.cu_seqlens[p.n_seq + 2 + n * p.H + h];
+            tok0 -= first_out * C;
+            len += first_out * C;
+        }
+    }
     // where this CTA's final state goes (null: nowhere)
     float *fin = is_map ? p.map_state : p.final_state;
     size_t fin_off = state_off;
-    if (p.seg_pass == 3 && fin) {
+    if (p.seg_pass >= 3 && fin) {
         if (n % p.seg_G != p.seg_G - 1) fin = nullptr;
         else fin_off = (((size_t)(n / p.seg_G) * p.H + h) * D) * D + (size_t)sl * NS;
     }
@@ -993,10 +1010,10 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             // transition map: start from the identity (columns sl * NS + hf * 32 .. of I)
 #pragma unroll
             for (int c = 0; c < 32; ++c) S[c] = (srow == sl * NS + hf * 32 + c) ? 1.f : 0.f;
-        } else if (s_act && p.init_state) {
+        } else if (s_act && init) {
 #pragma unroll
             for (int c = 0; c < 32; c += 4) {
-                const float4 x = *reinterpret_cast<const float4 *>(p.init_state + state_off + (size_t)srow * D + hf * 32 + c);
+                const float4 x = *reinterpret_cast<const float4 *>(init + init_off + (size_t)srow * D + hf * 32 + c);
                 S[c] = x.x; S[c + 1] = x.y; S[c + 2] = x.z; S[c + 3] = x.w;
             }
         } else {
@@ -1111,6 +1128,7 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             if (no_out) continue;
             if (!wait(B_D4_DONE, ph)) break;
             tc_fence_after();
+            const int rows_out = c < first_out ? 0 : rows;   // warm-up chunks are computed like any other and not stored
             {
                 // This thread's accumulator values are column pairs cp + 8j (j = 0..3) of rows i0 and i1; a 4 x 4 transpose
                 // over the four lanes of a quad gives each lane 8 consecutive columns of both rows, so that every
@@ -1141,8 +1159,8 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     }
                     quad_transpose(a, t4);
                     quad_transpose(b, t4);
-                    if (i0 < rows) *reinterpret_cast<uint4 *>(o0) = make_uint4(a[0], a[1], a[2], a[3]);
-                    if (i1 < rows) *reinterpret_cast<uint4 *>(o1) = make_uint4(b[0], b[1], b[2], b[3]);
+                    if (i0 < rows_out) *reinterpret_cast<uint4 *>(o0) = make_uint4(a[0], a[1], a[2], a[3]);
+                    if (i1 < rows_out) *reinterpret_cast<uint4 *>(o1) = make_uint4(b[0], b[1], b[2], b[3]);
                 } else {
                     uint32_t ax[4], ay[4], bx[4], by[4];
 #pragma unroll
@@ -1156,11 +1174,11 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     quad_transpose(ay, t4);
                     quad_transpose(bx, t4);
                     quad_transpose(by, t4);
-                    if (i0 < rows) {
+                    if (i0 < rows_out) {
                         *reinterpret_cast<uint4 *>(o0) = make_uint4(ax[0], ay[0], ax[1], ay[1]);
                         *reinterpret_cast<uint4 *>(o0 + 4) = make_uint4(ax[2], ay[2], ax[3], ay[3]);
                     }
-                    if (i1 < rows) {
+                    if (i1 < rows_out) {
                         *reinterpret_cast<uint4 *>(o1) = make_uint4(bx[0], by[0], bx[1], by[1]);
                         *reinterpret_cast<uint4 *>(o1 + 4) = make_uint4(bx[2], by[2], bx[3], by[3]);
                     }

@@ -25,6 +25,9 @@ struct ChunkParams {
     //               started at the identity, v = 0) and write it to map_state.
     //   seg_pass 3: every segment from its true start state; only the last segment of a sequence writes
     //               final_state, at the sequence's index.
+    //   seg_pass 4: every segment but a sequence's first from the zero state, started as many chunks early as the plan
+    //               after the segment bounds says (outputs of those chunks are not stored); init_state is per sequence.
+    //   Passes 1 and 3 return at once when the plan word (cu_seqlens[n_seq + 1]) is 1, pass 4 when it is not.
     int32_t seg_pass, seg_G;
     int32_t variant;     // bit 0: beta_t = eta_t instead of Eq. 3; bit 1: read-out divided by ||q_t||; bit 2: test hook; bits 3, 4: see VARIANT_NO_PAIR, VARIANT_WY
     union {
@@ -60,12 +63,19 @@ cudaError_t launch_chunk_tc(const ChunkParams &p, int d, int io_dtype, int out_d
 // Head dimension 128, the two slices of a head as a cluster of two CTAs (chunk_wy.cu); called by launch_chunk_tc.
 cudaError_t launch_chunk_wy(const ChunkParams &p, int out_dtype, cudaStream_t stream);
 // Segment-parallel helpers (segscan.cu).  cu_seg[b * G + g] = b * T + min(g * seg_len, T), one more entry = B * T.
-cudaError_t launch_seg_bounds(int32_t *cu_seg, int B, int T, int G, int seg_len, cudaStream_t stream);
+// After the bounds come the plan word (cu_seg[B G + 1]; `try_warm` is its initial value) and, from cu_seg[B G + 2] on, one
+// warm-up length in chunks per (segment, head): seg_plan_ints(B, G, H) int32 in all.
+cudaError_t launch_seg_bounds(int32_t *cu_seg, int B, int T, int G, int seg_len, int try_warm, cudaStream_t stream);
+inline size_t seg_plan_ints(int B, int G, int H) { return (size_t)B * G + 2 + (size_t)B * G * H; }
+// Decides whether the segments may start from decay-bounded warm-up runs and how long each must be (clears the plan word if not).
+cudaError_t launch_seg_warm_plan(int32_t *cu_seg, const float *log_alpha, const float *eta, int B, int T, int H, int G,
+                                 int seg_len, cudaStream_t stream);
 // order[r] = index of the sequence with the r-th largest length (ties by index); n_seq small (quadratic work)
 cudaError_t launch_seq_order(const int32_t *cu_seqlens, int n_seq, int32_t *order, cudaStream_t stream);
 // start[b, 0] = init (or 0); start[b, g + 1] = map[b, g] . start[b, g] + local[b, g]   (d x d products, fp32)
+// (`skip_if_one`: null, or a device word; the kernel does nothing when it holds 1)
 cudaError_t launch_seg_combine(const float *init_state, const float *map, const float *local, float *start, int B, int H,
-                               int G, int d, cudaStream_t stream);
+                               int G, int d, const int32_t *skip_if_one, cudaStream_t stream);
 // Diagonal-gated recurrence, token by token on CUDA cores (dg_scan.cu); log_alpha [n_tok, H, d].
 cudaError_t launch_dg_scan(const void *q, const void *k, const void *v, const float *log_alpha, const float *eta,
                            const float *init_state, void *out, float *final_state, const int32_t *cu_seqlens, int T, int H,

@@ -12,16 +12,70 @@ namespace kla {
 
 namespace {
 
-__global__ void seg_bounds_kernel(int32_t *cu_seg, int B, int T, int G, int seg_len)
+// Segment bounds, and after them the plan word (cu_seg[B G + 1]): 1 = the segments are to start from decay-bounded warm-up
+// runs unless seg_warm_plan_kernel finds a reason against it, 0 = from chained transition maps.
+__global__ void seg_bounds_kernel(int32_t *cu_seg, int B, int T, int G, int seg_len, int try_warm)
 {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i > B * G) return;
+    if (i > B * G + 1) return;
+    if (i == B * G + 1) {
+        cu_seg[i] = try_warm;
+        return;
+    }
     if (i == B * G) {
         cu_seg[i] = B * T;
         return;
     }
     const int b = i / G, g = i % G;
     cu_seg[i] = b * T + min(g * seg_len, T);
+}
+
+// Decay-bounded segment starts.  The state map over a run of tokens is Phi = prod_t alpha_t (I - beta_t k_t k_t^T); every
+// factor is symmetric with eigenvalues alpha_t and alpha_t (1 - beta_t ||k_t||^2), and beta_t ||k_t||^2 = eta_t ||k_t||^2 /
+// (||k_t||^2 + eps) lies in [0, eta_t] (Eq. 3), so for 0 <= eta_t <= 2 the factor's norm is at most alpha_t and
+// ||Phi||_2 <= exp(sum_t log alpha_t).  A segment that is run from the ZERO state starting w chunks early therefore reaches
+// its first token with an error of at most exp(sum of log alpha over those w chunks) x ||S||: with the sum below -40
+// (4e-18) that is nothing in fp32, and the segment needs neither its predecessors' transition maps nor a second pass.
+// One warp per (segment, head): warm[(n H + h)] = the smallest such w, at most max_warm chunks; if there is none, or if
+// any eta is outside [0, 2] (blocks past the planning warps check eta), the plan word is cleared and the transition-map
+// passes run instead.
+constexpr float WARM_LOG_DECAY = -40.f;
+__global__ void seg_warm_plan_kernel(int32_t *cu_seg, const float *log_alpha, const float *eta, int n_seg, int G, int H,
+                                     int max_warm, int plan_blocks, long long n_gate)
+{
+    int32_t *plan = cu_seg + n_seg + 1, *warm = cu_seg + n_seg + 2;
+    if ((int)blockIdx.x >= plan_blocks) {   // eta in [0, 2] everywhere (a NaN fails the test)
+        bool bad = false;
+        for (long long i = (long long)(blockIdx.x - plan_blocks) * blockDim.x + threadIdx.x; i < n_gate;
+             i += (long long)(gridDim.x - plan_blocks) * blockDim.x) {
+            const float e = eta[i];
+            bad |= !(e >= 0.f && e <= 2.f);
+        }
+        if (bad) *plan = 0;
+        return;
+    }
+    const int unit = blockIdx.x * (blockDim.x / 32) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (unit >= n_seg * H) return;
+    const int n = unit / H, h = unit % H;
+    if (n % G == 0) {
+        if (lane == 0) warm[unit] = 0;
+        return;
+    }
+    const int start = cu_seg[n];   // first token of the segment (a multiple of 64 tokens into its sequence)
+    float acc = 0.f;
+    int w = 0;
+    while (w < max_warm && acc > WARM_LOG_DECAY) {
+        ++w;
+        const size_t t = (size_t)(start - w * 64 + 2 * lane);
+        float x = log_alpha[t * H + h] + log_alpha[(t + 1) * H + h];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+        acc += x;
+    }
+    if (lane == 0) {
+        warm[unit] = w;
+        if (!(acc <= WARM_LOG_DECAY)) *plan = 0;   // (also when a gate is NaN)
+    }
 }
 
 // Rank of every sequence by decreasing length (ties by index): order[rank] = sequence.
@@ -41,8 +95,9 @@ __global__ void seq_order_kernel(const int32_t *cu_seqlens, int n_seq, int32_t *
 // One CTA per (sequence, head, 16-column slice of the state); thread r owns row r of the slice.
 template <int D>
 __global__ void __launch_bounds__(D) seg_combine_kernel(const float *init_state, const float *map, const float *local,
-                                                        float *start, int H, int G)
+                                                        float *start, int H, int G, const int32_t *skip_if_one)
 {
+    if (skip_if_one && *skip_if_one == 1) return;   // the segments start from warm-up runs: no maps to chain
     constexpr int W = 16;
     const int sl = blockIdx.x % (D / W);
     const int h = (blockIdx.x / (D / W)) % H;
@@ -99,10 +154,22 @@ __global__ void __launch_bounds__(D) seg_combine_kernel(const float *init_state,
 
 }  // namespace
 
-cudaError_t launch_seg_bounds(int32_t *cu_seg, int B, int T, int G, int seg_len, cudaStream_t stream)
+cudaError_t launch_seg_bounds(int32_t *cu_seg, int B, int T, int G, int seg_len, int try_warm, cudaStream_t stream)
 {
-    const int n = B * G + 1;
-    seg_bounds_kernel<<<(n + 127) / 128, 128, 0, stream>>>(cu_seg, B, T, G, seg_len);
+    const int n = B * G + 2;
+    seg_bounds_kernel<<<(n + 127) / 128, 128, 0, stream>>>(cu_seg, B, T, G, seg_len, try_warm);
+    count_launch(1);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_seg_warm_plan(int32_t *cu_seg, const float *log_alpha, const float *eta, int B, int T, int H, int G,
+                                 int seg_len, cudaStream_t stream)
+{
+    const int n_seg = B * G, plan_blocks = (n_seg * H + 3) / 4;   // four planning warps per block
+    const long long n_gate = (long long)B * T * H;
+    const int eta_blocks = (int)((n_gate + 128 * 16 - 1) / (128 * 16) < 256 ? (n_gate + 128 * 16 - 1) / (128 * 16) : 256);
+    const int max_warm = seg_len / 64 / 2 < 32 ? seg_len / 64 / 2 : 32;   // at most half a segment, and 2048 tokens
+    seg_warm_plan_kernel<<<plan_blocks + eta_blocks, 128, 0, stream>>>(cu_seg, log_alpha, eta, n_seg, G, H, max_warm, plan_blocks, n_gate);
     count_launch(1);
     return cudaGetLastError();
 }
@@ -115,12 +182,12 @@ cudaError_t launch_seq_order(const int32_t *cu_seqlens, int n_seq, int32_t *orde
 }
 
 cudaError_t launch_seg_combine(const float *init_state, const float *map, const float *local, float *start, int B, int H,
-                               int G, int d, cudaStream_t stream)
+                               int G, int d, const int32_t *skip_if_one, cudaStream_t stream)
 {
     if (d == 128)
-        seg_combine_kernel<128><<<B * H * (128 / 16), 128, 0, stream>>>(init_state, map, local, start, H, G);
+        seg_combine_kernel<128><<<B * H * (128 / 16), 128, 0, stream>>>(init_state, map, local, start, H, G, skip_if_one);
     else
-        seg_combine_kernel<64><<<B * H * (64 / 16), 64, 0, stream>>>(init_state, map, local, start, H, G);
+        seg_combine_kernel<64><<<B * H * (64 / 16), 64, 0, stream>>>(init_state, map, local, start, H, G, skip_if_one);
     count_launch(1);
     return cudaGetLastError();
 }

@@ -64,7 +64,7 @@ def oracle_chunk(w, heads=None, seqs=None):
     return out, fin, idx
 
 
-def gpu_chunk(w, out_dtype=torch.float32, flags=0, chunk=None, want_final_state=True):
+def gpu_chunk(w, out_dtype=torch.float32, flags=0, chunk=None, want_final_state=True, plan_word=None):
     from paper_2605_08587_b200 import kla_chunk_fwd
     dev = "cuda:0"
     cu = None if w.cu_seqlens is None else w.cu_seqlens.to(dev)
@@ -72,6 +72,6 @@ def gpu_chunk(w, out_dtype=torch.float32, flags=0, chunk=None, want_final_state=
                              chunk=chunk or w.chunk,
                              init_state=None if w.init_state is None else w.init_state.to(dev),
                              cu_seqlens=cu, host_seqlens=w.cu_seqlens, out_dtype=out_dtype, flags=flags,
-                             want_final_state=want_final_state)
+                             want_final_state=want_final_state, plan_word=plan_word)
     torch.cuda.synchronize()
     return out, fin

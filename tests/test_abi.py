@@ -124,12 +124,13 @@ def test_workspace_grows_only_when_sequences_are_cut_into_segments(lib):
     need = lib.kla_chunk_fwd_workspace_bytes(ctypes.byref(long1), 64)
     assert need > 0
     state = 8 * 128 * 128 * 4
-    G = (need - 256) // (3 * state)
-    assert 2 <= G <= 32 and need == 256 + 3 * G * state        # cu_seg (padded) + map, local, start per segment
+    plan = lambda B, G, H: ((B * G + 2 + B * G * H) * 4 + 255) // 256 * 256   # bounds, plan word, warm-up length per (segment, head)
+    G = need // (3 * state)
+    assert 2 <= G <= 32 and need == plan(1, G, 8) + 3 * G * state   # plan block (padded) + map, local, start per segment
     off = _desc(B=1, T=65536, H=8, d_k=128, d_v=128, n_seq=1, flags=2)
     assert lib.kla_chunk_fwd_workspace_bytes(ctypes.byref(off), 64) == 0
     forced = _desc(B=8, T=4096, H=8, d_k=128, d_v=128, n_seq=8, flags=4 << 8)
-    assert lib.kla_chunk_fwd_workspace_bytes(ctypes.byref(forced), 64) == 256 + 3 * 8 * 4 * state
+    assert lib.kla_chunk_fwd_workspace_bytes(ctypes.byref(forced), 64) == plan(8, 4, 8) + 3 * 8 * 4 * state
     assert lib.kla_chunk_fwd(ctypes.byref(forced), FAKE, FAKE, FAKE, FAKE, FAKE, 1e-6, 64, None, FAKE, None) == -7
     # fp32 inputs and chunk 32 go to the CUDA-core kernel: never segmented
     f32 = _desc(B=1, T=65536, H=8, d_k=128, d_v=128, n_seq=1, io_dtype=binding.KLA_F32)

@@ -123,6 +123,31 @@ def _dev(t, name, dtype=None):
     return t.data_ptr()
 
 
+_own_status = {}   # device index -> int32[1] the binding passes as status word when the caller gives none
+
+
+def _status_for(dev):
+    i = torch.device(dev).index
+    i = torch.cuda.current_device() if i is None else i
+    if i not in _own_status:
+        _own_status[i] = torch.zeros(1, dtype=torch.int32, device="cuda:%d" % i)
+    return _own_status[i]
+
+
+def check(device=None):
+    """Reads (and clears) the status word the binding passes to kla_chunk_fwd when the caller gives none: raises KlaError
+    if a kernel on `device` (default: the current one) gave up on a bounded wait since the last check -- its outputs are
+    then undefined.  Waits for the device; meant for the end of a step, not for the hot path."""
+    i = torch.cuda.current_device() if device is None else torch.device(device).index
+    word = _own_status.get(i)
+    if word is None:
+        return
+    code = int(word.item())
+    if code != 0:
+        word.zero_()
+        raise KlaError(code, status_str(code))
+
+
 def _stream(dev):
     return torch.cuda.current_stream(dev).cuda_stream
 
@@ -136,6 +161,8 @@ def kla_chunk_fwd(q, k, v, log_alpha, eta, eps, chunk=64, init_state=None, out=N
     Packed input: B = 1, cu_seqlens int32 CUDA [n_seq + 1] plus `host_seqlens` (CPU int32 copy;
     made from cu_seqlens with one D2H copy if omitted).
     Returns (out, final_state); buffers are allocated here unless passed in.
+    `status_word`: CUDA int32[1], zeroed by the caller, that receives KLA_ERR_TIMEOUT if a bounded device-side wait runs
+    out; if None the binding passes one of its own per device, read and cleared by `check()`.
     `plan_word`: a list; if given, the int32 of kla_chunk_fwd_plan_word_offset is read back after the call (which
     waits for the device) and appended: 1 = segments started from warm-up runs, 0 = from chained maps, None = no segments.
     `pass_ms`: a list; if given the call goes through kla_chunk_fwd_timed (which waits for the stream) and the four
@@ -165,6 +192,8 @@ def kla_chunk_fwd(q, k, v, log_alpha, eta, eps, chunk=64, init_state=None, out=N
         final_state = torch.empty((n_seq, H, d_k, d_v), device=q.device, dtype=torch.float32)
     if init_state is not None and tuple(init_state.shape) != (n_seq, H, d_k, d_v):
         raise ValueError("init_state must be [n_seq, H, d_k, d_v]")
+    if status_word is None:   # a timeout must not pass unnoticed: see check()
+        status_word = _status_for(q.device)
     desc = KlaDesc(B=B, T=T, H=H, d_k=d_k, d_v=d_v, n_seq=n_seq,
                    cu_seqlens=_dev(cu_seqlens, "cu_seqlens"), host_seqlens=hs.data_ptr() if hs is not None else None,
                    io_dtype=_dt(q), out_dtype=_dt(out), flags=flags, workspace=None, workspace_bytes=0,

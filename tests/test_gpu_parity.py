@@ -367,6 +367,24 @@ def test_bounded_wait_reports_timeout_and_context_stays_usable(no_pair):
     assert rel_err(np64(out), ro) <= TOL_BF16 and rel_err(np64(fin), rf) <= TOL_BF16
 
 
+def test_timeout_without_a_caller_status_word_is_raised_by_check():
+    """The binding passes a status word of its own when the caller gives none; check() reads and clears it."""
+    from paper_2605_08587_b200 import KlaError, binding, check, kla_chunk_fwd
+    w = W.config2(B=1, H=2, T=200, seed=502)
+    a = [t.to("cuda:0") for t in (w.q, w.k, w.v, w.log_alpha, w.eta)]
+    kla_chunk_fwd(*a, w.eps)
+    check("cuda:0")                               # nothing to report after an ordinary call
+    kla_chunk_fwd(*a, w.eps, flags=binding.KLA_INTERNAL_FLAG_TEST_TIMEOUT)
+    with pytest.raises(KlaError) as e:
+        check("cuda:0")
+    assert e.value.code == -10                    # KLA_ERR_TIMEOUT
+    check("cuda:0")                               # cleared
+    out, fin = kla_chunk_fwd(*a, w.eps, out_dtype=torch.float32)
+    check("cuda:0")
+    ro, rf = oracle_chunk(w)
+    assert rel_err(np64(out), ro) <= TOL_BF16 and rel_err(np64(fin), rf) <= TOL_BF16
+
+
 # ---- d_v = 128: the two slices of a head as a cluster that shares the solve (default) or as independent CTAs ----------
 from paper_2605_08587_b200 import KLA_FLAG_NO_PAIR  # noqa: E402
 

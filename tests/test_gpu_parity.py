@@ -259,6 +259,11 @@ def test_config3_full_size_every_head(out_dtype):
     _check_full("cfg3", out_dtype)
 
 
+def test_config3_full_size_from_chained_transition_maps():
+    from paper_2605_08587_b200 import binding
+    _check_full("cfg3", torch.float32, flags=binding.KLA_FLAG_EXACT_SEGMENTS)
+
+
 @pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16])
 def test_config5_full_size_every_sequence_and_head(out_dtype):
     out, fin, r = _check_full("cfg5", out_dtype)
@@ -272,14 +277,15 @@ def test_config5_full_size_every_sequence_and_head(out_dtype):
 
 
 # ---- segment-parallel scan (long sequences cut into segments; same result up to rounding) ------------------
-from paper_2605_08587_b200 import KLA_FLAG_NO_SEGMENTS, KLA_FLAG_SEGMENTS  # noqa: E402
+from paper_2605_08587_b200 import KLA_FLAG_EXACT_SEGMENTS, KLA_FLAG_NO_SEGMENTS, KLA_FLAG_SEGMENTS  # noqa: E402
 
 
+@pytest.mark.parametrize("exact", [KLA_FLAG_EXACT_SEGMENTS, 0])   # chained transition maps always / warm-up runs where they apply
 @pytest.mark.parametrize("G", [2, 3, 7])
 @pytest.mark.parametrize("d", [64, 128])
-def test_forced_segments_match_oracle(G, d):
+def test_forced_segments_match_oracle(G, d, exact):
     w = W.config3(B=2, H=2, T=1536 + 17, d=d, seed=200 + G)
-    _check_fixed(w, TOL_BF16, flags=KLA_FLAG_SEGMENTS(G))
+    _check_fixed(w, TOL_BF16, flags=KLA_FLAG_SEGMENTS(G) | exact)
 
 
 def test_segments_equal_plain_launch_closely():

@@ -185,23 +185,31 @@ __global__ void __launch_bounds__(NT, 1) kla_bwd_scan_kernel(BwdParams p)
     };
     // one forward step without read-out
     auto fstep = [&](const Stage<D> &st, int tok) {
-        float k[J], part[WC];
+        float2 k[J];   // (k_j, k_j)
+        float part[WC];
 #pragma unroll
-        for (int j = 0; j < J; ++j) k[j] = st.k[tok][lane + 32 * j];
+        for (int j = 0; j < J; ++j) k[j] = f2(st.k[tok][lane + 32 * j]);
         const float alpha = st.alpha[tok], beta = st.beta[tok];
 #pragma unroll
-        for (int c = 0; c < WC; ++c) {
-            float s = 0.f;
+        for (int c = 0; c < WC; c += 2) {
+            float2 s = f2(0.f);
 #pragma unroll
-            for (int j = 0; j < J; ++j) s += k[j] * S[j][c];
-            part[c] = s;
+            for (int j = 0; j < J; ++j) s = fma2(k[j], f2(S[j][c], S[j][c + 1]), s);
+            part[c] = s.x;
+            part[c + 1] = s.y;
         }
         const float e_mine = st.v[tok][warp * WC + myc] - alpha * reduce_scatter<WC>(part, lane);
+        const float2 a2 = f2(alpha);
 #pragma unroll
-        for (int c = 0; c < WC; ++c) {
-            const float be = beta * __shfl_sync(0xffffffffu, e_mine, lane_of_col<WC>(c));
+        for (int c = 0; c < WC; c += 2) {
+            const float2 be = f2(beta * __shfl_sync(0xffffffffu, e_mine, lane_of_col<WC>(c)),
+                                 beta * __shfl_sync(0xffffffffu, e_mine, lane_of_col<WC>(c + 1)));
 #pragma unroll
-            for (int j = 0; j < J; ++j) S[j][c] = alpha * S[j][c] + k[j] * be;
+            for (int j = 0; j < J; ++j) {
+                const float2 r = fma2(a2, f2(S[j][c], S[j][c + 1]), mul2(k[j], be));
+                S[j][c] = r.x;
+                S[j][c + 1] = r.y;
+            }
         }
     };
 
@@ -250,55 +258,80 @@ __global__ void __launch_bounds__(NT, 1) kla_bwd_scan_kernel(BwdParams p)
                 const float alpha = st.alpha[tok], beta = st.beta[tok], nrm = st.nrm[tok];
                 // forward quantities of the token: S~ = alpha S_{t-1} (in place), e = v - S~^T k
                 float part[WC], e[WC], de[WC];
+                float2 k2[J], q2[J];
 #pragma unroll
-                for (int c = 0; c < WC; ++c) {
-                    float s = 0.f;
+                for (int j = 0; j < J; ++j) {
+                    k2[j] = f2(k[j]);
+                    q2[j] = f2(q[j]);
+                }
+                const float2 a2 = f2(alpha);
+#pragma unroll
+                for (int c = 0; c < WC; c += 2) {
+                    float2 s = f2(0.f);
 #pragma unroll
                     for (int j = 0; j < J; ++j) {
-                        S[j][c] *= alpha;
-                        s += k[j] * S[j][c];
+                        const float2 st2 = mul2(a2, f2(S[j][c], S[j][c + 1]));
+                        S[j][c] = st2.x;
+                        S[j][c + 1] = st2.y;
+                        s = fma2(k2[j], st2, s);
                     }
-                    part[c] = s;
+                    part[c] = s.x;
+                    part[c + 1] = s.y;
                 }
                 const float e_mine = st.v[tok][warp * WC + myc] - reduce_scatter<WC>(part, lane);
 #pragma unroll
                 for (int c = 0; c < WC; ++c) e[c] = __shfl_sync(0xffffffffu, e_mine, lane_of_col<WC>(c));
-                // read-out: dqh = S_t dO with S_t = S~ + beta k e^T formed on the fly; G += qh dO^T; then u = G^T k
+                // read-out: dqh = S_t dO = S~ dO + k (beta e . dO); G += qh dO^T; then u = G^T k
                 float dq[J], dk[J];
+                float2 dq2[J];
+                float bed = 0.f;   // beta e . dO over this warp's columns
 #pragma unroll
-                for (int j = 0; j < J; ++j) dq[j] = 0.f;
+                for (int c = 0; c < WC; ++c) bed += e[c] * dout[c];
+                bed *= beta;
 #pragma unroll
-                for (int c = 0; c < WC; ++c) {
-                    const float be = beta * e[c];
-                    float s = 0.f;
+                for (int j = 0; j < J; ++j) dq2[j] = f2(0.f);
+#pragma unroll
+                for (int c = 0; c < WC; c += 2) {
+                    const float2 do2 = f2(dout[c], dout[c + 1]);
+                    float2 s = f2(0.f);
 #pragma unroll
                     for (int j = 0; j < J; ++j) {
-                        dq[j] += (S[j][c] + k[j] * be) * dout[c];
-                        G[j][c] += q[j] * dout[c];
-                        s += G[j][c] * k[j];
+                        dq2[j] = fma2(f2(S[j][c], S[j][c + 1]), do2, dq2[j]);
+                        const float2 g = fma2(q2[j], do2, f2(G[j][c], G[j][c + 1]));
+                        G[j][c] = g.x;
+                        G[j][c + 1] = g.y;
+                        s = fma2(g, k2[j], s);
                     }
-                    part[c] = s;
+                    part[c] = s.x;
+                    part[c + 1] = s.y;
                 }
+#pragma unroll
+                for (int j = 0; j < J; ++j) dq[j] = dq2[j].x + dq2[j].y + k[j] * bed;
                 const float u_mine = reduce_scatter<WC>(part, lane);
                 const float de_mine = beta * u_mine;                                                   // de = beta G^T k  (= dv)
                 const float dbeta = warp_sum((lane & (32 / WC - 1)) == 0 ? u_mine * e_mine : 0.f);   // this warp's columns of k^T G e
 #pragma unroll
                 for (int c = 0; c < WC; ++c) de[c] = __shfl_sync(0xffffffffu, de_mine, lane_of_col<WC>(c));
                 // dk = beta G e - S~ de;  G <- alpha (G - k de^T);  dlog_alpha = <G - k de^T, S~>
-                float dla = 0.f;
+                float2 dla2 = f2(0.f);
 #pragma unroll
                 for (int j = 0; j < J; ++j) {
-                    float ge = 0.f, sd = 0.f;
+                    float2 ge = f2(0.f), sd = f2(0.f);
+                    const float2 nk2 = f2(-k[j]);
 #pragma unroll
-                    for (int c = 0; c < WC; ++c) {
-                        ge += G[j][c] * e[c];
-                        sd += S[j][c] * de[c];
-                        const float g = G[j][c] - k[j] * de[c];
-                        dla += g * S[j][c];
-                        G[j][c] = alpha * g;
+                    for (int c = 0; c < WC; c += 2) {
+                        const float2 g0 = f2(G[j][c], G[j][c + 1]), s0 = f2(S[j][c], S[j][c + 1]), de2 = f2(de[c], de[c + 1]);
+                        ge = fma2(g0, f2(e[c], e[c + 1]), ge);
+                        sd = fma2(s0, de2, sd);
+                        const float2 g = fma2(nk2, de2, g0);
+                        dla2 = fma2(g, s0, dla2);
+                        const float2 ga = mul2(a2, g);
+                        G[j][c] = ga.x;
+                        G[j][c + 1] = ga.y;
                     }
-                    dk[j] = beta * ge - sd;
+                    dk[j] = beta * (ge.x + ge.y) - (sd.x + sd.y);
                 }
+                float dla = dla2.x + dla2.y;
                 dla = warp_sum(dla);
                 float deta = dbeta;
                 if (!p.coeff_eta) {   // beta = eta / n: deta = dbeta / n, dn = -dbeta eta / n^2 = -dbeta beta / n, dk += 2 k dn

@@ -39,4 +39,12 @@ __device__ __forceinline__ float warp_sum(float x)
     return x;
 }
 
+// Packed fp32 arithmetic (two lanes of one instruction, sm_100): the token-by-token kernels are bound by instruction issue,
+// and their inner loops run over pairs of adjacent state columns.
+__device__ __forceinline__ float2 f2(float a, float b) { return make_float2(a, b); }
+__device__ __forceinline__ float2 f2(float a) { return make_float2(a, a); }
+__device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c) { return __ffma2_rn(a, b, c); }
+__device__ __forceinline__ float2 mul2(float2 a, float2 b) { return __fmul2_rn(a, b); }
+__device__ __forceinline__ float2 add2(float2 a, float2 b) { return __fadd2_rn(a, b); }
+
 }  // namespace kla

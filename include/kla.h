@@ -289,8 +289,9 @@ kla_status kla_dg_decode_step(const kla_desc *desc, const void *q, const void *k
  *   dinit_state    [n_seq, H, d_k, d_v] fp32, dL/dinit_state, or NULL to skip; an empty sequence gets d_final_state
  * All arithmetic is fp32 on CUDA cores.  The forward states are not an input: they are recomputed (a state is kept every
  * 16 tokens on a forward sweep, the ones in between are re-run when the reverse sweep reaches them), which needs
- * desc->workspace of kla_bwd_workspace_bytes(desc) bytes: (B T / 16 + n_seq + 16 n_seq) x H x d_k x d_v fp32
- * (host function; 0 for an invalid descriptor).  Errors as kla_chunk_fwd.
+ * desc->workspace of kla_bwd_workspace_bytes(desc) bytes: (B T / 16 + n_seq) x H x d_k x d_v fp32 for the kept states,
+ * 16 x 64 x d_k fp32 of scratch per resident thread block (at most one per SM) and 256 bytes (host function; it reads
+ * the current device's SM count when a device is present; 0 for an invalid descriptor).  Errors as kla_chunk_fwd.
  */
 size_t kla_bwd_workspace_bytes(const kla_desc *desc);
 kla_status kla_bwd(const kla_desc *desc, const void *q, const void *k, const void *v,

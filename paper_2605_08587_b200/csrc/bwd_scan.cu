@@ -11,7 +11,8 @@
 //
 // The step needs S_{t-1}, which only a forward sweep can give.  States are kept every L = 16 tokens on the way forward
 // (one state per 16 tokens of workspace); on the way back each block of 16 tokens is first re-run from its stored state
-// with the state before every token written to a per-head scratch area (16 states, L2-resident), then walked in reverse.
+// with the state before every token written to the thread block's scratch area (16 states, L2-resident), then walked in
+// reverse.  One block per SM is resident; (sequence, head, half) units beyond that are taken in turn.
 // Every thread reads back only what it wrote itself, so no fence or barrier guards the stored states.
 //
 // Work split: columns of S and G never interact, so a block owns 64 columns of one (sequence, head), one warp 8 of them,
@@ -43,11 +44,13 @@ struct BwdParams {
     float *dlog_alpha, *deta;          // [n_tok, H]
     float *dinit;                      // [n_seq, H, D, D] or null
     float *stored;                     // states every L tokens: slot (tok0 / L + n + block) * H + h
-    float *scratch;                    // L states per (sequence, head)
+    float *scratch;                    // L states of 64 columns per resident block
     const int32_t *cu_seqlens;         // null: fixed length T
     int32_t T, H, n_seq;
     float eps;
     int32_t coeff_eta;
+    int32_t n_units;                   // (sequence, head, 64-column half) units; the resident blocks take them in turn
+    int32_t *next_unit;                // zeroed before the launch: units beyond the first gridDim.x are handed out in order
 };
 
 // One block of L tokens as the steps read it.
@@ -69,7 +72,14 @@ __global__ void __launch_bounds__(NT, 1) kla_bwd_scan_kernel(BwdParams p)
     float *const red_all = smem_all + 2 * sizeof(Stage<D>) / sizeof(float);            // [RL][WARPS][NRED]: the warps' partial sums over their columns
     auto red = [&](int slot, int w) { return red_all + ((size_t)slot * WARPS + w) * NRED; };
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int split = blockIdx.x % SPLIT, h = (blockIdx.x / SPLIT) % p.H, n = blockIdx.x / (SPLIT * p.H);
+    const int myc = col_of_lane<WC>(lane);       // the column whose row sums this lane ends up with
+    const IO *qp = reinterpret_cast<const IO *>(p.q), *kp = reinterpret_cast<const IO *>(p.k), *vp = reinterpret_cast<const IO *>(p.v);
+    const IO *dop = reinterpret_cast<const IO *>(p.dout);
+    // the scratch states belong to the block, not to the unit it is working on
+    float *const scratch = p.scratch + (size_t)blockIdx.x * L * 64 * D + ((size_t)warp * J * (WC / 4)) * 128 + lane * 4;
+    __shared__ int unit_s;
+    for (int unit = blockIdx.x; unit < p.n_units;) {
+    const int split = unit % SPLIT, h = (unit / SPLIT) % p.H, n = unit / (SPLIT * p.H);
     int tok0, len;
     if (p.cu_seqlens) {
         tok0 = p.cu_seqlens[n];
@@ -80,12 +90,10 @@ __global__ void __launch_bounds__(NT, 1) kla_bwd_scan_kernel(BwdParams p)
     }
     const int cg = split * WARPS + warp;         // column group within the head
     const int c0 = cg * WC;                      // first column of this warp
-    const int myc = col_of_lane<WC>(lane);       // the column whose row sums this lane ends up with
     const size_t sbase = ((size_t)n * p.H + h) * D * D;
     // Stored states use a layout of their own, [column group][j][quad of columns][lane] float4, so that every access is 512 contiguous bytes.
     const size_t soff = ((size_t)cg * J * (WC / 4)) * 128 + lane * 4;
     float *const stored = p.stored + ((size_t)(tok0 / L + n) * p.H + h) * D * D + soff;
-    float *const scratch = p.scratch + ((size_t)n * p.H + h) * L * D * D + soff;
     auto put = [&](float *dst, const float (&S)[J][WC]) {
 #pragma unroll
         for (int j = 0; j < J; ++j)
@@ -113,9 +121,6 @@ __global__ void __launch_bounds__(NT, 1) kla_bwd_scan_kernel(BwdParams p)
                 S[j][c] = a.x; S[j][c + 1] = a.y; S[j][c + 2] = a.z; S[j][c + 3] = a.w;
             }
     };
-
-    const IO *qp = reinterpret_cast<const IO *>(p.q), *kp = reinterpret_cast<const IO *>(p.k), *vp = reinterpret_cast<const IO *>(p.v);
-    const IO *dop = reinterpret_cast<const IO *>(p.dout);
 
     float S[J][WC], G[J][WC];
     get_natural(p.init_state, S);
@@ -236,13 +241,13 @@ __global__ void __launch_bounds__(NT, 1) kla_bwd_scan_kernel(BwdParams p)
             if (b != n_blocks - 1) get(stored + (size_t)b * p.H * D * D, S);
             // the state before every token of the block (the last one stays in registers)
             for (int tok = 0; tok + 1 < cnt; ++tok) {
-                put(scratch + (size_t)tok * D * D, S);
+                put(scratch + (size_t)tok * 64 * D, S);
                 fstep(st, tok);
             }
             for (int tok = cnt - 1; tok >= 0; --tok) {
                 // S holds the state before this token; the one before the previous token is requested now, used next iteration
                 float Sn[J][WC];
-                if (tok > 0) get(scratch + (size_t)(tok - 1) * D * D, Sn);
+                if (tok > 0) get(scratch + (size_t)(tok - 1) * 64 * D, Sn);
                 const size_t th = (size_t)(tok0 + i0 + tok) * p.H + h;
                 float q[J], k[J], dout[WC];
 #pragma unroll
@@ -395,13 +400,28 @@ __global__ void __launch_bounds__(NT, 1) kla_bwd_scan_kernel(BwdParams p)
             for (int c = 0; c < WC; c += 4)
                 store4(p.dinit + sbase + (size_t)(lane + 32 * j) * D + c0 + c, make_float4(G[j][c], G[j][c + 1], G[j][c + 2], G[j][c + 3]));
     }
+    // the next unit, in the order blocks become free (packed input: lengths differ)
+    __syncthreads();
+    if (threadIdx.x == 0) unit_s = (int)gridDim.x + atomicAdd(p.next_unit, 1);
+    __syncthreads();
+    unit = unit_s;
+    }   // units
+}
+
+// One block per SM (registers and shared memory); more units than that are taken in turn.
+int bwd_resident_blocks()
+{
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+        return 148;
+    return n;
 }
 
 template <int D, typename IO>
 cudaError_t launch_io(const BwdParams &p, int qnorm, cudaStream_t stream)
 {
-    const int blocks = p.n_seq * p.H * (D / 64);
-    if (blocks == 0) return cudaSuccess;
+    if (p.n_units == 0) return cudaSuccess;
+    const int blocks = p.n_units < bwd_resident_blocks() ? p.n_units : bwd_resident_blocks();
     constexpr int smem = 2 * (int)sizeof(Stage<D>) + RL * WARPS * (2 * D + 2) * (int)sizeof(float);
     auto kern = qnorm ? kla_bwd_scan_kernel<D, IO, true> : kla_bwd_scan_kernel<D, IO, false>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
@@ -416,7 +436,9 @@ cudaError_t launch_io(const BwdParams &p, int qnorm, cudaStream_t stream)
 size_t bwd_workspace_bytes(int n_seq, long long n_tok, int H, int d)
 {
     const size_t state = (size_t)d * d * sizeof(float);
-    return ((size_t)(n_tok / L + n_seq) * H + (size_t)n_seq * H * L) * state;
+    const long long units = (long long)n_seq * H * (d / 64);
+    const size_t blocks = (size_t)(units < bwd_resident_blocks() ? units : bwd_resident_blocks());
+    return 256 + (size_t)(n_tok / L + n_seq) * H * state + blocks * L * 64 * d * sizeof(float);   // (256: the unit counter)
 }
 
 cudaError_t launch_bwd_scan(const void *q, const void *k, const void *v, const float *log_alpha, const float *eta,
@@ -430,12 +452,15 @@ cudaError_t launch_bwd_scan(const void *q, const void *k, const void *v, const f
     p.log_alpha = log_alpha; p.eta = eta;
     p.init_state = init_state; p.dfinal = dfinal;
     p.dq = dq; p.dk = dk; p.dv = dv; p.dlog_alpha = dlog_alpha; p.deta = deta; p.dinit = dinit;
-    p.stored = reinterpret_cast<float *>(workspace);
+    p.next_unit = reinterpret_cast<int32_t *>(workspace);
+    p.stored = reinterpret_cast<float *>(reinterpret_cast<char *>(workspace) + 256);
     p.scratch = p.stored + (size_t)(n_tok / L + n_seq) * H * d * d;
+    if (cudaMemsetAsync(p.next_unit, 0, sizeof(int32_t), stream) != cudaSuccess) return cudaGetLastError();
     p.cu_seqlens = cu_seqlens;
     p.T = T; p.H = H; p.n_seq = n_seq;
     p.eps = eps;
     p.coeff_eta = coeff_eta;
+    p.n_units = n_seq * H * (d / 64);
     if (d == 128) {   // two blocks per head add into the outputs that are sums over columns
         cudaError_t e = cudaMemsetAsync(dq, 0, (size_t)n_tok * H * d * sizeof(float), stream);
         if (e == cudaSuccess) e = cudaMemsetAsync(dk, 0, (size_t)n_tok * H * d * sizeof(float), stream);

@@ -127,7 +127,8 @@ def test_workspace_is_checked_and_a_caller_supplied_one_is_used():
     args = [x.to(DEV) for x in (w.q, w.k, w.v, w.log_alpha, w.eta)]
     desc = binding.KlaDesc(B=1, T=64, H=2, d_k=64, d_v=64, n_seq=1, io_dtype=binding.KLA_BF16, out_dtype=binding.KLA_F32)
     need = int(binding.load().kla_bwd_workspace_bytes(ctypes.byref(desc)))
-    assert need == (64 // 16 + 1 + 16) * 2 * 64 * 64 * 4
+    # kept states (one per 16 tokens and one more per sequence) per head, scratch of the two resident blocks, unit counter
+    assert need == (64 // 16 + 1) * 2 * 64 * 64 * 4 + 2 * 16 * 64 * 64 * 4 + 256
     with pytest.raises(KlaError) as e:
         kla_bwd(*args, w.eps, do.to(DEV), workspace=torch.empty(need - 16, device=DEV, dtype=torch.uint8))
     assert e.value.code == -7   # KLA_ERR_WORKSPACE

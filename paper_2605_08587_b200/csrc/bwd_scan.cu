@@ -79,333 +79,333 @@ __global__ void __launch_bounds__(NT, 1) kla_bwd_scan_kernel(BwdParams p)
     float *const scratch = p.scratch + (size_t)blockIdx.x * L * 64 * D + ((size_t)warp * J * (WC / 4)) * 128 + lane * 4;
     __shared__ int unit_s;
     for (int unit = blockIdx.x; unit < p.n_units;) {
-    const int split = unit % SPLIT, h = (unit / SPLIT) % p.H, n = unit / (SPLIT * p.H);
-    int tok0, len;
-    if (p.cu_seqlens) {
-        tok0 = p.cu_seqlens[n];
-        len = p.cu_seqlens[n + 1] - tok0;
-    } else {
-        tok0 = n * p.T;
-        len = p.T;
-    }
-    const int cg = split * WARPS + warp;         // column group within the head
-    const int c0 = cg * WC;                      // first column of this warp
-    const size_t sbase = ((size_t)n * p.H + h) * D * D;
-    // Stored states use a layout of their own, [column group][j][quad of columns][lane] float4, so that every access is 512 contiguous bytes.
-    const size_t soff = ((size_t)cg * J * (WC / 4)) * 128 + lane * 4;
-    float *const stored = p.stored + ((size_t)(tok0 / L + n) * p.H + h) * D * D + soff;
-    auto put = [&](float *dst, const float (&S)[J][WC]) {
-#pragma unroll
-        for (int j = 0; j < J; ++j)
-#pragma unroll
-            for (int c = 0; c < WC; c += 4)
-                store4(dst + (j * (WC / 4) + c / 4) * 128, make_float4(S[j][c], S[j][c + 1], S[j][c + 2], S[j][c + 3]));
-    };
-    auto get = [&](const float *src, float (&S)[J][WC]) {
-#pragma unroll
-        for (int j = 0; j < J; ++j)
-#pragma unroll
-            for (int c = 0; c < WC; c += 4) {
-                const float4 a = load4(src + (j * (WC / 4) + c / 4) * 128);
-                S[j][c] = a.x; S[j][c + 1] = a.y; S[j][c + 2] = a.z; S[j][c + 3] = a.w;
-            }
-    };
-    // the caller's states are [row][column]
-    auto get_natural = [&](const float *src, float (&S)[J][WC]) {
-#pragma unroll
-        for (int j = 0; j < J; ++j)
-#pragma unroll
-            for (int c = 0; c < WC; c += 4) {
-                float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (src) a = load4(src + sbase + (size_t)(lane + 32 * j) * D + c0 + c);
-                S[j][c] = a.x; S[j][c + 1] = a.y; S[j][c + 2] = a.z; S[j][c + 3] = a.w;
-            }
-    };
-
-    float S[J][WC], G[J][WC];
-    get_natural(p.init_state, S);
-    get_natural(p.dfinal, G);
-    const int n_blocks = (len + L - 1) / L;
-
-    // ---- operands of one block of L tokens, staged in shared memory as fp32 together with the per-token scalars ----
-    // Each warp fetches whole tokens (TPW of them): the raw values are requested into registers before the block in hand
-    // is processed and touched only after it (a use, even a conversion, would wait for them), then converted, reduced to
-    // alpha, beta (Eq. 3), ||k||^2 + eps and 1 / ||q||, and written to the buffer that is not being read.
-    constexpr int TPW = L / WARPS;
-    struct Pre { IO k[J], q[J]; IO v[2], dout[2]; float la, eta; };
-    Pre pre[TPW];
-    auto request_block = [&](int b, bool full) {
-#pragma unroll
-        for (int u = 0; u < TPW; ++u) {
-            const int i = min(b * L + warp + u * WARPS, len - 1);
-            const size_t th = (size_t)(tok0 + i) * p.H + h;
-#pragma unroll
-            for (int j = 0; j < J; ++j) {
-                pre[u].k[j] = kp[th * D + lane + 32 * j];
-                if (full) pre[u].q[j] = qp[th * D + lane + 32 * j];
-            }
-            const size_t col = th * D + split * 64 + 2 * lane;   // this block's 64 columns, two per lane
-            if constexpr (sizeof(IO) == 2) {
-                *reinterpret_cast<uint32_t *>(pre[u].v) = *reinterpret_cast<const uint32_t *>(vp + col);
-                if (full) *reinterpret_cast<uint32_t *>(pre[u].dout) = *reinterpret_cast<const uint32_t *>(dop + col);
-            } else {
-                *reinterpret_cast<float2 *>(pre[u].v) = *reinterpret_cast<const float2 *>(vp + col);
-                if (full) *reinterpret_cast<float2 *>(pre[u].dout) = *reinterpret_cast<const float2 *>(dop + col);
-            }
-            pre[u].la = p.log_alpha[th];
-            pre[u].eta = p.eta[th];
+        const int split = unit % SPLIT, h = (unit / SPLIT) % p.H, n = unit / (SPLIT * p.H);
+        int tok0, len;
+        if (p.cu_seqlens) {
+            tok0 = p.cu_seqlens[n];
+            len = p.cu_seqlens[n + 1] - tok0;
+        } else {
+            tok0 = n * p.T;
+            len = p.T;
         }
-    };
-    auto commit_block = [&](Stage<D> &st, bool full) {
+        const int cg = split * WARPS + warp;         // column group within the head
+        const int c0 = cg * WC;                      // first column of this warp
+        const size_t sbase = ((size_t)n * p.H + h) * D * D;
+        // Stored states use a layout of their own, [column group][j][quad of columns][lane] float4, so that every access is 512 contiguous bytes.
+        const size_t soff = ((size_t)cg * J * (WC / 4)) * 128 + lane * 4;
+        float *const stored = p.stored + ((size_t)(tok0 / L + n) * p.H + h) * D * D + soff;
+        auto put = [&](float *dst, const float (&S)[J][WC]) {
 #pragma unroll
-        for (int u = 0; u < TPW; ++u) {
-            const int tok = warp + u * WARPS;
-            float nk = 0.f, nq = 0.f, q[J];
+            for (int j = 0; j < J; ++j)
 #pragma unroll
-            for (int j = 0; j < J; ++j) {
-                const float k = to_f32(pre[u].k[j]);
-                st.k[tok][lane + 32 * j] = k;
-                nk += k * k;
-                if (full) {
-                    q[j] = to_f32(pre[u].q[j]);
-                    nq += q[j] * q[j];
-                }
-            }
-            const float nrm = warp_sum(nk) + p.eps;
-            float qinv = 1.f;
-            if (QN && full) qinv = rsqrtf(warp_sum(nq));
-            store2(&st.v[tok][2 * lane], to_f32(pre[u].v[0]), to_f32(pre[u].v[1]));
-            if (full) {
+                for (int c = 0; c < WC; c += 4)
+                    store4(dst + (j * (WC / 4) + c / 4) * 128, make_float4(S[j][c], S[j][c + 1], S[j][c + 2], S[j][c + 3]));
+        };
+        auto get = [&](const float *src, float (&S)[J][WC]) {
 #pragma unroll
-                for (int j = 0; j < J; ++j) st.q[tok][lane + 32 * j] = q[j] * qinv;   // qh
-                store2(&st.dout[tok][2 * lane], to_f32(pre[u].dout[0]), to_f32(pre[u].dout[1]));
-            }
-            if (lane == 0) {
-                st.alpha[tok] = __expf(pre[u].la);
-                st.beta[tok] = p.coeff_eta ? pre[u].eta : pre[u].eta / nrm;   // Eq. 3
-                st.nrm[tok] = nrm;
-                st.qinv[tok] = qinv;
-            }
-        }
-    };
-    // one forward step without read-out
-    auto fstep = [&](const Stage<D> &st, int tok) {
-        float2 k[J];   // (k_j, k_j)
-        float part[WC];
-#pragma unroll
-        for (int j = 0; j < J; ++j) k[j] = f2(st.k[tok][lane + 32 * j]);
-        const float alpha = st.alpha[tok], beta = st.beta[tok];
-#pragma unroll
-        for (int c = 0; c < WC; c += 2) {
-            float2 s = f2(0.f);
-#pragma unroll
-            for (int j = 0; j < J; ++j) s = fma2(k[j], f2(S[j][c], S[j][c + 1]), s);
-            part[c] = s.x;
-            part[c + 1] = s.y;
-        }
-        const float e_mine = st.v[tok][warp * WC + myc] - alpha * reduce_scatter<WC>(part, lane);
-        const float2 a2 = f2(alpha);
-#pragma unroll
-        for (int c = 0; c < WC; c += 2) {
-            const float2 be = f2(beta * __shfl_sync(0xffffffffu, e_mine, lane_of_col<WC>(c)),
-                                 beta * __shfl_sync(0xffffffffu, e_mine, lane_of_col<WC>(c + 1)));
-#pragma unroll
-            for (int j = 0; j < J; ++j) {
-                const float2 r = fma2(a2, f2(S[j][c], S[j][c + 1]), mul2(k[j], be));
-                S[j][c] = r.x;
-                S[j][c + 1] = r.y;
-            }
-        }
-    };
-
-    if (n_blocks > 0) {
-        int cur = 0;
-        request_block(0, n_blocks == 1);
-        commit_block(stage[0], n_blocks == 1);
-        __syncthreads();
-        // forward sweep up to the start of the last block, keeping the state at the start of every block
-        for (int b = 0; b + 1 < n_blocks; ++b) {
-            const bool next_full = b + 2 == n_blocks;   // the last block is the first one the reverse sweep works on
-            request_block(b + 1, next_full);
-            put(stored + (size_t)b * p.H * D * D, S);
-            for (int tok = 0; tok < L; ++tok) fstep(stage[cur], tok);
-            commit_block(stage[cur ^ 1], next_full);
-            __syncthreads();   // one barrier per block: the buffer written is the one nobody reads
-            cur ^= 1;
-        }
-        // ---- reverse sweep, block by block ----
-        for (int b = n_blocks - 1; b >= 0; --b) {
-            const int i0 = b * L, cnt = min(L, len - i0);
-            const Stage<D> &st = stage[cur];
-            if (b > 0) request_block(b - 1, true);
-            if (b != n_blocks - 1) get(stored + (size_t)b * p.H * D * D, S);
-            // the state before every token of the block (the last one stays in registers)
-            for (int tok = 0; tok + 1 < cnt; ++tok) {
-                put(scratch + (size_t)tok * 64 * D, S);
-                fstep(st, tok);
-            }
-            for (int tok = cnt - 1; tok >= 0; --tok) {
-                // S holds the state before this token; the one before the previous token is requested now, used next iteration
-                float Sn[J][WC];
-                if (tok > 0) get(scratch + (size_t)(tok - 1) * 64 * D, Sn);
-                const size_t th = (size_t)(tok0 + i0 + tok) * p.H + h;
-                float q[J], k[J], dout[WC];
-#pragma unroll
-                for (int j = 0; j < J; ++j) {
-                    q[j] = st.q[tok][lane + 32 * j];   // qh
-                    k[j] = st.k[tok][lane + 32 * j];
-                }
+            for (int j = 0; j < J; ++j)
 #pragma unroll
                 for (int c = 0; c < WC; c += 4) {
-                    const float4 x = load4(&st.dout[tok][warp * WC + c]);
-                    dout[c] = x.x; dout[c + 1] = x.y; dout[c + 2] = x.z; dout[c + 3] = x.w;
+                    const float4 a = load4(src + (j * (WC / 4) + c / 4) * 128);
+                    S[j][c] = a.x; S[j][c + 1] = a.y; S[j][c + 2] = a.z; S[j][c + 3] = a.w;
                 }
-                const float alpha = st.alpha[tok], beta = st.beta[tok], nrm = st.nrm[tok];
-                // forward quantities of the token: S~ = alpha S_{t-1} (in place), e = v - S~^T k
-                float part[WC], e[WC], de[WC];
-                float2 k2[J], q2[J];
+        };
+        // the caller's states are [row][column]
+        auto get_natural = [&](const float *src, float (&S)[J][WC]) {
+#pragma unroll
+            for (int j = 0; j < J; ++j)
+#pragma unroll
+                for (int c = 0; c < WC; c += 4) {
+                    float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (src) a = load4(src + sbase + (size_t)(lane + 32 * j) * D + c0 + c);
+                    S[j][c] = a.x; S[j][c + 1] = a.y; S[j][c + 2] = a.z; S[j][c + 3] = a.w;
+                }
+        };
+
+        float S[J][WC], G[J][WC];
+        get_natural(p.init_state, S);
+        get_natural(p.dfinal, G);
+        const int n_blocks = (len + L - 1) / L;
+
+        // ---- operands of one block of L tokens, staged in shared memory as fp32 together with the per-token scalars ----
+        // Each warp fetches whole tokens (TPW of them): the raw values are requested into registers before the block in hand
+        // is processed and touched only after it (a use, even a conversion, would wait for them), then converted, reduced to
+        // alpha, beta (Eq. 3), ||k||^2 + eps and 1 / ||q||, and written to the buffer that is not being read.
+        constexpr int TPW = L / WARPS;
+        struct Pre { IO k[J], q[J]; IO v[2], dout[2]; float la, eta; };
+        Pre pre[TPW];
+        auto request_block = [&](int b, bool full) {
+#pragma unroll
+            for (int u = 0; u < TPW; ++u) {
+                const int i = min(b * L + warp + u * WARPS, len - 1);
+                const size_t th = (size_t)(tok0 + i) * p.H + h;
 #pragma unroll
                 for (int j = 0; j < J; ++j) {
-                    k2[j] = f2(k[j]);
-                    q2[j] = f2(q[j]);
+                    pre[u].k[j] = kp[th * D + lane + 32 * j];
+                    if (full) pre[u].q[j] = qp[th * D + lane + 32 * j];
                 }
-                const float2 a2 = f2(alpha);
-#pragma unroll
-                for (int c = 0; c < WC; c += 2) {
-                    float2 s = f2(0.f);
-#pragma unroll
-                    for (int j = 0; j < J; ++j) {
-                        const float2 st2 = mul2(a2, f2(S[j][c], S[j][c + 1]));
-                        S[j][c] = st2.x;
-                        S[j][c + 1] = st2.y;
-                        s = fma2(k2[j], st2, s);
-                    }
-                    part[c] = s.x;
-                    part[c + 1] = s.y;
+                const size_t col = th * D + split * 64 + 2 * lane;   // this block's 64 columns, two per lane
+                if constexpr (sizeof(IO) == 2) {
+                    *reinterpret_cast<uint32_t *>(pre[u].v) = *reinterpret_cast<const uint32_t *>(vp + col);
+                    if (full) *reinterpret_cast<uint32_t *>(pre[u].dout) = *reinterpret_cast<const uint32_t *>(dop + col);
+                } else {
+                    *reinterpret_cast<float2 *>(pre[u].v) = *reinterpret_cast<const float2 *>(vp + col);
+                    if (full) *reinterpret_cast<float2 *>(pre[u].dout) = *reinterpret_cast<const float2 *>(dop + col);
                 }
-                const float e_mine = st.v[tok][warp * WC + myc] - reduce_scatter<WC>(part, lane);
+                pre[u].la = p.log_alpha[th];
+                pre[u].eta = p.eta[th];
+            }
+        };
+        auto commit_block = [&](Stage<D> &st, bool full) {
 #pragma unroll
-                for (int c = 0; c < WC; ++c) e[c] = __shfl_sync(0xffffffffu, e_mine, lane_of_col<WC>(c));
-                // read-out: dqh = S_t dO = S~ dO + k (beta e . dO); G += qh dO^T; then u = G^T k
-                float dq[J], dk[J];
-                float2 dq2[J];
-                float bed = 0.f;   // beta e . dO over this warp's columns
-#pragma unroll
-                for (int c = 0; c < WC; ++c) bed += e[c] * dout[c];
-                bed *= beta;
-#pragma unroll
-                for (int j = 0; j < J; ++j) dq2[j] = f2(0.f);
-#pragma unroll
-                for (int c = 0; c < WC; c += 2) {
-                    const float2 do2 = f2(dout[c], dout[c + 1]);
-                    float2 s = f2(0.f);
-#pragma unroll
-                    for (int j = 0; j < J; ++j) {
-                        dq2[j] = fma2(f2(S[j][c], S[j][c + 1]), do2, dq2[j]);
-                        const float2 g = fma2(q2[j], do2, f2(G[j][c], G[j][c + 1]));
-                        G[j][c] = g.x;
-                        G[j][c + 1] = g.y;
-                        s = fma2(g, k2[j], s);
-                    }
-                    part[c] = s.x;
-                    part[c + 1] = s.y;
-                }
-#pragma unroll
-                for (int j = 0; j < J; ++j) dq[j] = dq2[j].x + dq2[j].y + k[j] * bed;
-                const float u_mine = reduce_scatter<WC>(part, lane);
-                const float de_mine = beta * u_mine;                                                   // de = beta G^T k  (= dv)
-                const float dbeta = warp_sum((lane & (32 / WC - 1)) == 0 ? u_mine * e_mine : 0.f);   // this warp's columns of k^T G e
-#pragma unroll
-                for (int c = 0; c < WC; ++c) de[c] = __shfl_sync(0xffffffffu, de_mine, lane_of_col<WC>(c));
-                // dk = beta G e - S~ de;  G <- alpha (G - k de^T);  dlog_alpha = <G - k de^T, S~>
-                float2 dla2 = f2(0.f);
+            for (int u = 0; u < TPW; ++u) {
+                const int tok = warp + u * WARPS;
+                float nk = 0.f, nq = 0.f, q[J];
 #pragma unroll
                 for (int j = 0; j < J; ++j) {
-                    float2 ge = f2(0.f), sd = f2(0.f);
-                    const float2 nk2 = f2(-k[j]);
-#pragma unroll
-                    for (int c = 0; c < WC; c += 2) {
-                        const float2 g0 = f2(G[j][c], G[j][c + 1]), s0 = f2(S[j][c], S[j][c + 1]), de2 = f2(de[c], de[c + 1]);
-                        ge = fma2(g0, f2(e[c], e[c + 1]), ge);
-                        sd = fma2(s0, de2, sd);
-                        const float2 g = fma2(nk2, de2, g0);
-                        dla2 = fma2(g, s0, dla2);
-                        const float2 ga = mul2(a2, g);
-                        G[j][c] = ga.x;
-                        G[j][c + 1] = ga.y;
+                    const float k = to_f32(pre[u].k[j]);
+                    st.k[tok][lane + 32 * j] = k;
+                    nk += k * k;
+                    if (full) {
+                        q[j] = to_f32(pre[u].q[j]);
+                        nq += q[j] * q[j];
                     }
-                    dk[j] = beta * (ge.x + ge.y) - (sd.x + sd.y);
                 }
-                float dla = dla2.x + dla2.y;
-                dla = warp_sum(dla);
-                float deta = dbeta;
-                if (!p.coeff_eta) {   // beta = eta / n: deta = dbeta / n, dn = -dbeta eta / n^2 = -dbeta beta / n, dk += 2 k dn
-                    deta = dbeta / nrm;
-                    const float dn2 = -2.f * dbeta * beta / nrm;
+                const float nrm = warp_sum(nk) + p.eps;
+                float qinv = 1.f;
+                if (QN && full) qinv = rsqrtf(warp_sum(nq));
+                store2(&st.v[tok][2 * lane], to_f32(pre[u].v[0]), to_f32(pre[u].v[1]));
+                if (full) {
 #pragma unroll
-                    for (int j = 0; j < J; ++j) dk[j] += k[j] * dn2;
-                }
-                if (QN) {   // o = S^T q / ||q||: dq = (dqh - qh (qh . dqh)) / ||q||, a linear map, applied to this warp's part
-                    float pr = 0.f;
-#pragma unroll
-                    for (int j = 0; j < J; ++j) pr += q[j] * dq[j];
-                    pr = warp_sum(pr);
-                    const float qinv = st.qinv[tok];
-#pragma unroll
-                    for (int j = 0; j < J; ++j) dq[j] = (dq[j] - q[j] * pr) * qinv;
-                }
-                if ((lane & (32 / WC - 1)) == 0) p.dv[th * D + c0 + myc] = de_mine;
-                // this warp's part of the sums over columns; added up every RL tokens
-                float *mine = red(tok % RL, warp);
-#pragma unroll
-                for (int j = 0; j < J; ++j) {
-                    mine[lane + 32 * j] = dq[j];
-                    mine[D + lane + 32 * j] = dk[j];
+                    for (int j = 0; j < J; ++j) st.q[tok][lane + 32 * j] = q[j] * qinv;   // qh
+                    store2(&st.dout[tok][2 * lane], to_f32(pre[u].dout[0]), to_f32(pre[u].dout[1]));
                 }
                 if (lane == 0) {
-                    mine[2 * D] = dla;
-                    mine[2 * D + 1] = deta;
-                }
-                if (tok > 0) {
-#pragma unroll
-                    for (int j = 0; j < J; ++j)
-#pragma unroll
-                        for (int c = 0; c < WC; ++c) S[j][c] = Sn[j][c];
-                }
-                if (tok % RL == 0) {   // add up the partial sums of tokens tok .. tok + RL - 1 (fewer at the end of the sequence)
-                    __syncthreads();
-                    const int n_sum = min(RL, cnt - tok);
-                    for (int idx = threadIdx.x; idx < n_sum * NRED; idx += NT) {
-                        const int slot = idx / NRED, x = idx - slot * NRED;
-                        float s = 0.f;
-#pragma unroll
-                        for (int w = 0; w < WARPS; ++w) s += red(slot, w)[x];
-                        const size_t tq = th + (size_t)slot * p.H;
-                        float *dst = x < D ? p.dq + tq * D + x : x < 2 * D ? p.dk + tq * D + (x - D) : x == 2 * D ? p.dlog_alpha + tq : p.deta + tq;
-                        if (SPLIT == 1) *dst = s;
-                        else atomicAdd(dst, s);
-                    }
-                    __syncthreads();
+                    st.alpha[tok] = __expf(pre[u].la);
+                    st.beta[tok] = p.coeff_eta ? pre[u].eta : pre[u].eta / nrm;   // Eq. 3
+                    st.nrm[tok] = nrm;
+                    st.qinv[tok] = qinv;
                 }
             }
-            if (b > 0) commit_block(stage[cur ^ 1], true);
+        };
+        // one forward step without read-out
+        auto fstep = [&](const Stage<D> &st, int tok) {
+            float2 k[J];   // (k_j, k_j)
+            float part[WC];
+#pragma unroll
+            for (int j = 0; j < J; ++j) k[j] = f2(st.k[tok][lane + 32 * j]);
+            const float alpha = st.alpha[tok], beta = st.beta[tok];
+#pragma unroll
+            for (int c = 0; c < WC; c += 2) {
+                float2 s = f2(0.f);
+#pragma unroll
+                for (int j = 0; j < J; ++j) s = fma2(k[j], f2(S[j][c], S[j][c + 1]), s);
+                part[c] = s.x;
+                part[c + 1] = s.y;
+            }
+            const float e_mine = st.v[tok][warp * WC + myc] - alpha * reduce_scatter<WC>(part, lane);
+            const float2 a2 = f2(alpha);
+#pragma unroll
+            for (int c = 0; c < WC; c += 2) {
+                const float2 be = f2(beta * __shfl_sync(0xffffffffu, e_mine, lane_of_col<WC>(c)),
+                                     beta * __shfl_sync(0xffffffffu, e_mine, lane_of_col<WC>(c + 1)));
+#pragma unroll
+                for (int j = 0; j < J; ++j) {
+                    const float2 r = fma2(a2, f2(S[j][c], S[j][c + 1]), mul2(k[j], be));
+                    S[j][c] = r.x;
+                    S[j][c + 1] = r.y;
+                }
+            }
+        };
+
+        if (n_blocks > 0) {
+            int cur = 0;
+            request_block(0, n_blocks == 1);
+            commit_block(stage[0], n_blocks == 1);
             __syncthreads();
-            cur ^= 1;
+            // forward sweep up to the start of the last block, keeping the state at the start of every block
+            for (int b = 0; b + 1 < n_blocks; ++b) {
+                const bool next_full = b + 2 == n_blocks;   // the last block is the first one the reverse sweep works on
+                request_block(b + 1, next_full);
+                put(stored + (size_t)b * p.H * D * D, S);
+                for (int tok = 0; tok < L; ++tok) fstep(stage[cur], tok);
+                commit_block(stage[cur ^ 1], next_full);
+                __syncthreads();   // one barrier per block: the buffer written is the one nobody reads
+                cur ^= 1;
+            }
+            // ---- reverse sweep, block by block ----
+            for (int b = n_blocks - 1; b >= 0; --b) {
+                const int i0 = b * L, cnt = min(L, len - i0);
+                const Stage<D> &st = stage[cur];
+                if (b > 0) request_block(b - 1, true);
+                if (b != n_blocks - 1) get(stored + (size_t)b * p.H * D * D, S);
+                // the state before every token of the block (the last one stays in registers)
+                for (int tok = 0; tok + 1 < cnt; ++tok) {
+                    put(scratch + (size_t)tok * 64 * D, S);
+                    fstep(st, tok);
+                }
+                for (int tok = cnt - 1; tok >= 0; --tok) {
+                    // S holds the state before this token; the one before the previous token is requested now, used next iteration
+                    float Sn[J][WC];
+                    if (tok > 0) get(scratch + (size_t)(tok - 1) * 64 * D, Sn);
+                    const size_t th = (size_t)(tok0 + i0 + tok) * p.H + h;
+                    float q[J], k[J], dout[WC];
+#pragma unroll
+                    for (int j = 0; j < J; ++j) {
+                        q[j] = st.q[tok][lane + 32 * j];   // qh
+                        k[j] = st.k[tok][lane + 32 * j];
+                    }
+#pragma unroll
+                    for (int c = 0; c < WC; c += 4) {
+                        const float4 x = load4(&st.dout[tok][warp * WC + c]);
+                        dout[c] = x.x; dout[c + 1] = x.y; dout[c + 2] = x.z; dout[c + 3] = x.w;
+                    }
+                    const float alpha = st.alpha[tok], beta = st.beta[tok], nrm = st.nrm[tok];
+                    // forward quantities of the token: S~ = alpha S_{t-1} (in place), e = v - S~^T k
+                    float part[WC], e[WC], de[WC];
+                    float2 k2[J], q2[J];
+#pragma unroll
+                    for (int j = 0; j < J; ++j) {
+                        k2[j] = f2(k[j]);
+                        q2[j] = f2(q[j]);
+                    }
+                    const float2 a2 = f2(alpha);
+#pragma unroll
+                    for (int c = 0; c < WC; c += 2) {
+                        float2 s = f2(0.f);
+#pragma unroll
+                        for (int j = 0; j < J; ++j) {
+                            const float2 st2 = mul2(a2, f2(S[j][c], S[j][c + 1]));
+                            S[j][c] = st2.x;
+                            S[j][c + 1] = st2.y;
+                            s = fma2(k2[j], st2, s);
+                        }
+                        part[c] = s.x;
+                        part[c + 1] = s.y;
+                    }
+                    const float e_mine = st.v[tok][warp * WC + myc] - reduce_scatter<WC>(part, lane);
+#pragma unroll
+                    for (int c = 0; c < WC; ++c) e[c] = __shfl_sync(0xffffffffu, e_mine, lane_of_col<WC>(c));
+                    // read-out: dqh = S_t dO = S~ dO + k (beta e . dO); G += qh dO^T; then u = G^T k
+                    float dq[J], dk[J];
+                    float2 dq2[J];
+                    float bed = 0.f;   // beta e . dO over this warp's columns
+#pragma unroll
+                    for (int c = 0; c < WC; ++c) bed += e[c] * dout[c];
+                    bed *= beta;
+#pragma unroll
+                    for (int j = 0; j < J; ++j) dq2[j] = f2(0.f);
+#pragma unroll
+                    for (int c = 0; c < WC; c += 2) {
+                        const float2 do2 = f2(dout[c], dout[c + 1]);
+                        float2 s = f2(0.f);
+#pragma unroll
+                        for (int j = 0; j < J; ++j) {
+                            dq2[j] = fma2(f2(S[j][c], S[j][c + 1]), do2, dq2[j]);
+                            const float2 g = fma2(q2[j], do2, f2(G[j][c], G[j][c + 1]));
+                            G[j][c] = g.x;
+                            G[j][c + 1] = g.y;
+                            s = fma2(g, k2[j], s);
+                        }
+                        part[c] = s.x;
+                        part[c + 1] = s.y;
+                    }
+#pragma unroll
+                    for (int j = 0; j < J; ++j) dq[j] = dq2[j].x + dq2[j].y + k[j] * bed;
+                    const float u_mine = reduce_scatter<WC>(part, lane);
+                    const float de_mine = beta * u_mine;                                                   // de = beta G^T k  (= dv)
+                    const float dbeta = warp_sum((lane & (32 / WC - 1)) == 0 ? u_mine * e_mine : 0.f);   // this warp's columns of k^T G e
+#pragma unroll
+                    for (int c = 0; c < WC; ++c) de[c] = __shfl_sync(0xffffffffu, de_mine, lane_of_col<WC>(c));
+                    // dk = beta G e - S~ de;  G <- alpha (G - k de^T);  dlog_alpha = <G - k de^T, S~>
+                    float2 dla2 = f2(0.f);
+#pragma unroll
+                    for (int j = 0; j < J; ++j) {
+                        float2 ge = f2(0.f), sd = f2(0.f);
+                        const float2 nk2 = f2(-k[j]);
+#pragma unroll
+                        for (int c = 0; c < WC; c += 2) {
+                            const float2 g0 = f2(G[j][c], G[j][c + 1]), s0 = f2(S[j][c], S[j][c + 1]), de2 = f2(de[c], de[c + 1]);
+                            ge = fma2(g0, f2(e[c], e[c + 1]), ge);
+                            sd = fma2(s0, de2, sd);
+                            const float2 g = fma2(nk2, de2, g0);
+                            dla2 = fma2(g, s0, dla2);
+                            const float2 ga = mul2(a2, g);
+                            G[j][c] = ga.x;
+                            G[j][c + 1] = ga.y;
+                        }
+                        dk[j] = beta * (ge.x + ge.y) - (sd.x + sd.y);
+                    }
+                    float dla = dla2.x + dla2.y;
+                    dla = warp_sum(dla);
+                    float deta = dbeta;
+                    if (!p.coeff_eta) {   // beta = eta / n: deta = dbeta / n, dn = -dbeta eta / n^2 = -dbeta beta / n, dk += 2 k dn
+                        deta = dbeta / nrm;
+                        const float dn2 = -2.f * dbeta * beta / nrm;
+#pragma unroll
+                        for (int j = 0; j < J; ++j) dk[j] += k[j] * dn2;
+                    }
+                    if (QN) {   // o = S^T q / ||q||: dq = (dqh - qh (qh . dqh)) / ||q||, a linear map, applied to this warp's part
+                        float pr = 0.f;
+#pragma unroll
+                        for (int j = 0; j < J; ++j) pr += q[j] * dq[j];
+                        pr = warp_sum(pr);
+                        const float qinv = st.qinv[tok];
+#pragma unroll
+                        for (int j = 0; j < J; ++j) dq[j] = (dq[j] - q[j] * pr) * qinv;
+                    }
+                    if ((lane & (32 / WC - 1)) == 0) p.dv[th * D + c0 + myc] = de_mine;
+                    // this warp's part of the sums over columns; added up every RL tokens
+                    float *mine = red(tok % RL, warp);
+#pragma unroll
+                    for (int j = 0; j < J; ++j) {
+                        mine[lane + 32 * j] = dq[j];
+                        mine[D + lane + 32 * j] = dk[j];
+                    }
+                    if (lane == 0) {
+                        mine[2 * D] = dla;
+                        mine[2 * D + 1] = deta;
+                    }
+                    if (tok > 0) {
+#pragma unroll
+                        for (int j = 0; j < J; ++j)
+#pragma unroll
+                            for (int c = 0; c < WC; ++c) S[j][c] = Sn[j][c];
+                    }
+                    if (tok % RL == 0) {   // add up the partial sums of tokens tok .. tok + RL - 1 (fewer at the end of the sequence)
+                        __syncthreads();
+                        const int n_sum = min(RL, cnt - tok);
+                        for (int idx = threadIdx.x; idx < n_sum * NRED; idx += NT) {
+                            const int slot = idx / NRED, x = idx - slot * NRED;
+                            float s = 0.f;
+#pragma unroll
+                            for (int w = 0; w < WARPS; ++w) s += red(slot, w)[x];
+                            const size_t tq = th + (size_t)slot * p.H;
+                            float *dst = x < D ? p.dq + tq * D + x : x < 2 * D ? p.dk + tq * D + (x - D) : x == 2 * D ? p.dlog_alpha + tq : p.deta + tq;
+                            if (SPLIT == 1) *dst = s;
+                            else atomicAdd(dst, s);
+                        }
+                        __syncthreads();
+                    }
+                }
+                if (b > 0) commit_block(stage[cur ^ 1], true);
+                __syncthreads();
+                cur ^= 1;
+            }
         }
-    }
-    if (p.dinit) {
+        if (p.dinit) {
 #pragma unroll
-        for (int j = 0; j < J; ++j)
+            for (int j = 0; j < J; ++j)
 #pragma unroll
-            for (int c = 0; c < WC; c += 4)
-                store4(p.dinit + sbase + (size_t)(lane + 32 * j) * D + c0 + c, make_float4(G[j][c], G[j][c + 1], G[j][c + 2], G[j][c + 3]));
+                for (int c = 0; c < WC; c += 4)
+                    store4(p.dinit + sbase + (size_t)(lane + 32 * j) * D + c0 + c, make_float4(G[j][c], G[j][c + 1], G[j][c + 2], G[j][c + 3]));
+        }
+        // the next unit, in the order blocks become free (packed input: lengths differ)
+        __syncthreads();
+        if (threadIdx.x == 0) unit_s = (int)gridDim.x + atomicAdd(p.next_unit, 1);
+        __syncthreads();
+        unit = unit_s;
     }
-    // the next unit, in the order blocks become free (packed input: lengths differ)
-    __syncthreads();
-    if (threadIdx.x == 0) unit_s = (int)gridDim.x + atomicAdd(p.next_unit, 1);
-    __syncthreads();
-    unit = unit_s;
-    }   // units
 }
 
 // One block per SM (registers and shared memory); more units than that are taken in turn.

@@ -494,6 +494,8 @@ def run_ours(args):
         extras["decode_l2_defeating_B512"] = decode_leg(dev, 128, 5, 1, peaks, B=512)
         extras["chunk_cfg3_long_context"] = chunk_leg(W.config3(), dev, 20, 3, peaks, torch.bfloat16)
         extras["chunk_cfg5_varlen"] = chunk_leg(W.config5(), dev, 20, 3, peaks, torch.bfloat16)
+        # a packed batch that one long sequence dominates: cut into pieces that start from warm-up runs
+        extras["chunk_packed_one_long_sequence"] = chunk_leg(W.config5_skewed(), dev, 10, 3, peaks, torch.bfloat16)
         extras["chunk_cfg2_wy_form"] = wy_leg(w, t, dev, 20, 3)
         extras["dg_fwd_layer_shape"] = dg_leg(dev, 10, 3, peaks)
         extras["bwd_layer_shape"] = bwd_leg(w, dev, 10, 3, peaks, not args.no_cpu_baseline)

@@ -96,7 +96,12 @@ typedef enum { KLA_F32 = 0, KLA_BF16 = 1 } kla_dtype;
  * everywhere; for every segment and head a warm-up of at most min(half a segment, 2048 tokens)); if they hold, one pass
  * over the segments (plus their warm-up chunks) does the work, otherwise the transition-map passes do.  The decision is
  * taken on the device, the call stays asynchronous; the workspace need is the same either way.  Not attempted with
- * KLA_FLAG_COEFF_ETA (no bound on beta ||k||^2), KLA_FLAG_WY_FORM or KLA_FLAG_EXACT_SEGMENTS. */
+ * KLA_FLAG_COEFF_ETA (no bound on beta ||k||^2), KLA_FLAG_WY_FORM or KLA_FLAG_EXACT_SEGMENTS.
+ * Packed input (cu_seqlens, tensor-core path, 2 <= n_seq <= 4096) is cut the same way, and only this way: when one
+ * sequence would set the length of the launch (it is well beyond the work per SM of an even spread), or when
+ * KLA_FLAG_SEGMENTS(g) asks for it (the longest sequence in g pieces, every sequence in pieces of that length), the long
+ * sequences are cut into pieces that start from warm-up runs; if the decay does not allow that, the plain launch runs
+ * instead (again decided on the device).  The workspace then also holds the piece tables. */
 #define KLA_FLAG_NO_SEGMENTS 2            /* never cut sequences into segments                              */
 #define KLA_FLAG_EXACT_SEGMENTS 128       /* segments always from chained transition maps, never from warm-up runs */
 #define KLA_FLAG_SEGMENTS(g) ((g) << 8)   /* force g segments per sequence, 2 <= g <= 255 (fewer if T is short) */

@@ -72,6 +72,51 @@ static size_t order_bytes(const kla_desc *d, int32_t chunk)
     return ((size_t)d->n_seq * sizeof(int32_t) + 255) & ~(size_t)255;
 }
 
+// Packed input, tensor-core path: long sequences are cut into pieces that start from decay-bounded warm-up runs when one
+// sequence would otherwise set the length of the launch (or when the caller forces a number of pieces for the longest).
+struct PackedPlan {
+    int seg_len = 0;      // tokens per piece (a multiple of 64); 0: sequences are not cut
+    int n_units = 0;      // pieces in all
+    size_t off_plan = 0, bytes = 0;   // the piece tables follow the longest-first order array in the workspace
+};
+
+static int sm_count();
+
+static PackedPlan plan_packed(const kla_desc *d, int32_t chunk)
+{
+    PackedPlan pp;
+    if (!order_bytes(d, chunk) || !d->host_seqlens) return pp;
+    if (d->flags & (KLA_FLAG_NO_SEGMENTS | KLA_FLAG_EXACT_SEGMENTS | KLA_FLAG_COEFF_ETA)) return pp;
+    if ((d->flags & KLA_FLAG_WY_FORM) && d->d_k == 128) return pp;
+    long long total = 0;
+    int longest = 0;
+    for (int n = 0; n < d->n_seq; ++n) {
+        if (d->host_seqlens[n + 1] < d->host_seqlens[n]) return pp;   // (refused by the argument check anyway)
+        const int c = (d->host_seqlens[n + 1] - d->host_seqlens[n] + 63) / 64;
+        total += c;
+        longest = c > longest ? c : longest;
+    }
+    const int forced = (d->flags >> 8) & 0xff;
+    int seg_chunks = 0;
+    if (forced >= 2) {
+        seg_chunks = (longest + forced - 1) / forced;
+    } else {
+        // chunks per SM if the work were spread evenly; a sequence well beyond that sets the length of the launch
+        const long long even = total * d->H * (d->d_k / 64) / sm_count();
+        const int target = even > 32 ? (int)even : 32;
+        if (longest >= target + target / 4 + 8) seg_chunks = target;
+    }
+    if (seg_chunks < 2) return pp;   // (the warm-up may take at most half a piece)
+    pp.seg_len = seg_chunks * 64;
+    for (int n = 0; n < d->n_seq; ++n)
+        pp.n_units += (d->host_seqlens[n + 1] - d->host_seqlens[n] + pp.seg_len - 1) / pp.seg_len;
+    if (pp.n_units <= d->n_seq) return PackedPlan();   // nothing is actually cut
+    pp.off_plan = order_bytes(d, chunk);
+    // bounds (n_units + 1), plan word, warm-up lengths (n_units x H), piece table (n_units)
+    pp.bytes = pp.off_plan + ((((size_t)pp.n_units * (d->H + 2) + 2) * sizeof(int32_t) + 255) & ~(size_t)255);
+    return pp;
+}
+
 // ---- segment-parallel scan: when to use it, and the workspace it needs ----------------------------------------------
 struct SegPlan {
     int G = 0;            // segments per sequence (0: plain launch)
@@ -141,7 +186,10 @@ size_t kla_chunk_fwd_workspace_bytes(const kla_desc *desc, int32_t chunk)
     if (check_common(desc) != KLA_OK) return 0;
     // the chunk kernels keep every intermediate on chip; scratch is needed by the segment-parallel scan and, for
     // packed input on the tensor-core path, by the longest-first order of the sequences
-    if (order_bytes(desc, chunk)) return order_bytes(desc, chunk);
+    if (order_bytes(desc, chunk)) {
+        const PackedPlan pp = plan_packed(desc, chunk);
+        return pp.seg_len ? pp.bytes : order_bytes(desc, chunk);
+    }
     return plan_segments(desc, chunk).bytes;
 }
 
@@ -149,7 +197,9 @@ size_t kla_chunk_fwd_plan_word_offset(const kla_desc *desc, int32_t chunk)
 {
     if (check_common(desc) != KLA_OK) return (size_t)-1;
     const SegPlan pl = plan_segments(desc, chunk);
-    return pl.G >= 2 ? ((size_t)desc->B * pl.G + 1) * sizeof(int32_t) : (size_t)-1;
+    if (pl.G >= 2) return ((size_t)desc->B * pl.G + 1) * sizeof(int32_t);
+    const PackedPlan pp = plan_packed(desc, chunk);
+    return pp.seg_len ? pp.off_plan + ((size_t)pp.n_units + 1) * sizeof(int32_t) : (size_t)-1;
 }
 
 }  // extern "C"
@@ -233,13 +283,31 @@ static kla_status chunk_fwd_impl(const kla_desc *desc, const void *q, const void
         return err == cudaSuccess ? KLA_OK : KLA_ERR_LAUNCH;
     }
     if (!(desc->flags & KLA_FLAG_FORCE_SIMT) && chunk_tc_supported(desc->d_k, chunk, desc->io_dtype)) {
+        const PackedPlan pp = plan_packed(desc, chunk);
         if (order_bytes(desc, chunk)) {
             int32_t *order = (int32_t *)desc->workspace;
             if (launch_seq_order(desc->cu_seqlens, desc->n_seq, order, stream) != cudaSuccess) return KLA_ERR_LAUNCH;
             p.seq_order = order;
         }
-        mark(1); mark(2); mark(3);
-        err = launch_chunk_tc(p, desc->d_k, desc->io_dtype, desc->out_dtype, stream);
+        if (pp.seg_len) {
+            // pieces from warm-up runs (pass 5) if the decay allows, else the plain launch (pass 6): a device word decides
+            int32_t *ub = (int32_t *)((char *)desc->workspace + pp.off_plan);
+            int32_t *unit_seq = ub + pp.n_units + 2 + (size_t)pp.n_units * desc->H;
+            if (launch_packed_units(desc->cu_seqlens, desc->n_seq, pp.seg_len, pp.n_units, ub, unit_seq, log_alpha, eta,
+                                    (long long)desc->T, desc->H, init_state, final_state, desc->d_k, stream) != cudaSuccess)
+                return KLA_ERR_LAUNCH;
+            mark(1); mark(2); mark(3);
+            ChunkParams p5 = p;
+            p5.cu_seqlens = ub; p5.n_seq = pp.n_units;
+            p5.seg_pass = 5; p5.seg_G = 0; p5.map_state = nullptr;
+            if (launch_chunk_tc(p5, desc->d_k, desc->io_dtype, desc->out_dtype, stream) != cudaSuccess) return KLA_ERR_LAUNCH;
+            p.seg_pass = 6;
+            p.seg_G = (int32_t)((ub + pp.n_units + 1) - p.seq_order);   // where the plan word is, counted from the order array
+            err = launch_chunk_tc(p, desc->d_k, desc->io_dtype, desc->out_dtype, stream);
+        } else {
+            mark(1); mark(2); mark(3);
+            err = launch_chunk_tc(p, desc->d_k, desc->io_dtype, desc->out_dtype, stream);
+        }
     }
     else {
         mark(1); mark(2); mark(3);

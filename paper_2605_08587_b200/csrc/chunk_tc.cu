@@ -416,12 +416,17 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     const int sl = sl2 % SLICES;
     const int h = (blockIdx.x / nslices) % p.H;
     int n = blockIdx.x / (nslices * p.H);
-    if (p.seg_pass == 1) n = (n / (p.seg_G - 1)) * p.seg_G + n % (p.seg_G - 1);
-    else if (p.seg_pass == 0 && p.seq_order) n = p.seq_order[n];   // packed input: longest sequences first
     const bool no_out = p.seg_pass == 1;
     // Segment passes: the word after the segment bounds says whether the segments start from decay-bounded warm-up runs
-    // (pass 4 alone does the work) or from chained transition maps (passes 1 and 3 do); the other kind returns at once.
-    if (p.seg_pass != 0 && (p.seg_pass == 4) != (p.cu_seqlens[p.n_seq + 1] == 1)) return;
+    // (pass 4, or 5 for packed input, alone does the work) or not (passes 1 and 3, or the plain packed launch 6, do);
+    // the other kind returns at once.
+    if (p.seg_pass == 6) {
+        if (p.seq_order[p.seg_G] != 0) return;
+    } else if (p.seg_pass != 0 && (p.seg_pass >= 4) != (p.cu_seqlens[p.n_seq + 1] == 1)) {
+        return;
+    }
+    if (p.seg_pass == 1) n = (n / (p.seg_G - 1)) * p.seg_G + n % (p.seg_G - 1);
+    else if ((p.seg_pass == 0 || p.seg_pass == 6) && p.seq_order) n = p.seq_order[n];   // packed input: longest sequences first
 
     int tok0, len;
     if (p.cu_seqlens) {
@@ -431,11 +436,20 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         tok0 = n * p.T;
         len = p.T;
     }
-    const size_t state_off = (((size_t)n * p.H + h) * D) * D + (size_t)sl * NS;
+    // packed input cut into pieces: the piece's sequence, and whether it is the first and the last piece of it
+    const int32_t piece = p.seg_pass == 5 ? p.cu_seqlens[p.n_seq + 2 + p.n_seq * p.H + n] : 0;
+    const int sq = p.seg_pass == 5 ? (piece & 0x1fffffff) : n;   // index of the states this CTA reads and writes
+    const size_t state_off = (((size_t)sq * p.H + h) * D) * D + (size_t)sl * NS;
     // the state before the first token (null: zero) and the number of leading chunks whose outputs are not stored
     const float *init = p.init_state;
     size_t init_off = state_off;
     int first_out = 0;
+    if (p.seg_pass == 5 && !((piece >> 29) & 1)) {   // not a sequence's first piece: from zero, so many chunks early
+        init = nullptr;
+        first_out = p.cu_seqlens[p.n_seq + 2 + n * p.H + h];
+        tok0 -= first_out * C;
+        len += first_out * C;
+    }
     if (p.seg_pass == 4) {
         if (n % p.seg_G == 0) {   // first segment: the sequence's own initial state
             init_off = (((size_t)(n / p.seg_G) * p.H + h) * D) * D + (size_t)sl * NS;
@@ -449,7 +463,9 @@ kla_chunk_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     // where this CTA's final state goes (null: nowhere)
     float *fin = is_map ? p.map_state : p.final_state;
     size_t fin_off = state_off;
-    if (p.seg_pass >= 3 && fin) {
+    if (p.seg_pass == 5) {
+        if (!((piece >> 30) & 1)) fin = nullptr;   // only a sequence's last piece holds its final state
+    } else if (p.seg_pass >= 3 && p.seg_pass <= 4 && fin) {
         if (n % p.seg_G != p.seg_G - 1) fin = nullptr;
         else fin_off = (((size_t)(n / p.seg_G) * p.H + h) * D) * D + (size_t)sl * NS;
     }

@@ -27,7 +27,11 @@ struct ChunkParams {
     //               final_state, at the sequence's index.
     //   seg_pass 4: every segment but a sequence's first from the zero state, started as many chunks early as the plan
     //               after the segment bounds says (outputs of those chunks are not stored); init_state is per sequence.
-    //   Passes 1 and 3 return at once when the plan word (cu_seqlens[n_seq + 1]) is 1, pass 4 when it is not.
+    //   seg_pass 5: packed input cut into pieces (launch_packed_units): cu_seqlens = the piece bounds, n_seq = the number of
+    //               pieces; the table after the warm-up lengths (cu_seqlens[n_seq + 2 + n_seq H + u]) names each piece's
+    //               sequence and says whether it is the first (initial state) and the last (final state) of it.
+    //   seg_pass 6: the plain packed launch, taken only if the pieces' plan word, seq_order[seg_G], is 0.
+    //   Passes 1 and 3 return at once when the plan word (cu_seqlens[n_seq + 1]) is 1, passes 4 and 5 when it is not.
     int32_t seg_pass, seg_G;
     int32_t variant;     // bit 0: beta_t = eta_t instead of Eq. 3; bit 1: read-out divided by ||q_t||; bit 2: test hook; bits 3, 4: see VARIANT_NO_PAIR, VARIANT_WY
     union {
@@ -73,6 +77,12 @@ cudaError_t launch_seg_warm_plan(int32_t *cu_seg, const float *log_alpha, const 
 // order[r] = index of the sequence with the r-th largest length (ties by index); n_seq small (quadratic work)
 cudaError_t launch_seq_order(const int32_t *cu_seqlens, int n_seq, int32_t *order, cudaStream_t stream);
 // start[b, 0] = init (or 0); start[b, g + 1] = map[b, g] . start[b, g] + local[b, g]   (d x d products, fp32)
+// Packed input cut into pieces of at most seg_len tokens (n_units of them, counted by the caller from the host copy of the
+// offsets): piece bounds ub[n_units + 1], plan word ub[n_units + 1] = 1, warm-up lengths from ub[n_units + 2] on (cleared
+// plan word if some piece has none), unit_seq[n_units]; final states of empty sequences.  Two launches.
+cudaError_t launch_packed_units(const int32_t *cu_seqlens, int n_seq, int seg_len, int n_units, int32_t *ub, int32_t *unit_seq,
+                                const float *log_alpha, const float *eta, long long n_tok, int H, const float *init_state,
+                                float *final_state, int d, cudaStream_t stream);
 // (`skip_if_one`: null, or a device word; the kernel does nothing when it holds 1)
 cudaError_t launch_seg_combine(const float *init_state, const float *map, const float *local, float *start, int B, int H,
                                int G, int d, const int32_t *skip_if_one, cudaStream_t stream);

@@ -41,7 +41,7 @@ __global__ void seg_bounds_kernel(int32_t *cu_seg, int B, int T, int G, int seg_
 // passes run instead.
 constexpr float WARM_LOG_DECAY = -40.f;
 __global__ void seg_warm_plan_kernel(int32_t *cu_seg, const float *log_alpha, const float *eta, int n_seg, int G, int H,
-                                     int max_warm, int plan_blocks, long long n_gate)
+                                     int max_warm, int plan_blocks, long long n_gate, const int32_t *unit_seq)
 {
     int32_t *plan = cu_seg + n_seg + 1, *warm = cu_seg + n_seg + 2;
     if ((int)blockIdx.x >= plan_blocks) {   // eta in [0, 2] everywhere (a NaN fails the test)
@@ -57,7 +57,8 @@ __global__ void seg_warm_plan_kernel(int32_t *cu_seg, const float *log_alpha, co
     const int unit = blockIdx.x * (blockDim.x / 32) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
     if (unit >= n_seg * H) return;
     const int n = unit / H, h = unit % H;
-    if (n % G == 0) {
+    // a sequence's first piece starts from the initial state: G equal segments per sequence, or (packed input) the table
+    if (unit_seq ? (unit_seq[n] >> 29) & 1 : n % G == 0) {
         if (lane == 0) warm[unit] = 0;
         return;
     }
@@ -75,6 +76,46 @@ __global__ void seg_warm_plan_kernel(int32_t *cu_seg, const float *log_alpha, co
     if (lane == 0) {
         warm[unit] = w;
         if (!(acc <= WARM_LOG_DECAY)) *plan = 0;   // (also when a gate is NaN)
+    }
+}
+
+// Packed input: every sequence longer than seg_len tokens is cut into pieces of seg_len (the last one shorter).  One block.
+//   ub[u], ub[u + 1]   token range of piece u (pieces tile the packed token axis; empty sequences have none)
+//   ub[n_units + 1]    plan word, set to 1 (seg_warm_plan_kernel may clear it)
+//   unit_seq[u]        sequence of piece u | first piece << 29 | last piece << 30
+// Empty sequences get their final state here (no piece will write it).
+constexpr int MAX_PACKED_SEQ = 4096;
+__global__ void __launch_bounds__(256) packed_units_kernel(const int32_t *cu_seqlens, int n_seq, int seg_len, int n_units,
+                                                           int32_t *ub, int32_t *unit_seq, const float *init_state,
+                                                           float *final_state, int state_elems)
+{
+    __shared__ int first_unit[MAX_PACKED_SEQ + 1];
+    for (int n = threadIdx.x; n < n_seq; n += blockDim.x) {
+        const int len = cu_seqlens[n + 1] - cu_seqlens[n];
+        first_unit[n + 1] = (len + seg_len - 1) / seg_len;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        first_unit[0] = 0;
+        for (int n = 0; n < n_seq; ++n) first_unit[n + 1] += first_unit[n];
+        ub[n_units] = cu_seqlens[n_seq];
+        ub[n_units + 1] = 1;
+    }
+    __syncthreads();
+    for (int n = threadIdx.x; n < n_seq; n += blockDim.x) {
+        const int t0 = cu_seqlens[n], t1 = cu_seqlens[n + 1], u0 = first_unit[n], cnt = first_unit[n + 1] - u0;
+        for (int g = 0; g < cnt; ++g) {
+            ub[u0 + g] = t0 + g * seg_len;
+            unit_seq[u0 + g] = n | (g == 0 ? 1 << 29 : 0) | (g == cnt - 1 ? 1 << 30 : 0);
+        }
+        (void)t1;
+    }
+    if (final_state) {
+        for (int n = 0; n < n_seq; ++n) {
+            if (cu_seqlens[n + 1] != cu_seqlens[n]) continue;
+            for (int i = threadIdx.x; i < state_elems; i += blockDim.x)
+                final_state[(size_t)n * state_elems + i] = init_state ? init_state[(size_t)n * state_elems + i] : 0.f;
+        }
     }
 }
 
@@ -169,8 +210,23 @@ cudaError_t launch_seg_warm_plan(int32_t *cu_seg, const float *log_alpha, const 
     const long long n_gate = (long long)B * T * H;
     const int eta_blocks = (int)((n_gate + 128 * 16 - 1) / (128 * 16) < 256 ? (n_gate + 128 * 16 - 1) / (128 * 16) : 256);
     const int max_warm = seg_len / 64 / 2 < 32 ? seg_len / 64 / 2 : 32;   // at most half a segment, and 2048 tokens
-    seg_warm_plan_kernel<<<plan_blocks + eta_blocks, 128, 0, stream>>>(cu_seg, log_alpha, eta, n_seg, G, H, max_warm, plan_blocks, n_gate);
+    seg_warm_plan_kernel<<<plan_blocks + eta_blocks, 128, 0, stream>>>(cu_seg, log_alpha, eta, n_seg, G, H, max_warm, plan_blocks, n_gate, nullptr);
     count_launch(1);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_packed_units(const int32_t *cu_seqlens, int n_seq, int seg_len, int n_units, int32_t *ub, int32_t *unit_seq,
+                                const float *log_alpha, const float *eta, long long n_tok, int H, const float *init_state,
+                                float *final_state, int d, cudaStream_t stream)
+{
+    if (n_seq > MAX_PACKED_SEQ) return cudaErrorInvalidValue;
+    packed_units_kernel<<<1, 256, 0, stream>>>(cu_seqlens, n_seq, seg_len, n_units, ub, unit_seq, init_state, final_state, H * d * d);
+    const int plan_blocks = (n_units * H + 3) / 4;
+    const long long n_gate = n_tok * H;
+    const int eta_blocks = (int)((n_gate + 128 * 16 - 1) / (128 * 16) < 256 ? (n_gate + 128 * 16 - 1) / (128 * 16) : 256);
+    const int max_warm = seg_len / 64 / 2 < 32 ? seg_len / 64 / 2 : 32;
+    seg_warm_plan_kernel<<<plan_blocks + eta_blocks, 128, 0, stream>>>(ub, log_alpha, eta, n_units, 1, H, max_warm, plan_blocks, n_gate, unit_seq);
+    count_launch(2);
     return cudaGetLastError();
 }
 

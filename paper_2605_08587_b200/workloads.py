@@ -146,3 +146,12 @@ def upstream_grads(w: ChunkWorkload, seed=6, final=True):
     H, d_k, d_v = w.q.shape[2], w.q.shape[3], w.v.shape[3]
     d_final = torch.randn((w.n_seq, H, d_k, d_v), generator=gen).float().contiguous() if final else None
     return d_out, d_final
+
+
+def config5_skewed(long_len=65536, n_short=31, max_short=2048, H=16, d=64, seed=7):
+    """A packed batch that one sequence dominates: one sequence of `long_len` tokens and `n_short` sequences with lengths
+    uniform in [1, max_short]; value distributions of config 5."""
+    lens = [long_len] + torch.randint(1, max_short + 1, (n_short,), generator=torch.Generator().manual_seed(seed + 1000)).tolist()
+    w = config5(H=H, d=d, seed=seed, lengths=lens)
+    w.name = "packed_skewed_1x%d_plus_%d_short_H%d_d%d" % (long_len, n_short, H, d)
+    return w

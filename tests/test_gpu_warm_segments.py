@@ -111,3 +111,78 @@ def test_long_context_workload_by_default_every_head():
     out, fin, word = _run(w, 0)
     assert word == 1
     _check(w, out, fin)
+
+
+# ---- packed input: long sequences cut into pieces that start from warm-up runs ------------------------------------------------
+def _skewed(lens, H=2, d=64, seed=960, init=True):
+    w = W.config5(H=H, d=d, lengths=lens, seed=seed)
+    w.log_alpha = (w.log_alpha * 12).contiguous()   # config 5 draws -softplus / 8 ... scaled so that exp(-40) needs ~4 chunks
+    if init:
+        w.init_state = (0.02 * torch.randn(len(lens), H, d, d, generator=torch.Generator().manual_seed(seed + 1))).float()
+    return w
+
+
+def _check_packed(w, out, fin):
+    ro, rf = oracle_chunk(w)[:2]
+    o = np64(out)[0]
+    assert rel_err(o, ro) <= TOL_BF16
+    assert rel_err(np64(fin), rf) <= TOL_BF16
+    cu = w.cu_seqlens.numpy()
+    for n in range(len(cu) - 1):   # no sequence hides behind the others
+        if cu[n + 1] > cu[n]:
+            assert rel_err(o[cu[n]:cu[n + 1]], ro[cu[n]:cu[n + 1]]) <= 5 * TOL_BF16
+
+
+@pytest.mark.parametrize("d", [64, 128])
+def test_one_long_sequence_among_short_ones_is_cut_by_default(d):
+    lens = [40, 20000 + 37, 0, 64, 130, 1]
+    w = _skewed(lens, d=d, seed=961)
+    out, fin, word = _run(w, 0)
+    assert word == 1            # the library decided to cut, and the decay allowed warm-up starts
+    _check_packed(w, out, fin)
+    assert torch.equal(fin[2].cpu(), w.init_state[2])   # the empty sequence keeps its state
+
+
+def test_forced_pieces_match_the_plain_launch_and_the_oracle():
+    lens = [3000, 700, 5000 + 11, 64, 0, 2048]
+    w = _skewed(lens, d=128, seed=962)
+    o_c, f_c, word = _run(w, KLA_FLAG_SEGMENTS(4))        # the longest sequence in four pieces; pieces of that length everywhere
+    o_p, f_p, none = _run(w, KLA_FLAG_NO_SEGMENTS)
+    assert word == 1 and none is None
+    _check_packed(w, o_c, f_c)
+    assert rel_err(np64(o_c), np64(o_p)) <= 2e-4 and rel_err(np64(f_c), np64(f_p)) <= 2e-4
+
+
+def test_packed_pieces_fall_back_to_the_plain_launch_on_weak_decay():
+    lens = [3000, 700, 5000 + 11, 64]
+    w = _skewed(lens, d=64, seed=963)
+    w.log_alpha = (w.log_alpha * 1e-3).contiguous()
+    out, fin, word = _run(w, KLA_FLAG_SEGMENTS(4))
+    assert word == 0
+    _check_packed(w, out, fin)
+    plain = gpu_chunk(w, flags=KLA_FLAG_NO_SEGMENTS)
+    assert torch.equal(out, plain[0]) and torch.equal(fin, plain[1])   # the fallback IS the plain launch
+
+
+def test_packed_pieces_without_initial_state_bf16_out():
+    lens = [9000, 100, 4100]
+    w = _skewed(lens, d=128, seed=964, init=False)
+    word = []
+    out, fin = gpu_chunk(w, out_dtype=torch.bfloat16, flags=KLA_FLAG_SEGMENTS(3), plan_word=word)
+    assert word[0] == 1
+    ro, rf = oracle_chunk(w)[:2]
+    assert_bf16_out_close(out[0], ro)
+    assert rel_err(np64(fin), rf) <= TOL_BF16
+
+
+def test_the_packed_benchmark_workload_is_not_cut():
+    # lengths uniform in [1, 8192]: the launch is bound by total work, no sequence stands out
+    from paper_2605_08587_b200 import binding
+    import ctypes
+    w = W.config5()
+    hs = w.cu_seqlens.contiguous()
+    desc = binding.KlaDesc(B=1, T=w.q.shape[1], H=16, d_k=64, d_v=64, n_seq=32, cu_seqlens=1 << 20, host_seqlens=hs.data_ptr(),
+                           io_dtype=binding.KLA_BF16, out_dtype=binding.KLA_BF16)
+    lib = binding.load()
+    assert lib.kla_chunk_fwd_plan_word_offset(ctypes.byref(desc), 64) == ctypes.c_size_t(-1).value
+    assert lib.kla_chunk_fwd_workspace_bytes(ctypes.byref(desc), 64) == 256   # the longest-first order array alone

@@ -84,7 +84,7 @@ typedef enum { KLA_F32 = 0, KLA_BF16 = 1 } kla_dtype;
  * taken in fp16 (11 significand bits), which holds the 2e-3 bound on layer-shaped inputs but not on inputs with
  * heavy-tailed key norms, and needs the state and W inside the fp16 range. */
 #define KLA_FLAG_WY_FORM 64
-/* Segment-parallel scan of the tensor-core path (fixed-length input only).  Every chunk step is affine in the
+/* Segment-parallel scan of the tensor-core path (the transition-map form: fixed-length input only).  Every chunk step is affine in the
  * incoming state (Eqs. 7-9), so a sequence can be cut into G segments whose transition maps are found in
  * parallel, chained, and the segments then run in parallel from their true start states: the same result up
  * to rounding, about three times the state work, G times the parallelism.  By default the library decides

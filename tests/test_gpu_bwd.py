@@ -142,3 +142,17 @@ def test_config2_full_size_every_sequence_and_head():
     w = W.config2()
     g, do, df = _gpu(w)
     _assert_close(g, _ref(w, do, df), TOL_BF16)
+
+
+def test_packed_benchmark_workload_full_size_every_sequence_and_head():
+    # 32 sequences of 1..8192 tokens, 16 heads, d = 64, heavy-tailed key norms with near-zero and zero keys
+    w = W.config5()
+    g, do, df = _gpu(w, cu=w.cu_seqlens)
+    _assert_close(g, _ref(w, do, df), TOL_BF16)
+
+
+def test_long_context_workload_full_size_every_head():
+    # one sequence of 65 536 tokens: 4096 kept states per head, gradients carried back through all of them
+    w = W.config3()
+    g, do, df = _gpu(w)
+    _assert_close(g, _ref(w, do, df), TOL_BF16)
